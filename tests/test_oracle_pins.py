@@ -1,0 +1,404 @@
+"""Pins for the CPU oracle: each check ties an oracle function to something the
+paper or the mathematics fixes independently of the oracle's own code (closed
+forms, library quantile functions, asymptotics on samples of a known law,
+brute force on tiny inputs, scripted adaptation sequences)."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.special as sps
+import scipy.stats as sst
+
+from oracle import sidco_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "closed_forms.txt")
+
+
+def golden():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            out[line[0]] = float(line[1])
+    return out
+
+
+def rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def laplace_acc(n, b, seed):
+    return rng(seed).laplace(0.0, b, n).astype(np.float32)
+
+
+# ------------------------------------------------------------------ stage ratios
+
+def test_stage_cap_values():
+    # largest M with 0.25^(M-1) > delta
+    assert O.stage_cap(0.1, 0.25) == 2
+    assert O.stage_cap(0.01, 0.25) == 4
+    assert O.stage_cap(0.001, 0.25) == 5
+    assert O.stage_cap(0.25, 0.25) == 1
+    assert O.stage_cap(0.5, 0.25) == 1
+
+
+@pytest.mark.parametrize("delta", [0.1, 0.01, 0.001, 3e-4])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5])
+def test_stage_ratios_product_is_delta(delta, M):
+    M = min(M, O.stage_cap(delta, 0.25))
+    r = O.stage_ratios(delta, M, 0.25)
+    assert len(r) == M
+    assert all(0.0 < x < 1.0 for x in r)
+    assert math.prod(r) == pytest.approx(delta, rel=1e-14)
+    assert all(x == 0.25 for x in r[:-1])
+
+
+# ------------------------------------------------------------------ exponential
+
+def test_exp_closed_form_golden():
+    g = golden()
+    assert O.exp_quantile_step(1e-3, 0.01) == pytest.approx(g["exp_eta_b1e-3_delta0.01"], rel=1e-14)
+    assert O.exp_quantile_step(1e-3, 0.25) == pytest.approx(g["exp_eta1_b1e-3_delta0.25"], rel=1e-14)
+    assert O.exp_quantile_step(1e-3, 0.04) == pytest.approx(g["exp_inc_b1e-3_delta0.04"], rel=1e-14)
+
+
+def test_exp_threshold_is_library_quantile():
+    # eta must be the (1-delta) quantile of Exp(scale = mean): library ppf.
+    for mean, delta in [(0.3, 0.1), (2e-4, 0.001)]:
+        assert O.exp_quantile_step(mean, delta) == pytest.approx(
+            sst.expon(scale=mean).ppf(1.0 - delta), rel=1e-10)
+
+
+def test_config1_single_stage_converges_to_b_log_inv_delta():
+    g = golden()
+    x = laplace_acc(262144, 1e-3, 0)
+    res = O.sidco_compress(x, np.zeros_like(x), [0, x.size], 0.01, O.SID_EXP, -1)
+    eta = res.report[0].eta[-1]
+    # estimator std of the mean of n exponentials is b/sqrt(n)
+    assert eta == pytest.approx(g["exp_eta_b1e-3_delta0.01"], rel=5 / math.sqrt(x.size))
+    k = 0.01 * x.size
+    assert abs(int(res.out_k[0]) - k) <= 5 * (50.9 + 23.6)
+
+
+def test_config1_two_stage_memoryless():
+    g = golden()
+    x = laplace_acc(262144, 1e-3, 0)
+    res = O.sidco_compress(x, np.zeros_like(x), [0, x.size], 0.01, O.SID_EXP, -2)
+    rep = res.report[0]
+    assert rep.M_used == 2
+    assert rep.eta[0] == pytest.approx(g["exp_eta1_b1e-3_delta0.25"], rel=5 / math.sqrt(x.size))
+    assert abs(rep.k_stage[0] - 65536) <= 5 * math.sqrt(x.size * 0.25 * 0.75) + 0.01 * 65536
+    # the increment is fitted on ~65k exceedances
+    assert rep.eta[1] - rep.eta[0] == pytest.approx(g["exp_inc_b1e-3_delta0.04"], rel=5 / math.sqrt(65536))
+    assert rep.eta[1] == pytest.approx(g["exp_eta_b1e-3_delta0.01"], rel=0.02)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4])
+def test_exp_multistage_hits_target_ratio_on_exponential_data(M):
+    # memorylessness: on Laplace data every stage count gives k/n -> delta
+    n, delta = 400000, 0.01
+    x = laplace_acc(n, 3e-2, 11)
+    res = O.sidco_compress(x, np.zeros_like(x), [0, n], delta, O.SID_EXP, -M)
+    k = delta * n
+    assert abs(int(res.out_k[0]) - k) < 6 * math.sqrt(k) + 0.03 * k
+
+
+# ------------------------------------------------------------------ GPD
+
+def test_gpd_threshold_closed_form_golden_and_library():
+    g = golden()
+    a, b, delta = 0.2, 1.0, 0.01
+    # population moments of GP(shape a, scale b)
+    mean = b / (1 - a)
+    var = b * b / ((1 - a) ** 2 * (1 - 2 * a))
+    eta, deg = O.gpd_quantile_step(mean, var, delta)
+    assert not deg
+    assert eta == pytest.approx(g["gpd_eta_a0.2_b1_delta0.01"], rel=1e-12)
+    assert eta == pytest.approx(sst.genpareto(c=a, scale=b).ppf(1 - delta), rel=1e-10)
+
+
+@pytest.mark.parametrize("a,b", [(0.2, 1.0), (-0.2, 3.0), (0.05, 1e-3), (0.35, 0.1)])
+@pytest.mark.parametrize("delta", [0.25, 0.01])
+def test_gpd_moment_match_inverts_population_moments(a, b, delta):
+    dist = sst.genpareto(c=a, scale=b)
+    eta, _ = O.gpd_quantile_step(dist.mean(), dist.var(), delta)
+    assert eta == pytest.approx(dist.ppf(1 - delta), rel=1e-9)
+
+
+def test_gpd_alpha_to_zero_is_exponential():
+    mean = 0.7
+    eta, _ = O.gpd_quantile_step(mean, mean * mean, 0.01)      # R = 1 -> alpha = 0
+    assert eta == pytest.approx(O.exp_quantile_step(mean, 0.01), rel=1e-12)
+    eta2, _ = O.gpd_quantile_step(mean, mean * mean * (1 + 1e-9), 0.01)
+    assert eta2 == pytest.approx(eta, rel=1e-7)
+
+
+def test_gpd_zero_variance_is_limit_of_formula():
+    mean = 2.5
+    lim, deg = O.gpd_quantile_step(mean, 0.0, 0.01)
+    assert deg and lim == mean
+    near, _ = O.gpd_quantile_step(mean, mean * mean * 1e-9, 0.01)
+    assert near == pytest.approx(lim, rel=1e-8)
+
+
+def gp_sample(n, a, b, seed):
+    u = rng(seed).random(n)
+    x = (b / a) * np.expm1(-a * np.log1p(-u))          # inverse CDF of the paper's GPD
+    sign = np.where(rng(seed + 1).random(n) < 0.5, -1.0, 1.0)
+    return (sign * x).astype(np.float32)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3])
+def test_gpd_on_gp_data_hits_target_ratio(M):
+    # threshold stability of the GP family: every stage count should select ~delta*n
+    n, delta = 1000000, 0.01
+    x = gp_sample(n, 0.2, 1e-2, 5)
+    res = O.sidco_compress(x, np.zeros_like(x), [0, n], delta, O.SID_GPD, -M)
+    k = delta * n
+    assert abs(int(res.out_k[0]) - k) < 6 * math.sqrt(k) + 0.10 * k
+    eta = res.report[0].eta
+    assert all(eta[i] < eta[i + 1] for i in range(len(eta) - 1))
+    assert eta[-1] == pytest.approx(sst.genpareto(c=0.2, scale=1e-2).ppf(1 - delta), rel=0.06)
+
+
+def test_gpd_on_exponential_data_matches_exp():
+    n = 1000000
+    x = laplace_acc(n, 1e-2, 6)
+    r_g = O.sidco_compress(x, np.zeros_like(x), [0, n], 0.01, O.SID_GPD, -1).report[0]
+    r_e = O.sidco_compress(x, np.zeros_like(x), [0, n], 0.01, O.SID_EXP, -1).report[0]
+    assert r_g.eta[0] == pytest.approx(r_e.eta[0], rel=0.02)
+
+
+# ------------------------------------------------------------------ gamma
+
+@pytest.mark.parametrize("s", [1e-3, 0.05, 0.5772156649015329, 2.0, 9.0])
+def test_gamma_shape_is_root_of_quadratic(s):
+    al = O.gamma_shape(s)
+    assert al > 0
+    assert abs(6 * s * al * al - (3 - s) * al - 1) < 1e-10 * max(1.0, al * al * s)
+
+
+def test_gamma_shape_at_euler_gamma_golden():
+    assert O.gamma_shape(0.5772156649015329) == pytest.approx(
+        golden()["gamma_shape_at_euler_gamma"], abs=5e-7)
+
+
+@pytest.mark.parametrize("alpha,bias", [(0.2, -0.010), (0.4, -0.014), (0.6, -0.013), (1.0, -0.009), (2.0, -0.004)])
+def test_gamma_shape_population_bias(alpha, bias):
+    s = math.log(alpha) - sps.digamma(alpha)       # population value of log(mean) - mean(log)
+    assert O.gamma_shape(s) / alpha - 1 == pytest.approx(bias, abs=1.5e-3)
+
+
+def gamma_sample(n, alpha, theta, seed):
+    r = rng(seed)
+    return (np.where(r.random(n) < 0.5, -1.0, 1.0) * r.gamma(alpha, theta, n)).astype(np.float32)
+
+
+def test_gamma_first_stage_matches_formula_with_library_pieces():
+    n, alpha, theta, delta = 500000, 0.6, 2e-3, 0.01
+    x = gamma_sample(n, alpha, theta, 9)
+    a = np.abs(x).astype(np.float64)
+    eta, deg = O.gamma_first_stage(a, delta)
+    assert not deg
+    # fitted shape near the population bias for alpha = 0.6 and scale consistent with it
+    s = math.log(a.mean()) - np.log(a).mean()
+    al = O.gamma_shape(s)
+    assert al / alpha - 1 == pytest.approx(-0.013, abs=0.01)
+    assert eta == pytest.approx(-(a.mean() / al) * (math.log(delta) + sps.gammaln(al)), rel=1e-12)
+
+
+@pytest.mark.parametrize("alpha", [0.3, 0.6, 0.9, 1.0])
+@pytest.mark.parametrize("delta", [0.01, 0.001])
+def test_gamma_closed_form_upper_bounds_exact_quantile(alpha, delta):
+    # Corollary 1.2: -[log delta + log Gamma(alpha)] >= P^-1(alpha, 1-delta) for alpha <= 1
+    # whenever the exact quantile is >= 1, with equality at alpha = 1.
+    exact = sps.gammaincinv(alpha, 1.0 - delta)
+    assert exact >= 1.0
+    closed = -(math.log(delta) + math.lgamma(alpha))
+    assert closed >= exact * (1 - 1e-12)
+    if alpha == 1.0:
+        assert closed == pytest.approx(exact, rel=1e-10)
+
+
+def test_gamma_on_exponential_data_close_to_exp_threshold():
+    # exponential magnitudes are Gamma(1): shape -> 0.9909, threshold within a few % of b*ln(1/delta)
+    n = 1000000
+    x = laplace_acc(n, 1e-2, 12)
+    rep = O.sidco_compress(x, np.zeros_like(x), [0, n], 0.01, O.SID_GAMMA, -1).report[0]
+    assert rep.eta[0] == pytest.approx(1e-2 * math.log(100), rel=0.03)
+
+
+def test_gamma_ignores_zeros_and_rescales_tail():
+    # half the entries zero: the fit sees only nonzeros; tail prob becomes 2*delta among them
+    n = 400000
+    x = gamma_sample(n, 0.9, 1e-2, 21)
+    z = np.concatenate([x, np.zeros(n, np.float32)])
+    e_full, _ = O.gamma_first_stage(np.abs(z).astype(np.float64), 0.01)
+    e_half, _ = O.gamma_first_stage(np.abs(x).astype(np.float64), 0.02)
+    assert e_full == pytest.approx(e_half, rel=1e-12)
+
+
+def test_gamma_clamp_and_constant_rules():
+    # delta * Gamma(alpha_hat) >= 1 -> clamp to 0
+    x = gamma_sample(200000, 0.05, 1.0, 3)
+    eta, deg = O.gamma_first_stage(np.abs(x).astype(np.float64), 0.25)
+    assert deg and eta == 0.0
+    # constant magnitudes -> exponential formula
+    c = np.full(1000, 0.125)
+    eta, deg = O.gamma_first_stage(c, 0.01)
+    assert deg and eta == pytest.approx(0.125 * math.log(100), rel=1e-12)
+
+
+# ------------------------------------------------------------------ selection, residual, brute force
+
+def brute_force_count(acc, eta):
+    srt = sorted((abs(float(v)) for v in acc), reverse=True)
+    c = 0
+    for v in srt:
+        if v >= eta:
+            c += 1
+        else:
+            break
+    return c
+
+
+@pytest.mark.parametrize("n", [1, 3, 31, 32, 33, 64, 1000])
+@pytest.mark.parametrize("sid", [O.SID_EXP, O.SID_GAMMA, O.SID_GPD])
+@pytest.mark.parametrize("M", [1, 2, 3])
+def test_selection_brute_force_tiny(n, sid, M):
+    g = laplace_acc(n, 1e-2, 100 + n)
+    r = laplace_acc(n, 3e-3, 200 + n)
+    res = O.sidco_compress(g, r, [0, n], 0.1, sid, -M)
+    acc = (g + r).astype(np.float32)
+    assert np.array_equal(res.acc, acc)
+    eta = res.report[0].eta[-1]
+    assert int(res.out_k[0]) == brute_force_count(acc, eta) == res.idx.size
+    assert np.all(np.diff(res.idx) > 0)
+    assert np.array_equal(res.val, acc[res.idx])
+    # residual + scatter(idx, val) == acc bit for bit, residual exactly zero on idx
+    rebuilt = res.residual.copy()
+    rebuilt[res.idx] += res.val
+    assert np.array_equal(rebuilt, acc)
+    assert np.all(res.residual[res.idx] == 0)
+    mask = np.ones(n, bool)
+    mask[res.idx] = False
+    assert np.array_equal(res.residual[mask].view(np.uint32), acc[mask].view(np.uint32))
+    # stage thresholds never decrease
+    e = res.report[0].eta
+    assert all(e[i] <= e[i + 1] for i in range(len(e) - 1))
+
+
+def test_exceedance_counts_brute_force_each_stage():
+    n = 500
+    g = laplace_acc(n, 1.0, 77)
+    res = O.sidco_compress(g, np.zeros_like(g), [0, n], 0.01, O.SID_GPD, -3)
+    rep = res.report[0]
+    mags = [abs(float(v)) for v in g]
+    for m in range(rep.M_used - 1):
+        assert rep.k_stage[m] == sum(1 for v in mags if v > rep.eta[m])
+    assert rep.k_stage[-1] == sum(1 for v in mags if v >= rep.eta[-1])
+
+
+def test_intermediate_exceedance_is_strict():
+    # gamma first stage clamps to eta_1 = 0 here; the stage-2 exceedance set is |x| > 0
+    # (strict, as in the stage loop of Algorithm 1), so exact zeros must not enter the refit
+    x = np.concatenate([gamma_sample(200000, 0.05, 1.0, 3), np.zeros(1000, np.float32)])
+    res = O.sidco_compress(x, np.zeros_like(x), [0, x.size], 0.1, O.SID_GAMMA, -2)
+    rep = res.report[0]
+    assert rep.eta[0] == 0.0
+    assert rep.k_stage[0] == sum(1 for v in x if v != 0.0)
+
+
+def test_two_stage_exp_hand_example():
+    # |x| = 1..8, delta = 0.125, delta_1 = 0.25: eta_1 = 4.5 ln 4 = 6.238..;
+    # exceedances {7, 8}: mean shift = 7.5 - eta_1; delta_2 = 0.5
+    x = np.array([1, -2, 3, -4, 5, -6, 7, -8], dtype=np.float32)
+    res = O.sidco_compress(x, np.zeros_like(x), [0, 8], 0.125, O.SID_EXP, -2)
+    eta1 = 4.5 * math.log(4.0)
+    eta2 = eta1 + (7.5 - eta1) * math.log(2.0)
+    assert res.report[0].eta[0] == pytest.approx(eta1, rel=1e-14)
+    assert res.report[0].eta[1] == pytest.approx(eta2, rel=1e-14)
+    assert res.report[0].k_stage == [2, 1]
+    assert list(res.idx) == [7] and list(res.val) == [-8.0]
+
+
+def test_binomial_achieved_ratio_per_segment():
+    # k_hat ~ Binomial(n, delta) (+ estimator error) when the family is right
+    sizes = [50000, 120000, 80000]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    r = rng(31)
+    g = np.concatenate([r.laplace(0, b, n) for b, n in zip([1e-4, 1e-2, 1.0], sizes)]).astype(np.float32)
+    res = O.sidco_compress(g, np.zeros_like(g), off, 0.01, O.SID_EXP, -1)
+    for s, n in enumerate(sizes):
+        k = 0.01 * n
+        assert abs(int(res.out_k[s]) - k) < 5 * math.sqrt(k) + 5 * k * math.log(100) / math.sqrt(n)
+    assert int(res.out_k[-1]) == res.idx.size == int(res.out_k[:-1].sum())
+    # indices are segment-major ascending and fall in their segment
+    bounds = np.cumsum(res.out_k[:-1])
+    for s in range(3):
+        part = res.idx[(bounds[s] - res.out_k[s]):bounds[s]]
+        assert np.all((part >= off[s]) & (part < off[s + 1]))
+
+
+def test_degenerate_segments():
+    sizes = [0, 5, 7, 1, 6]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    g = np.zeros(19, np.float32)
+    g[5:12] = 0.5 * np.array([1, -1, 1, -1, 1, -1, 1], np.float32)   # constant magnitude
+    g[12] = 3.0                                                     # single element
+    g[13:19] = [1, 2, np.nan, 4, 5, 6]                              # NaN segment
+    for sid in (O.SID_EXP, O.SID_GAMMA, O.SID_GPD):
+        res = O.sidco_compress(g, np.zeros_like(g), off, 0.1, sid, -2)
+        assert res.out_k[0] == 0
+        assert res.out_k[1] == 0 and res.report[1].status & O.ST_ALL_ZERO
+        assert math.isinf(res.report[1].eta[-1])
+        assert res.out_k[4] == 0 and res.report[4].status & O.ST_NONFINITE
+    res = O.sidco_compress(g, np.zeros_like(g), off, 0.1, O.SID_GPD, -1)
+    # zero variance -> eta = mean -> ties at the threshold are all selected (>=)
+    assert res.report[2].eta[0] == 0.5 and res.out_k[2] == 7
+    assert res.report[3].eta[0] == 3.0 and res.out_k[3] == 1
+
+
+# ------------------------------------------------------------------ adaptation
+
+def test_adapt_stages_transition_table():
+    k, eH, eL = 100.0, 0.2, 0.2
+    assert O.adapt_stages(2, 121.0, k, eH, eL, 4) == 1      # too many -> fewer stages
+    assert O.adapt_stages(2, 79.0, k, eH, eL, 4) == 3       # too few -> more stages
+    assert O.adapt_stages(2, 120.0, k, eH, eL, 4) == 2      # boundary values stay
+    assert O.adapt_stages(2, 80.0, k, eH, eL, 4) == 2
+    assert O.adapt_stages(1, 500.0, k, eH, eL, 4) == 1      # clamped below
+    assert O.adapt_stages(4, 1.0, k, eH, eL, 4) == 4        # clamped above
+
+
+def test_adapt_update_scripted_sequence():
+    p = O.Params()
+    st = O.SegState()
+    k = 100.0
+    history = []
+    script = [50] * 5 + [100] * 5 + [300] * 5 + [50, 50, 50, 50, 350]
+    for kh in script:
+        O.adapt_update(st, kh, k, p, 3)
+        history.append(st.M)
+    # changes only at calls 5, 10, 15, 20 and by at most one
+    assert history[:4] == [1] * 4 and history[4] == 2
+    assert history[5:10] == [2] * 5                      # mean 100 within tolerance
+    assert history[10:14] == [2] * 4 and history[14] == 1
+    assert history[19] == 1                              # mean 110 within tolerance
+    assert st.k_sum == 0 and st.calls == 20
+
+
+def test_adaptive_compress_moves_M_on_misfit_data():
+    # Gamma(0.6) magnitudes with the gamma SID under-select at delta = 0.001 -> M grows
+    n = 300000
+    state = O.new_state(1)
+    used = []
+    for call in range(10):
+        g = gamma_sample(n, 0.6, 1e-3, 500 + call)
+        res = O.sidco_compress(g, np.zeros_like(g), [0, n], 0.001, O.SID_GAMMA, 4, state=state)
+        used.append(res.report[0].M_used)
+    assert used[:5] == [1] * 5
+    assert used[5] == 2
+    assert all(1 <= m <= 4 for m in used)
+    assert all(abs(used[i + 1] - used[i]) <= 1 for i in range(9))
