@@ -1,0 +1,157 @@
+/*
+ * sidco.h - C ABI of the B200 (sm_100a) SIDCo gradient sparsifier.
+ *
+ * The library implements one call of the paper's compressor (Algorithm 1,
+ * function Sparsify, wrapped in error compensation) over a flattened model
+ * gradient that is split into contiguous segments (layers).  Every step runs
+ * in CUDA kernels of this library; there is no CPU fallback.
+ *
+ * Conventions
+ *   - "device" pointers refer to memory of the CUDA device that is current
+ *     when the function is called; "host" pointers are ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Functions return 0 on success, a negative SIDCO_E_* code for an argument
+ *     error found on the host before anything was enqueued, or a positive
+ *     cudaError_t value if a CUDA runtime call failed.
+ *   - Device-side conditions never trap.  They set bits in a per-segment status
+ *     word that sidco_get_debug() returns (SIDCO_ST_*).
+ *   - The caller owns every buffer it passes in.  The library owns, per
+ *     `residual` pointer (the persistent identity of one model's error
+ *     compensation memory): the tile table derived from `seg_offsets`, a
+ *     scratch workspace (sidco_workspace_bytes) and the stage-adaptation state.
+ *   - One call per `residual` may be in flight at a time; calls for different
+ *     `residual` pointers are independent.
+ */
+#ifndef SIDCO_H_
+#define SIDCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Sparsity-inducing distribution of the first stage and the family of the
+ * later stages (Section 2.4, paragraph after Corollary 2.1):
+ * exponential -> exponential, gamma -> generalised Pareto, GPD -> GPD. */
+#define SIDCO_SID_EXP   0
+#define SIDCO_SID_GAMMA 1
+#define SIDCO_SID_GPD   2
+
+#define SIDCO_MAX_STAGES 8      /* hard upper limit on |max_stages| */
+
+/* argument errors (returned before any work is enqueued) */
+#define SIDCO_E_NULL        (-1)   /* a required pointer is NULL */
+#define SIDCO_E_SEGMENTS    (-2)   /* n_segs < 1, offsets[0] != 0, offsets decreasing, or d too large */
+#define SIDCO_E_DELTA       (-3)   /* delta not in (0, 1) */
+#define SIDCO_E_SID         (-4)   /* unknown sid_type */
+#define SIDCO_E_STAGES      (-5)   /* max_stages == 0 or |max_stages| > SIDCO_MAX_STAGES */
+#define SIDCO_E_PARAMS      (-6)   /* sidco_set_params: value out of range */
+#define SIDCO_E_UNKNOWN_KEY (-7)   /* no state exists for this residual pointer */
+#define SIDCO_E_WORKSPACE   (-8)   /* caller-provided workspace too small or misaligned */
+#define SIDCO_E_ALIAS       (-9)   /* grad and residual overlap */
+#define SIDCO_E_SIZE        (-10)  /* size beyond the limit of this entry point */
+
+/* per-segment status bits */
+#define SIDCO_ST_NONFINITE  1   /* a magnitude was NaN/Inf: nothing is selected in the segment */
+#define SIDCO_ST_DEGENERATE 2   /* a fit took one of its degenerate-case rules */
+#define SIDCO_ST_ALL_ZERO   4   /* every magnitude is zero: nothing is selected */
+#define SIDCO_ST_TIMEOUT    8   /* a bounded wait inside the kernel ran out; results are invalid */
+
+typedef struct sidco_seg_debug {
+    int32_t M_used;                       /* stages used by the last call (after the cap for delta) */
+    int32_t M_next;                       /* stage count the next adaptive call starts from */
+    int32_t status;                       /* SIDCO_ST_* bits of the last call */
+    int32_t calls;                        /* adaptive calls seen so far */
+    int64_t k_sum;                        /* sum of k_hat since the last adaptation point */
+    double  eta[SIDCO_MAX_STAGES];        /* eta_1 .. eta_{M_used} */
+    int32_t k_stage[SIDCO_MAX_STAGES];    /* #{|x| > eta_m} for m < M_used, #{|x| >= eta_M} for the last */
+} sidco_seg_debug;
+
+/*
+ * sidco_compress - one iteration of the sparsifier on device buffers.
+ *
+ * Computes, for every segment s = [seg_offsets[s], seg_offsets[s+1]) independently:
+ *   1. error compensation  acc_j = grad_j + residual_j                    (one fp32 add; appendix on
+ *      gradient distributions, memory-based compression);
+ *   2. the threshold eta_M by multi-stage fitting (Section 2.4, Lemma 2, Corollary 2.1) with the first
+ *      stage from Corollary 1.1 (EXP), 1.2 (GAMMA) or 1.3 (GPD); the first-stage ratio is delta_1 (0.25 by
+ *      default), every non-final stage keeps delta_1 and the last stage takes delta / delta_1^(M-1);
+ *   3. threshold sparsification (Section 2.3): K = { j : |acc_j| >= eta_M };
+ *   4. residual_j <- +0.0f for j in K and acc_j otherwise;
+ *   5. if max_stages > 0, stage adaptation (Algorithm 1, Adapt_Stages) every Q calls.
+ *
+ * grad        device, float[d], read only, d = seg_offsets[n_segs].
+ * residual    device, float[d], in/out.  Must not overlap grad.
+ * seg_offsets HOST, int64[n_segs + 1], seg_offsets[0] = 0, non-decreasing (empty segments allowed),
+ *             d <= 2^31 - 2^16.  Read during the call only.
+ * n_segs      >= 1.
+ * delta       target ratio k/d, 0 < delta < 1 (the float value is used as is, widened to double).
+ * sid_type    SIDCO_SID_*.
+ * max_stages  > 0: adaptive, M starts at 1 and moves within [1, max_stages];
+ *             < 0: fixed M = -max_stages, no adaptation.  M is additionally capped so that the last
+ *             stage's ratio stays below one.
+ * out_idx     device, int32, capacity >= d.  Flat indices of the survivors, strictly ascending.
+ * out_val     device, float, capacity >= d.  out_val[t] = acc[out_idx[t]], bit exact.
+ * out_k       device, int32[n_segs + 1].  out_k[s] = survivors of segment s, out_k[n_segs] = total;
+ *             segment s occupies positions [sum_{t<s} out_k[t], +out_k[s]) of out_idx/out_val.
+ * stream      all device work is enqueued here; the call does not synchronise, except that the first
+ *             call for a residual pointer (or for a new segment table) allocates and uploads tables.
+ *
+ * 16-byte aligned grad and residual take the vectorised path; other alignments are handled with scalar
+ * accesses.
+ */
+int sidco_compress(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs,
+                   float delta, int sid_type, int max_stages,
+                   int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
+
+/*
+ * sidco_compress_host - the same operation with HOST buffers (pinned memory gives full copy speed).
+ * Copies grad and residual to device staging buffers owned by the library, runs sidco_compress,
+ * copies residual, out_k and the first out_k[n_segs] entries of out_idx/out_val back, and
+ * synchronises `stream` before returning.  State is keyed by the host `residual` pointer.
+ * out_idx/out_val need capacity >= d on the host as well.
+ */
+int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs,
+                        float delta, int sid_type, int max_stages,
+                        int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
+
+/* Bytes of device scratch one residual key needs for a vector of d elements in n_segs segments. */
+size_t sidco_workspace_bytes(int64_t d, int n_segs);
+
+/* Optional: let the library use caller-owned device memory (256-byte aligned, at least
+ * sidco_workspace_bytes) as the workspace of `residual` instead of allocating its own.  Must be called
+ * before the first sidco_compress for that residual; the memory must outlive the state. */
+int sidco_set_workspace(const float* residual, void* device_ptr, size_t bytes);
+
+/* Constants of Algorithm 1 for subsequent calls (defaults: the paper's experimental settings,
+ * delta_1 = 0.25, eps_H = eps_L = 0.2, Q = 5).  0 < delta1 < 1, 0 <= eps < 1, Q >= 1. */
+int sidco_set_params(double delta1, double eps_H, double eps_L, int Q);
+
+/* Forget the adaptation state of `residual` (M back to 1, counters to 0).  Synchronises the device. */
+int sidco_reset_state(const float* residual);
+
+/* Copy per-segment thresholds, counts, stage counts and status of the last call to host memory
+ * (`out` has room for n_segs entries).  Synchronises the device; meant for tests and logging. */
+int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);
+
+/* Checkpointing of the adaptation state (Algorithm 1 keeps M and the running k_hat sum across
+ * iterations): host blobs of 3 int64 per segment (M, calls, k_sum).  Both synchronise the device. */
+int sidco_state_save(const float* residual, int64_t* host_blob, int n_segs);
+int sidco_state_load(const float* residual, const int64_t* host_blob, int n_segs);
+
+/* Free everything the library holds for `residual` / for all keys.  Synchronises the device. */
+int sidco_release(const float* residual);
+int sidco_release_all(void);
+
+/* Number of kernel launches the library has enqueued since it was loaded. */
+int64_t sidco_launch_count(void);
+
+const char* sidco_error_string(int code);
+int sidco_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SIDCO_H_ */

@@ -1,0 +1,208 @@
+"""ctypes binding of libsidco.so: argument marshalling only.
+
+Every function has the name and the meaning of the C entry point declared in
+``include/sidco.h``; tensors are passed as raw device (or host) pointers and
+nothing is computed here.  Loading fails loudly if the library has not been
+built (``python -m paper_2101_10761_b200.build``): there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsidco.so")
+
+SID_EXP, SID_GAMMA, SID_GPD = 0, 1, 2
+MAX_STAGES = 8
+
+ST_NONFINITE, ST_DEGENERATE, ST_ALL_ZERO, ST_TIMEOUT = 1, 2, 4, 8
+
+
+class SegDebug(C.Structure):
+    _fields_ = [
+        ("M_used", C.c_int32),
+        ("M_next", C.c_int32),
+        ("status", C.c_int32),
+        ("calls", C.c_int32),
+        ("k_sum", C.c_int64),
+        ("eta", C.c_double * MAX_STAGES),
+        ("k_stage", C.c_int32 * MAX_STAGES),
+    ]
+
+
+EXPORTS = [
+    "sidco_compress", "sidco_compress_host", "sidco_workspace_bytes", "sidco_set_workspace",
+    "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
+    "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
+]
+
+_lib = None
+
+
+class SidcoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().sidco_error_string(code).decode()
+        super().__init__(f"{where} failed with code {code}: {msg}")
+
+
+def lib() -> C.CDLL:
+    """Load libsidco.so once.  Raises if it is missing: the CUDA path is the only path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2101_10761_b200.build` "
+            "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, f32, i64, dbl = C.c_void_p, C.c_int, C.c_float, C.c_int64, C.c_double
+    compress_sig = [vp, vp, C.POINTER(i64), i32, f32, i32, i32, vp, vp, vp, vp]
+    L.sidco_compress.argtypes = compress_sig
+    L.sidco_compress.restype = i32
+    L.sidco_compress_host.argtypes = compress_sig
+    L.sidco_compress_host.restype = i32
+    L.sidco_workspace_bytes.argtypes = [i64, i32]
+    L.sidco_workspace_bytes.restype = C.c_size_t
+    L.sidco_set_workspace.argtypes = [vp, vp, C.c_size_t]
+    L.sidco_set_workspace.restype = i32
+    L.sidco_set_params.argtypes = [dbl, dbl, dbl, i32]
+    L.sidco_set_params.restype = i32
+    L.sidco_reset_state.argtypes = [vp]
+    L.sidco_reset_state.restype = i32
+    L.sidco_get_debug.argtypes = [vp, C.POINTER(SegDebug), i32]
+    L.sidco_get_debug.restype = i32
+    L.sidco_state_save.argtypes = [vp, C.POINTER(i64), i32]
+    L.sidco_state_save.restype = i32
+    L.sidco_state_load.argtypes = [vp, C.POINTER(i64), i32]
+    L.sidco_state_load.restype = i32
+    L.sidco_release.argtypes = [vp]
+    L.sidco_release.restype = i32
+    L.sidco_release_all.argtypes = []
+    L.sidco_release_all.restype = i32
+    L.sidco_launch_count.argtypes = []
+    L.sidco_launch_count.restype = i64
+    L.sidco_error_string.argtypes = [i32]
+    L.sidco_error_string.restype = C.c_char_p
+    L.sidco_version.argtypes = []
+    L.sidco_version.restype = i32
+    _lib = L
+    return L
+
+
+def _ptr(x) -> Optional[int]:
+    """Raw address of a torch tensor, a numpy array or an int; None stays NULL."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()
+
+
+def _offsets(seg_offsets: Sequence[int]):
+    arr = np.ascontiguousarray(np.asarray(seg_offsets, dtype=np.int64))
+    return arr, arr.ctypes.data_as(C.POINTER(C.c_int64)), int(arr.size - 1)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def sidco_compress(grad, residual, seg_offsets, delta: float, sid_type: int, max_stages: int,
+                   out_idx, out_val, out_k, stream=None) -> None:
+    """Device buffers (torch CUDA tensors or raw addresses); enqueues on `stream`
+    (default: torch's current stream) and returns without synchronising."""
+    arr, p, n = _offsets(seg_offsets)
+    rc = lib().sidco_compress(_ptr(grad), _ptr(residual), p, n, delta, sid_type, max_stages,
+                              _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_compress")
+
+
+def sidco_compress_host(grad, residual, seg_offsets, delta: float, sid_type: int, max_stages: int,
+                        out_idx, out_val, out_k, stream=None) -> None:
+    """Host buffers (numpy arrays or pinned torch CPU tensors); copies in, compresses,
+    copies back and synchronises."""
+    arr, p, n = _offsets(seg_offsets)
+    rc = lib().sidco_compress_host(_ptr(grad), _ptr(residual), p, n, delta, sid_type, max_stages,
+                                   _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_compress_host")
+
+
+def sidco_workspace_bytes(d: int, n_segs: int) -> int:
+    return int(lib().sidco_workspace_bytes(d, n_segs))
+
+
+def sidco_set_workspace(residual, device_ptr, nbytes: int) -> None:
+    rc = lib().sidco_set_workspace(_ptr(residual), _ptr(device_ptr), nbytes)
+    if rc:
+        raise SidcoError(rc, "sidco_set_workspace")
+
+
+def sidco_set_params(delta1: float = 0.25, eps_H: float = 0.2, eps_L: float = 0.2, Q: int = 5) -> None:
+    rc = lib().sidco_set_params(delta1, eps_H, eps_L, Q)
+    if rc:
+        raise SidcoError(rc, "sidco_set_params")
+
+
+def sidco_reset_state(residual) -> None:
+    rc = lib().sidco_reset_state(_ptr(residual))
+    if rc:
+        raise SidcoError(rc, "sidco_reset_state")
+
+
+def sidco_get_debug(residual, n_segs: int):
+    buf = (SegDebug * n_segs)()
+    rc = lib().sidco_get_debug(_ptr(residual), buf, n_segs)
+    if rc:
+        raise SidcoError(rc, "sidco_get_debug")
+    return list(buf)
+
+
+def sidco_state_save(residual, n_segs: int) -> np.ndarray:
+    blob = np.zeros(3 * n_segs, dtype=np.int64)
+    rc = lib().sidco_state_save(_ptr(residual), blob.ctypes.data_as(C.POINTER(C.c_int64)), n_segs)
+    if rc:
+        raise SidcoError(rc, "sidco_state_save")
+    return blob
+
+
+def sidco_state_load(residual, blob: np.ndarray) -> None:
+    blob = np.ascontiguousarray(blob, dtype=np.int64)
+    rc = lib().sidco_state_load(_ptr(residual), blob.ctypes.data_as(C.POINTER(C.c_int64)), blob.size // 3)
+    if rc:
+        raise SidcoError(rc, "sidco_state_load")
+
+
+def sidco_release(residual) -> None:
+    rc = lib().sidco_release(_ptr(residual))
+    if rc:
+        raise SidcoError(rc, "sidco_release")
+
+
+def sidco_release_all() -> None:
+    lib().sidco_release_all()
+
+
+def sidco_launch_count() -> int:
+    return int(lib().sidco_launch_count())
+
+
+def sidco_version() -> int:
+    return int(lib().sidco_version())
+
+
+def sidco_error_string(code: int) -> str:
+    return lib().sidco_error_string(code).decode()

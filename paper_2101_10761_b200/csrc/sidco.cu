@@ -1,0 +1,547 @@
+// Host side of the SIDCo sparsifier library: argument checks, tile tables, workspace,
+// per-residual state, and the cooperative launch of the persistent kernel.
+#include "sidco_kernel.cuh"
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/sidco.h"
+
+namespace {
+
+using sidco::Args;
+using sidco::Control;
+using sidco::SegDev;
+using sidco::kThreads;
+using sidco::kTile;
+
+struct Params {
+    double delta1 = 0.25, eps_H = 0.2, eps_L = 0.2;
+    int Q = 5;
+};
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int ctas_per_sm = 0;     // min over the kernel instantiations
+    bool ready = false;
+};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Offsets of the workspace parts for (d, S, T, G).
+struct Layout {
+    size_t tile_start, tile_seg, seg_tile0, seg_n, cta_tile0;
+    size_t part, part_n, side_cnt, tile_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, seg, ctl;
+    size_t total;
+};
+
+Layout make_layout(int64_t d, int S, int64_t T, int G) {
+    Layout L{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+    L.tile_start = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.tile_seg = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.seg_tile0 = take(sizeof(int32_t) * (size_t)(S + 1));
+    L.seg_n = take(sizeof(int32_t) * (size_t)(S + 1));
+    L.cta_tile0 = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.part = take(sizeof(double) * 3 * (size_t)(T + 1));
+    L.part_n = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.side_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.tile_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.side_idx = take(sizeof(int32_t) * (size_t)(d + 4));
+    L.side_val = take(sizeof(float) * (size_t)(d + 4));
+    L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
+    L.stage_val = take(sizeof(float) * (size_t)(d + 4));
+    L.cta_total = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
+    L.ctl = take(sizeof(Control));
+    L.total = o;
+    return L;
+}
+
+// Upper bound on the tile count: every window and every segment start opens at most one tile.
+int64_t max_tiles(int64_t d, int S) { return (d + kTile - 1) / kTile + S + 1; }
+
+constexpr int kMaxGrid = 148 * 8 * 2;   // generous bound used only for sizing sidco_workspace_bytes
+
+struct Context {
+    int device = -1;
+    int64_t d = 0;
+    int S = 0, T = 0, G = 0;
+    std::vector<int64_t> offsets;          // segment table the device tables were built from
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    bool ws_owned = false;
+    bool tables_valid = false;
+    Layout L{};
+    // staging for sidco_compress_host
+    float* h_grad = nullptr; float* h_res = nullptr;
+    int32_t* h_idx = nullptr; float* h_val = nullptr; int32_t* h_k = nullptr;
+    int64_t staging_d = -1; int staging_S = -1;
+};
+
+std::mutex g_mu;
+Params g_params;
+std::unordered_map<const void*, Context*> g_ctx;
+std::unordered_map<int, DeviceInfo> g_dev;
+std::atomic<int64_t> g_launches{0};
+
+template <int SID>
+cudaError_t occupancy(int* out) {
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sidco::sidco_persistent_kernel<SID>, kThreads, 0);
+}
+
+cudaError_t device_info(int dev, DeviceInfo** out) {
+    DeviceInfo& di = g_dev[dev];
+    if (!di.ready) {
+        cudaDeviceProp prop;
+        cudaError_t e = cudaGetDeviceProperties(&prop, dev);
+        if (e != cudaSuccess) return e;
+        if (!prop.cooperativeLaunch) return cudaErrorNotSupported;
+        int a = 0, b = 0, c = 0;
+        if ((e = occupancy<0>(&a)) != cudaSuccess) return e;
+        if ((e = occupancy<1>(&b)) != cudaSuccess) return e;
+        if ((e = occupancy<2>(&c)) != cudaSuccess) return e;
+        int occ = a < b ? a : b;
+        occ = occ < c ? occ : c;
+        if (occ < 1) return cudaErrorLaunchOutOfResources;
+        if (const char* env = getenv("SIDCO_CTAS_PER_SM")) {
+            int want = atoi(env);
+            if (want >= 1 && want < occ) occ = want;
+        }
+        di.sm_count = prop.multiProcessorCount;
+        di.ctas_per_sm = occ;
+        di.ready = true;
+    }
+    *out = &di;
+    return cudaSuccess;
+}
+
+void free_context(Context* c) {
+    if (c->ws_owned && c->ws) cudaFree(c->ws);
+    if (c->h_grad) cudaFree(c->h_grad);
+    if (c->h_res) cudaFree(c->h_res);
+    if (c->h_idx) cudaFree(c->h_idx);
+    if (c->h_val) cudaFree(c->h_val);
+    if (c->h_k) cudaFree(c->h_k);
+    delete c;
+}
+
+int check_args(const void* grad, const void* residual, const int64_t* off, int n_segs, float delta, int sid,
+               int max_stages, const void* out_idx, const void* out_val, const void* out_k) {
+    if (!grad || !residual || !off || !out_idx || !out_val || !out_k) return SIDCO_E_NULL;
+    if (n_segs < 1 || off[0] != 0) return SIDCO_E_SEGMENTS;
+    for (int s = 0; s < n_segs; ++s)
+        if (off[s + 1] < off[s]) return SIDCO_E_SEGMENTS;
+    if (off[n_segs] > (int64_t)2147483647 - 65536) return SIDCO_E_SEGMENTS;
+    if (!(delta > 0.0f && delta < 1.0f)) return SIDCO_E_DELTA;
+    if (sid < 0 || sid > 2) return SIDCO_E_SID;
+    if (max_stages == 0 || max_stages > SIDCO_MAX_STAGES || max_stages < -SIDCO_MAX_STAGES) return SIDCO_E_STAGES;
+    return 0;
+}
+
+// Build the tile tables for a segment table and upload them together with fresh per-segment state.
+// keep_state: the adaptation state of an existing context survives a change of nothing but the tables.
+cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t stream) {
+    const int64_t d = off[S];
+    DeviceInfo* di = nullptr;
+    cudaError_t e = device_info(c->device, &di);
+    if (e != cudaSuccess) return e;
+    const int G = di->sm_count * di->ctas_per_sm;
+
+    std::vector<int32_t> tile_start, tile_seg, seg_tile0(S + 1), seg_n(S + 1, 0);
+    for (int s = 0; s < S; ++s) {
+        seg_tile0[s] = (int32_t)tile_start.size();
+        seg_n[s] = (int32_t)(off[s + 1] - off[s]);
+        int64_t at = off[s];
+        while (at < off[s + 1]) {
+            int64_t end = (at / kTile + 1) * kTile;
+            if (end > off[s + 1]) end = off[s + 1];
+            tile_start.push_back((int32_t)at);
+            tile_seg.push_back(s);
+            at = end;
+        }
+    }
+    const int T = (int)tile_start.size();
+    seg_tile0[S] = T;
+    tile_start.push_back((int32_t)d);
+    tile_seg.push_back(0);
+
+    // Static partition of the tiles over the CTAs, balanced by elements plus a per-tile overhead.
+    std::vector<int32_t> cta_tile0(G + 1, T);
+    {
+        const double per_tile = 1024.0;
+        double total = 0.0;
+        for (int t = 0; t < T; ++t) total += (tile_start[t + 1] - tile_start[t]) + per_tile;
+        double acc = 0.0;
+        int cta = 0;
+        cta_tile0[0] = 0;
+        for (int t = 0; t < T; ++t) {
+            // tile t goes to the CTA whose share contains the tile's midpoint
+            const double w = (tile_start[t + 1] - tile_start[t]) + per_tile;
+            const double mid = acc + 0.5 * w;
+            int want = (int)(mid / total * G);
+            if (want > G - 1) want = G - 1;
+            while (cta < want) cta_tile0[++cta] = t;
+            acc += w;
+        }
+        while (cta < G) cta_tile0[++cta] = T;
+    }
+
+    const Layout L = make_layout(d, S, T, G);
+    if (c->ws && c->ws_bytes < L.total) {
+        if (!c->ws_owned) return cudaErrorMemoryAllocation;
+        cudaFree(c->ws);
+        c->ws = nullptr;
+    }
+    bool fresh = false;
+    if (!c->ws) {
+        if ((e = cudaMalloc(&c->ws, L.total)) != cudaSuccess) return e;
+        c->ws_bytes = L.total;
+        c->ws_owned = true;
+        fresh = true;
+    }
+    const bool same_segments = c->tables_valid && c->S == S;
+    // keep adaptation state across a table rebuild only when the segment count is unchanged
+    std::vector<SegDev> seg_host(S + 1);
+    if (same_segments && !fresh) {
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
+        if ((e = cudaMemcpy(seg_host.data(), (char*)c->ws + c->L.seg, sizeof(SegDev) * S, cudaMemcpyDeviceToHost)) !=
+            cudaSuccess)
+            return e;
+        for (auto& sg : seg_host) sg.arrived = 0;
+    } else {
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
+        for (auto& sg : seg_host) {
+            std::memset(&sg, 0, sizeof(SegDev));
+            sg.M = 1;
+        }
+    }
+    char* base = (char*)c->ws;
+    auto up = [&](size_t at, const void* src, size_t bytes) {
+        return cudaMemcpy(base + at, src, bytes, cudaMemcpyHostToDevice);
+    };
+    if ((e = up(L.tile_start, tile_start.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = up(L.tile_seg, tile_seg.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg_tile0, seg_tile0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg_n, seg_n.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = up(L.cta_tile0, cta_tile0.data(), sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.tile_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+
+    c->L = L;
+    c->d = d;
+    c->S = S;
+    c->T = T;
+    c->G = G;
+    c->offsets.assign(off, off + S + 1);
+    c->tables_valid = true;
+    return cudaSuccess;
+}
+
+int compress_impl(Context* c, const float* grad, float* residual, const int64_t* off, int S, float delta, int sid,
+                  int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
+                  const Params& prm) {
+    cudaError_t e;
+    const bool same = c->tables_valid && c->S == S &&
+                      std::memcmp(c->offsets.data(), off, sizeof(int64_t) * (S + 1)) == 0;
+    if (!same) {
+        if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
+    }
+    char* base = (char*)c->ws;
+    const Layout& L = c->L;
+    Args a{};
+    a.grad = grad;
+    a.residual = residual;
+    a.out_idx = out_idx;
+    a.out_val = out_val;
+    a.out_k = out_k;
+    a.tile_start = (const int32_t*)(base + L.tile_start);
+    a.tile_seg = (const int32_t*)(base + L.tile_seg);
+    a.seg_tile0 = (const int32_t*)(base + L.seg_tile0);
+    a.seg_n = (const int32_t*)(base + L.seg_n);
+    a.cta_tile0 = (const int32_t*)(base + L.cta_tile0);
+    a.part = (double*)(base + L.part);
+    a.part_n = (int32_t*)(base + L.part_n);
+    a.side_cnt = (int32_t*)(base + L.side_cnt);
+    a.tile_cnt = (int32_t*)(base + L.tile_cnt);
+    a.side_idx = (int32_t*)(base + L.side_idx);
+    a.side_val = (float*)(base + L.side_val);
+    a.stage_idx = (int32_t*)(base + L.stage_idx);
+    a.stage_val = (float*)(base + L.stage_val);
+    a.cta_total = (int32_t*)(base + L.cta_total);
+    a.seg = (SegDev*)(base + L.seg);
+    a.ctl = (Control*)(base + L.ctl);
+    a.delta = (double)delta;
+    a.delta1 = prm.delta1;
+    a.eps_H = prm.eps_H;
+    a.eps_L = prm.eps_L;
+    a.Q = prm.Q;
+    a.sid = sid;
+    a.max_stages = max_stages;
+    a.T = c->T;
+    a.S = c->S;
+    a.G = c->G;
+    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
+
+    void* kargs[] = {(void*)&a};
+    const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
+                     : sid == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
+                                : (const void*)sidco::sidco_persistent_kernel<2>;
+    e = cudaLaunchCooperativeKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
+    if (e != cudaSuccess) return (int)e;
+    g_launches.fetch_add(1);
+    return 0;
+}
+
+Context* find_or_create(const void* key, int dev) {
+    auto it = g_ctx.find(key);
+    if (it != g_ctx.end()) {
+        if (it->second->device == dev) return it->second;
+        free_context(it->second);
+        g_ctx.erase(it);
+    }
+    Context* c = new Context();
+    c->device = dev;
+    g_ctx[key] = c;
+    return c;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sidco_compress(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
+                   int sid_type, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, void* stream) {
+    int rc = check_args(grad, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k);
+    if (rc) return rc;
+    const int64_t d = seg_offsets[n_segs];
+    if ((grad < residual + d) && (residual < grad + d) && d > 0) return SIDCO_E_ALIAS;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = find_or_create(residual, dev);
+    return compress_impl(c, grad, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k,
+                         (cudaStream_t)stream, g_params);
+}
+
+int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
+                        int sid_type, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k,
+                        void* stream_v) {
+    int rc = check_args(grad, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k);
+    if (rc) return rc;
+    const int64_t d = seg_offsets[n_segs];
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = find_or_create(residual, dev);
+    if (c->staging_d != d || c->staging_S != n_segs) {
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
+        if (c->h_grad) { cudaFree(c->h_grad); cudaFree(c->h_res); cudaFree(c->h_idx); cudaFree(c->h_val); cudaFree(c->h_k); }
+        c->h_grad = c->h_res = c->h_val = nullptr; c->h_idx = c->h_k = nullptr;
+        const size_t n = (size_t)d + 4;
+        if ((e = cudaMalloc(&c->h_grad, n * 4)) != cudaSuccess) return (int)e;
+        if ((e = cudaMalloc(&c->h_res, n * 4)) != cudaSuccess) return (int)e;
+        if ((e = cudaMalloc(&c->h_idx, n * 4)) != cudaSuccess) return (int)e;
+        if ((e = cudaMalloc(&c->h_val, n * 4)) != cudaSuccess) return (int)e;
+        if ((e = cudaMalloc(&c->h_k, sizeof(int32_t) * (size_t)(n_segs + 1))) != cudaSuccess) return (int)e;
+        c->staging_d = d;
+        c->staging_S = n_segs;
+    }
+    const size_t bytes = (size_t)d * 4;
+    if ((e = cudaMemcpyAsync(c->h_grad, grad, bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return (int)e;
+    if ((e = cudaMemcpyAsync(c->h_res, residual, bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return (int)e;
+    rc = compress_impl(c, c->h_grad, c->h_res, seg_offsets, n_segs, delta, sid_type, max_stages, c->h_idx, c->h_val,
+                       c->h_k, stream, g_params);
+    if (rc) return rc;
+    if ((e = cudaMemcpyAsync(out_k, c->h_k, sizeof(int32_t) * (size_t)(n_segs + 1), cudaMemcpyDeviceToHost, stream)) !=
+        cudaSuccess)
+        return (int)e;
+    if ((e = cudaMemcpyAsync(residual, c->h_res, bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return (int)e;
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
+    const size_t kb = (size_t)out_k[n_segs] * 4;
+    if (kb) {
+        if ((e = cudaMemcpyAsync(out_idx, c->h_idx, kb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaMemcpyAsync(out_val, c->h_val, kb, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
+    }
+    return 0;
+}
+
+size_t sidco_workspace_bytes(int64_t d, int n_segs) {
+    if (d < 0 || n_segs < 1) return 0;
+    return make_layout(d, n_segs, max_tiles(d, n_segs), kMaxGrid).total;
+}
+
+int sidco_set_workspace(const float* residual, void* device_ptr, size_t bytes) {
+    if (!residual || !device_ptr) return SIDCO_E_NULL;
+    if (((uintptr_t)device_ptr & (kAlign - 1)) != 0) return SIDCO_E_WORKSPACE;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = find_or_create(residual, dev);
+    if (c->tables_valid) return SIDCO_E_WORKSPACE;      // too late: a workspace is already in use
+    c->ws = device_ptr;
+    c->ws_bytes = bytes;
+    c->ws_owned = false;
+    return 0;
+}
+
+int sidco_set_params(double delta1, double eps_H, double eps_L, int Q) {
+    if (!(delta1 > 0.0 && delta1 < 1.0) || !(eps_H >= 0.0 && eps_H < 1.0) || !(eps_L >= 0.0 && eps_L < 1.0) || Q < 1)
+        return SIDCO_E_PARAMS;
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_params.delta1 = delta1;
+    g_params.eps_H = eps_H;
+    g_params.eps_L = eps_L;
+    g_params.Q = Q;
+    return 0;
+}
+
+static int with_segments(const float* residual, int n_segs, Context** out) {
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    if (n_segs != it->second->S) return SIDCO_E_SEGMENTS;
+    *out = it->second;
+    return 0;
+}
+
+int sidco_reset_state(const float* residual) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    Context* c = it->second;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    std::vector<SegDev> seg(c->S + 1);
+    for (auto& sg : seg) { std::memset(&sg, 0, sizeof(SegDev)); sg.M = 1; }
+    char* base = (char*)c->ws;
+    if ((e = cudaMemcpy(base + c->L.seg, seg.data(), sizeof(SegDev) * (c->S + 1), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return (int)e;
+    if ((e = cudaMemset(base + c->L.ctl, 0, sizeof(Control))) != cudaSuccess) return (int)e;
+    return 0;
+}
+
+int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs) {
+    if (!out) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = nullptr;
+    int rc = with_segments(residual, n_segs, &c);
+    if (rc) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    std::vector<SegDev> seg(c->S);
+    Control ctl;
+    char* base = (char*)c->ws;
+    if ((e = cudaMemcpy(seg.data(), base + c->L.seg, sizeof(SegDev) * c->S, cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return (int)e;
+    if ((e = cudaMemcpy(&ctl, base + c->L.ctl, sizeof(Control), cudaMemcpyDeviceToHost)) != cudaSuccess) return (int)e;
+    for (int s = 0; s < c->S; ++s) {
+        out[s].M_used = seg[s].M_eff;
+        out[s].M_next = seg[s].M;
+        out[s].status = seg[s].status | (ctl.timeout ? SIDCO_ST_TIMEOUT : 0);
+        out[s].calls = seg[s].calls;
+        out[s].k_sum = seg[s].k_sum;
+        for (int m = 0; m < SIDCO_MAX_STAGES; ++m) {
+            out[s].eta[m] = seg[s].eta[m];
+            out[s].k_stage[m] = seg[s].k_stage[m];
+        }
+    }
+    return 0;
+}
+
+int sidco_state_save(const float* residual, int64_t* blob, int n_segs) {
+    if (!blob) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = nullptr;
+    int rc = with_segments(residual, n_segs, &c);
+    if (rc) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    std::vector<SegDev> seg(c->S);
+    if ((e = cudaMemcpy(seg.data(), (char*)c->ws + c->L.seg, sizeof(SegDev) * c->S, cudaMemcpyDeviceToHost)) !=
+        cudaSuccess)
+        return (int)e;
+    for (int s = 0; s < c->S; ++s) {
+        blob[3 * s + 0] = seg[s].M;
+        blob[3 * s + 1] = seg[s].calls;
+        blob[3 * s + 2] = seg[s].k_sum;
+    }
+    return 0;
+}
+
+int sidco_state_load(const float* residual, const int64_t* blob, int n_segs) {
+    if (!blob) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = nullptr;
+    int rc = with_segments(residual, n_segs, &c);
+    if (rc) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    std::vector<SegDev> seg(c->S);
+    char* at = (char*)c->ws + c->L.seg;
+    if ((e = cudaMemcpy(seg.data(), at, sizeof(SegDev) * c->S, cudaMemcpyDeviceToHost)) != cudaSuccess) return (int)e;
+    for (int s = 0; s < c->S; ++s) {
+        if (blob[3 * s] < 1 || blob[3 * s] > SIDCO_MAX_STAGES || blob[3 * s + 1] < 0 || blob[3 * s + 2] < 0)
+            return SIDCO_E_PARAMS;
+        seg[s].M = (int32_t)blob[3 * s + 0];
+        seg[s].calls = (int32_t)blob[3 * s + 1];
+        seg[s].k_sum = blob[3 * s + 2];
+    }
+    if ((e = cudaMemcpy(at, seg.data(), sizeof(SegDev) * c->S, cudaMemcpyHostToDevice)) != cudaSuccess) return (int)e;
+    return 0;
+}
+
+int sidco_release(const float* residual) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end()) return SIDCO_E_UNKNOWN_KEY;
+    cudaDeviceSynchronize();
+    free_context(it->second);
+    g_ctx.erase(it);
+    return 0;
+}
+
+int sidco_release_all(void) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_ctx.empty()) cudaDeviceSynchronize();
+    for (auto& kv : g_ctx) free_context(kv.second);
+    g_ctx.clear();
+    return 0;
+}
+
+int64_t sidco_launch_count(void) { return g_launches.load(); }
+
+const char* sidco_error_string(int code) {
+    switch (code) {
+        case 0: return "success";
+        case SIDCO_E_NULL: return "a required pointer is NULL";
+        case SIDCO_E_SEGMENTS: return "bad segment table (n_segs < 1, offsets[0] != 0, decreasing, or d too large)";
+        case SIDCO_E_DELTA: return "delta must lie in (0, 1)";
+        case SIDCO_E_SID: return "unknown sid_type";
+        case SIDCO_E_STAGES: return "max_stages must be non-zero and at most SIDCO_MAX_STAGES in magnitude";
+        case SIDCO_E_PARAMS: return "parameter out of range";
+        case SIDCO_E_UNKNOWN_KEY: return "no state for this residual pointer";
+        case SIDCO_E_WORKSPACE: return "workspace too small, misaligned, or set too late";
+        case SIDCO_E_ALIAS: return "grad and residual overlap";
+        case SIDCO_E_SIZE: return "size beyond the limit of this entry point";
+        default: break;
+    }
+    if (code > 0) return cudaGetErrorString((cudaError_t)code);
+    return "unknown error";
+}
+
+int sidco_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,180 @@
+"""GPU-vs-oracle parity through the C ABI on the five benchmark configurations
+and on edge cases.  Tolerances: thresholds within 1e-6 relative; indices
+identical except inside the 1e-6*eta band; values and residual bit exact."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import sidco_oracle as O
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, check_parity, f32
+
+pytestmark = pytest.mark.gpu
+
+SIDS = [O.SID_EXP, O.SID_GAMMA, O.SID_GPD]
+
+
+def run_sequence(wl_offsets, grads, delta, sid, max_stages, residual0=None, base_shift=0, check_status=True):
+    """Feed the same gradients to both sides, carrying each side's own residual."""
+    delta = f32(delta)
+    off = np.asarray(wl_offsets, dtype=np.int64)
+    d = int(off[-1])
+    run = GpuRun(off, residual0, base_shift)
+    res_o = np.zeros(d, np.float32) if residual0 is None else np.asarray(residual0, np.float32).copy()
+    state = O.new_state(off.size - 1) if max_stages > 0 else None
+    bands = 0
+    try:
+        for g in grads:
+            ora = O.sidco_compress(g, res_o, off, delta, sid, max_stages, state=state)
+            gpu = run.step(g, delta, sid, max_stages)
+            b = check_parity(gpu, ora, off, state, check_status)
+            bands += b
+            # after a tolerated tie at the threshold both sides continue from the GPU's residual
+            res_o = gpu["residual"] if b else ora.residual
+    finally:
+        run.close()
+    return bands
+
+
+# ------------------------------------------------------------------ config 1
+
+@pytest.mark.parametrize("M", [1, 2])
+def test_config1_laplace(M):
+    wl = W.config(1)
+    run_sequence(wl.seg_offsets, [wl.draw(0)], 0.01, O.SID_EXP, -M)
+
+
+# ------------------------------------------------------------------ config 2
+
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("delta", [0.1, 0.01, 0.001])
+@pytest.mark.parametrize("max_stages", [-1, 4])
+def test_config2_resnet20_shaped(sid, delta, max_stages):
+    wl = W.config(2)
+    # nonzero residual: what one prior (oracle) step leaves behind
+    prior = O.sidco_compress(wl.draw(0), np.zeros(wl.d, np.float32), wl.seg_offsets, f32(delta), sid, -1)
+    run_sequence(wl.seg_offsets, [wl.draw(1)], delta, sid, max_stages, residual0=prior.residual)
+
+
+@pytest.mark.parametrize("sid", SIDS)
+def test_config2_adaptive_many_calls(sid):
+    wl = W.config(2)
+    run_sequence(wl.seg_offsets, [wl.draw(c) for c in range(12)], 0.001, sid, 4)
+
+
+# ------------------------------------------------------------------ config 3
+
+@pytest.mark.parametrize("max_stages", [-3, 3])
+def test_config3_vgg16_shaped(max_stages):
+    wl = W.config(3)
+    n = 1 if max_stages < 0 else 11
+    run_sequence(wl.seg_offsets, [wl.draw(c) for c in range(n)], 0.001, O.SID_GPD, max_stages)
+
+
+# ------------------------------------------------------------------ config 4 (full size, bench launch configuration)
+
+@pytest.fixture(scope="module")
+def config4_draws():
+    wl = W.config(4)
+    return wl, [wl.draw(c) for c in range(10)]
+
+
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("delta", [0.01, 0.001])
+def test_config4_resnet50_shaped_ten_calls(config4_draws, sid, delta):
+    wl, draws = config4_draws
+    run_sequence(wl.seg_offsets, draws, delta, sid, 4)
+
+
+# ------------------------------------------------------------------ config 5
+
+def test_config5_lstm_shaped_adaptive():
+    wl = W.config(5)
+    grads = (wl.draw(c) for c in range(11))
+    run_sequence(wl.seg_offsets, grads, 0.001, O.SID_EXP, 4)
+
+
+# ------------------------------------------------------------------ edge cases
+
+@pytest.mark.parametrize("n", [0, 1, 3, 31, 32, 33, 64, 1000, 8191, 8192, 8193, 20000])
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("M", [1, 3])
+def test_single_segment_sizes(n, sid, M):
+    g = W.ragged_case(50 + n, [n], 1e-2)
+    r = W.ragged_case(90 + n, [n], 3e-3)
+    run_sequence([0, n], [g], 0.1, sid, -M, residual0=r)
+
+
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("base_shift", [0, 1, 2, 3])
+def test_unaligned_offsets_and_pointers(sid, base_shift):
+    # offsets congruent to 1, 2, 3 (mod 4), empty segments, segments crossing tile windows
+    sizes = [5, 0, 8190, 3, 0, 9001, 2, 16385, 1, 777, 0]
+    off = W.offsets_from_sizes(sizes)
+    g = [W.ragged_case(300 + c, sizes, 1e-3) for c in range(6)]
+    run_sequence(off, g, 0.01, sid, 3, base_shift=base_shift)
+
+
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("M", [1, 2, 3])
+def test_degenerate_segments(sid, M):
+    sizes = [0, 5000, 7000, 1, 6, 3000]
+    off = W.offsets_from_sizes(sizes)
+    g = W.ragged_case(7, sizes, 1.0)
+    g[off[1]:off[2]] = 0.0                                             # all-zero segment
+    g[off[2]:off[3]] = 0.5 * np.where(np.arange(7000) % 2 == 0, 1, -1)  # constant magnitude
+    g[off[3]] = 3.0                                                    # single element
+    # last segment: half exact zeros
+    seg = g[off[5]:off[6]]
+    seg[::2] = 0.0
+    run_sequence(off, [g], 0.05, sid, -M)
+
+
+@pytest.mark.parametrize("sid", SIDS)
+def test_nan_and_inf_segments_select_nothing(sid):
+    import torch
+    from paper_2101_10761_b200 import binding as B
+    sizes = [4000, 4000, 4000]
+    off = W.offsets_from_sizes(sizes)
+    g = W.ragged_case(8, sizes, 1.0)
+    g[4100] = np.nan
+    g[8100] = np.inf
+    run = GpuRun(off)
+    try:
+        out = run.step(g, f32(0.05), sid, -2)
+    finally:
+        run.close()
+    ora = O.sidco_compress(g, np.zeros_like(g), off, f32(0.05), sid, -2)
+    assert out["out_k"][1] == 0 and out["out_k"][2] == 0
+    assert out["debug"][1].status & B.ST_NONFINITE and out["debug"][2].status & B.ST_NONFINITE
+    assert math.isnan(out["debug"][1].eta[1]) and math.isnan(out["debug"][2].eta[1])
+    assert np.array_equal(out["out_k"], ora.out_k)
+    assert np.array_equal(out["idx"], ora.idx)
+    assert np.array_equal(out["residual"], ora.residual, equal_nan=True)
+
+
+def test_thresholds_independent_of_grid_size():
+    """Deterministic two-level combine: the same input gives bit-identical thresholds whatever the
+    number of CTAs (checked by running in a child process with fewer CTAs per SM)."""
+    import json
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import json, sys, numpy as np, torch
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, f32
+wl = W.config(3)
+run = GpuRun(wl.seg_offsets)
+out = run.step(wl.draw(0), f32(0.001), 1, -3)
+print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [out["idx"][:50].tolist(), int(out["out_k"][-1])]))
+''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for ctas in ("1", "3", "8"):
+        env = dict(os.environ, SIDCO_CTAS_PER_SM=ctas)
+        r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        outs.append(json.loads(r.stdout.strip().splitlines()[-1]))
+    assert outs[0] == outs[1] == outs[2]
