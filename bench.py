@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the SIDCo compress hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one `sidco_compress` call (the whole hot path: error compensation,
+statistics, fits, multi-stage refits, ordered compaction, residual write-back,
+stage adaptation) on the ResNet-50-shaped synthetic gradient (d = 25,557,032,
+161 segments, delta = 1e-3), residual carried from step to step, gradients
+rotating over four distinct draws so that no input is L2-resident.
+
+Prints ONE JSON line.  `value` is GB/s on the minimal bytes the method must move
+(12 d + 8 k_hat per step), inputs resident in HBM; `e2e` is the same metric
+through `sidco_compress_host` with pinned host buffers (copies inside the timed
+region).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SIDCo compress GB/s on minimal bytes (12 d + 8 k_hat) at d=25.6M, delta=1e-3"
+UNIT = "GB/s"
+DELTA = float(np.float32(1e-3))
+SID_NAMES = {0: "EXP", 1: "GAMMA", 2: "GPD"}
+N_GRADS = 4
+
+# DRAM bytes per launch of the persistent kernel on this workload, from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML (read only) while a region is open."""
+
+    def __init__(self, index: int, uuid=None, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []          # (region, sm_mhz, reasons)
+        self.region = None
+        self._stop = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = None
+            if uuid is not None:
+                for cand in (uuid, "GPU-" + uuid):
+                    try:
+                        self.h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode())
+                        break
+                    except Exception:
+                        continue
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as exc:  # pragma: no cover - depends on the box
+            self.err = repr(exc)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._stop.is_set():
+            if self.region is not None:
+                try:
+                    mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                    try:
+                        reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    except Exception:
+                        reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                    self.samples.append((self.region, mhz, reasons))
+                except Exception:
+                    pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop.set()
+
+    def summary(self):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"]}
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+            getattr(nv, "nvmlClocksThrottleReasonApplicationsClocksSetting", 0x2): "applications_clocks",
+        }
+        timed = [s for s in self.samples if s[0] == "device"]
+        src = "timed region"
+        if len(timed) < 3:
+            timed = list(self.samples)
+            src = "timed region + e2e region (timed region too short for 3 samples)"
+        if not timed:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        seen = set()
+        for _, _, r in timed:
+            for bit, name in names.items():
+                if bit and (r & bit):
+                    seen.add(name)
+        return {"sm_mhz": statistics.median(s[1] for s in timed), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(seen), "samples": len(timed), "sampled": src}
+
+
+def make_inputs():
+    from paper_2101_10761_b200 import workloads as W
+    wl = W.config(4)
+    grads = [wl.draw(c) for c in range(N_GRADS)]
+    return wl, grads
+
+
+def oracle_rate(wl, grads, budget_s: float, sid: int):
+    """Time the oracle as it stands on whole calls of the workload for about budget_s."""
+    from oracle import sidco_oracle as O
+    res = np.zeros(wl.d, np.float32)
+    state = O.new_state(wl.n_segs)
+    t0 = time.perf_counter()
+    calls, bytes_min = 0, 0
+    while True:
+        out = O.sidco_compress(grads[calls % N_GRADS], res, wl.seg_offsets, DELTA, sid, 4, state=state)
+        res = out.residual
+        bytes_min += 12 * wl.d + 8 * int(out.out_k[-1])
+        calls += 1
+        if time.perf_counter() - t0 > budget_s or calls >= 64:
+            break
+    dt = time.perf_counter() - t0
+    return bytes_min / dt / 1e9, calls, dt
+
+
+def used_threads() -> int:
+    # the oracle's numpy calls (sum, abs, compare, log, nonzero) run on the calling thread only
+    return 1
+
+
+def run_reference(args):
+    """The oracle on the host cores, on a bounded sample of the same workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import sidco_oracle as O
+    from paper_2101_10761_b200 import workloads as W
+    wl = W.config(4)
+    # bounded sample: a prefix of whole segments sized so that K + W steps end within ~2 minutes
+    probe = wl.draw(0)
+    t0 = time.perf_counter()
+    O.sidco_compress(probe, np.zeros(wl.d, np.float32), wl.seg_offsets, DELTA, args.sid, 4, state=O.new_state(wl.n_segs))
+    per_elem = (time.perf_counter() - t0) / wl.d
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    off = wl.seg_offsets
+    n_seg = int(np.searchsorted(off, min(wl.d, max(1, int(budget / per_elem))), side="right") - 1)
+    n_seg = max(1, min(wl.n_segs, n_seg))
+    sub_off = off[: n_seg + 1]
+    d_sub = int(sub_off[-1])
+    grads = [probe[:d_sub]] + [wl.draw(c)[:d_sub] for c in range(1, N_GRADS)]
+    res = np.zeros(d_sub, np.float32)
+    state = O.new_state(n_seg)
+    for i in range(args.warmup):
+        res = O.sidco_compress(grads[i % N_GRADS], res, sub_off, DELTA, args.sid, 4, state=state).residual
+    bytes_min = 0
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        out = O.sidco_compress(grads[i % N_GRADS], res, sub_off, DELTA, args.sid, 4, state=state)
+        res = out.residual
+        bytes_min += 12 * d_sub + 8 * int(out.out_k[-1])
+    dt = time.perf_counter() - t0
+    value = bytes_min / dt / 1e9
+    sample = f"first {n_seg} of {wl.n_segs} segments ({d_sub} of {wl.d} elements) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "resnet50-shaped d=25557032 161 segments delta=1e-3", "sid": SID_NAMES[args.sid],
+                   "max_stages": 4, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "elements_per_s": d_sub * args.steps / dt,
+    }
+    print(json.dumps(line))
+
+
+def run_gpu(args):
+    import torch
+    from paper_2101_10761_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    B.lib()   # fail loudly here if the CUDA library is missing
+    wl, grads_h = make_inputs()
+    off = wl.seg_offsets
+    d, S = wl.d, wl.n_segs
+    grads = [torch.from_numpy(g).to(dev) for g in grads_h]
+    res = torch.zeros(d, dtype=torch.float32, device=dev)
+    out_idx = torch.empty(d, dtype=torch.int32, device=dev)
+    out_val = torch.empty(d, dtype=torch.float32, device=dev)
+    out_k = torch.zeros(S + 1, dtype=torch.int32, device=dev)
+    out_k_steps = torch.zeros(args.steps, S + 1, dtype=torch.int32, device=dev)   # one out_k per timed step
+
+    def step(i, k_buf=None):
+        B.sidco_compress(grads[i % N_GRADS], res, off, DELTA, args.sid, args.max_stages, out_idx, out_val,
+                         out_k if k_buf is None else k_buf)
+
+    uuid = getattr(torch.cuda.get_device_properties(local_rank), "uuid", None)
+    sampler = ClockSampler(local_rank, str(uuid) if uuid is not None else None)
+    sampler.start()
+
+    # untimed: bring the clocks up and pass the first adaptation points
+    step(0)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    i = 0
+    while time.perf_counter() - t0 < 0.3:
+        for _ in range(20):
+            step(i)
+            i += 1
+        torch.cuda.synchronize()
+    prewarm_steps = i
+    for w in range(args.warmup):
+        step(i + w)
+    i += args.warmup
+
+    # ---- timed region: device-resident inputs --------------------------------------------
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.sidco_launch_count()
+    barrier()
+    sampler.region = "device"
+    for s in range(args.steps):
+        ev[s][0].record()
+        step(i + s, out_k_steps[s])
+        ev[s][1].record()
+    barrier()
+    sampler.region = None
+    launches = B.sidco_launch_count() - launches0
+    total_ms = ev[0][0].elapsed_time(ev[-1][1])
+    kern_ms = [a.elapsed_time(b) for a, b in ev]
+    k_hats = out_k_steps[:, S].cpu().numpy().astype(np.int64)
+    bytes_min = int(12 * d * args.steps + 8 * k_hats.sum())
+    dbg = B.sidco_get_debug(res, S)
+    m_hist = {}
+    for sd in dbg:
+        m_hist[str(sd.M_used)] = m_hist.get(str(sd.M_used), 0) + 1
+    status_or = 0
+    for sd in dbg:
+        status_or |= sd.status
+    i += args.steps
+
+    # ---- end to end: pinned host buffers through sidco_compress_host ----------------------
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    h_grads = [torch.from_numpy(g).pin_memory() for g in grads_h]
+    h_res = torch.zeros(d, dtype=torch.float32).pin_memory()
+    h_idx = torch.empty(d, dtype=torch.int32).pin_memory()
+    h_val = torch.empty(d, dtype=torch.float32).pin_memory()
+    h_k = torch.zeros(S + 1, dtype=torch.int32).pin_memory()
+    for w in range(3):
+        B.sidco_compress_host(h_grads[w % N_GRADS], h_res, off, DELTA, args.sid, args.max_stages, h_idx, h_val, h_k)
+    barrier()
+    sampler.region = "e2e"
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    e2e_bytes_min, d2h = 0, 0
+    for s in range(e2e_steps):
+        B.sidco_compress_host(h_grads[s % N_GRADS], h_res, off, DELTA, args.sid, args.max_stages, h_idx, h_val, h_k)
+        kh = int(h_k[S])
+        e2e_bytes_min += 12 * d + 8 * kh
+        d2h += 4 * d + 4 * (S + 1) + 8 * kh
+    e1.record()
+    barrier()
+    sampler.region = None
+    e2e_ms = e0.elapsed_time(e1)
+    sampler.stop()
+
+    # ---- max over ranks, totals over ranks -------------------------------------------------
+    t_dev, t_e2e = total_ms, e2e_ms
+    tot_bytes, tot_e2e_bytes, tot_elems = bytes_min, e2e_bytes_min, d * args.steps
+    if dist is not None:
+        tmax = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        t_dev, t_e2e = float(tmax[0]), float(tmax[1])
+        tsum = torch.tensor([bytes_min, e2e_bytes_min, tot_elems], dtype=torch.float64, device=dev)
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        tot_bytes, tot_e2e_bytes, tot_elems = float(tsum[0]), float(tsum[1]), float(tsum[2])
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        value = tot_bytes / (t_dev * 1e-3) / 1e9
+        kern_avg_ms = sum(kern_ms) / len(kern_ms)
+        alg_bytes = bytes_min / args.steps
+        achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
+        cpu_val, cpu_calls, cpu_dt = oracle_rate(wl, grads_h, args.cpu_budget, args.sid)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": t_dev / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 data, f64 statistics and fits", "data": "synthetic",
+            "config": {
+                "workload": "resnet50-shaped d=25557032 161 segments delta=1e-3 (configs[3])",
+                "sid": SID_NAMES[args.sid], "max_stages": args.max_stages,
+                "M_used_hist_last_step": m_hist, "status_or": status_or,
+                "k_hat_mean": float(k_hats.mean()), "parallelism": "replicas only" if world > 1 else "1 GPU",
+                "l2": "inputs 204 MB per step exceed the 126 MB L2; gradients rotate over 4 distinct buffers",
+                "prewarm_steps": prewarm_steps,
+            },
+            "elements_per_s": tot_elems / (t_dev * 1e-3),
+            "pct_of_8TBs_on_min_bytes": 100.0 * value / world / 8000.0,
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "kernel": "sidco_persistent_kernel", "kernel_avg_ms": kern_avg_ms,
+                "kernel_min_ms": min(kern_ms), "algorithmic_bytes_per_launch": alg_bytes,
+            },
+            "cpu_baseline": {
+                "value": cpu_val, "unit": UNIT, "cores": used_threads(), "kind": "oracle",
+                "sample": f"{cpu_calls} whole calls of the same workload in {cpu_dt:.1f} s",
+            },
+            "e2e": {
+                "value": tot_e2e_bytes / (t_e2e * 1e-3) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": 8 * d, "d2h_bytes_per_step": d2h // e2e_steps, "steps": e2e_steps,
+                "ms_per_step": t_e2e / e2e_steps,
+            },
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+        }
+        print(json.dumps(line))
+    B.sidco_release_all()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None, help="default 1000 (reference arm: 50)")
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sid", type=int, default=0, help="0 EXP (default, the paper's SIDCo-E), 1 GAMMA, 2 GPD")
+    ap.add_argument("--max-stages", type=int, default=4, help=">0 adaptive up to this many stages, <0 fixed")
+    ap.add_argument("--e2e-steps", type=int, default=50)
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.steps is None:
+        args.steps = 50 if args.impl == "reference" else 1000
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

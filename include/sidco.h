@@ -136,6 +136,12 @@ int sidco_reset_state(const float* residual);
  * (`out` has room for n_segs entries).  Synchronises the device; meant for tests and logging. */
 int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);
 
+/* Phase breakdown of the last call in microseconds, from device timestamps taken by one CTA at the
+ * grid-wide barriers: us_out[0] error compensation + stage-1 statistics and fit, [1] stage-2 side-buffer
+ * compaction and fit, [2] stages 3..M, [3] survivor staging + residual zeroing, [4] final placement and
+ * adaptation, [5] whole kernel.  Synchronises the device; for profiling. */
+int sidco_get_phase_times(const float* residual, double* us_out);
+
 /* Checkpointing of the adaptation state (Algorithm 1 keeps M and the running k_hat sum across
  * iterations): host blobs of 3 int64 per segment (M, calls, k_sum).  Both synchronise the device. */
 int sidco_state_save(const float* residual, int64_t* host_blob, int n_segs);

@@ -38,6 +38,7 @@ EXPORTS = [
     "sidco_compress", "sidco_compress_host", "sidco_workspace_bytes", "sidco_set_workspace",
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
+    "sidco_get_phase_times",
 ]
 
 _lib = None
@@ -76,6 +77,8 @@ def lib() -> C.CDLL:
     L.sidco_reset_state.restype = i32
     L.sidco_get_debug.argtypes = [vp, C.POINTER(SegDebug), i32]
     L.sidco_get_debug.restype = i32
+    L.sidco_get_phase_times.argtypes = [vp, C.POINTER(dbl)]
+    L.sidco_get_phase_times.restype = i32
     L.sidco_state_save.argtypes = [vp, C.POINTER(i64), i32]
     L.sidco_state_save.restype = i32
     L.sidco_state_load.argtypes = [vp, C.POINTER(i64), i32]
@@ -206,3 +209,12 @@ def sidco_version() -> int:
 
 def sidco_error_string(code: int) -> str:
     return lib().sidco_error_string(code).decode()
+
+
+def sidco_get_phase_times(residual):
+    """Microseconds of the last call: [P1, stage 2, stages 3..M, staging, placement, total]."""
+    buf = (C.c_double * 6)()
+    rc = lib().sidco_get_phase_times(_ptr(residual), buf)
+    if rc:
+        raise SidcoError(rc, "sidco_get_phase_times")
+    return list(buf)

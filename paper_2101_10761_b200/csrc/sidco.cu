@@ -1,4 +1,4 @@
-// Host side of the SIDCo sparsifier library: argument checks, tile tables, workspace,
+// Host side of the SIDCo sparsifier library: argument checks, chunk tables, workspace,
 // per-residual state, and the cooperative launch of the persistent kernel.
 #include "sidco_kernel.cuh"
 
@@ -17,7 +17,7 @@ using sidco::Args;
 using sidco::Control;
 using sidco::SegDev;
 using sidco::kThreads;
-using sidco::kTile;
+using sidco::kChunk;
 
 struct Params {
     double delta1 = 0.25, eps_H = 0.2, eps_L = 0.2;
@@ -27,16 +27,17 @@ struct Params {
 struct DeviceInfo {
     int sm_count = 0;
     int ctas_per_sm = 0;     // min over the kernel instantiations
+    int grid = 0;            // CTAs per launch (all co-resident)
     bool ready = false;
 };
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Offsets of the workspace parts for (d, S, T, G).
+// Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
-    size_t tile_start, tile_seg, seg_tile0, seg_n, cta_tile0;
-    size_t part, part_n, side_cnt, tile_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, seg, ctl;
+    size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_chunk0;
+    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, seg, ctl;
     size_t total;
 };
 
@@ -44,15 +45,16 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     Layout L{};
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
-    L.tile_start = take(sizeof(int32_t) * (size_t)(T + 1));
-    L.tile_seg = take(sizeof(int32_t) * (size_t)(T + 1));
-    L.seg_tile0 = take(sizeof(int32_t) * (size_t)(S + 1));
+    L.chunk_start = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.chunk_seg = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.seg_chunk0 = take(sizeof(int32_t) * (size_t)(S + 1));
     L.seg_n = take(sizeof(int32_t) * (size_t)(S + 1));
-    L.cta_tile0 = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.seg_runs = take(sizeof(int32_t) * (size_t)(S + 1));
+    L.cta_chunk0 = take(sizeof(int32_t) * (size_t)(G + 1));
     L.part = take(sizeof(double) * 3 * (size_t)(T + 1));
     L.part_n = take(sizeof(int32_t) * (size_t)(T + 1));
     L.side_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
-    L.tile_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
+    L.chunk_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
     L.side_idx = take(sizeof(int32_t) * (size_t)(d + 4));
     L.side_val = take(sizeof(float) * (size_t)(d + 4));
     L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
@@ -64,8 +66,8 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     return L;
 }
 
-// Upper bound on the tile count: every window and every segment start opens at most one tile.
-int64_t max_tiles(int64_t d, int S) { return (d + kTile - 1) / kTile + S + 1; }
+// Upper bound on the chunk count: every window and every segment start opens at most one chunk.
+int64_t max_chunks(int64_t d, int S) { return (d + kChunk - 1) / kChunk + S + 1; }
 
 constexpr int kMaxGrid = 148 * 8 * 2;   // generous bound used only for sizing sidco_workspace_bytes
 
@@ -110,12 +112,14 @@ cudaError_t device_info(int dev, DeviceInfo** out) {
         int occ = a < b ? a : b;
         occ = occ < c ? occ : c;
         if (occ < 1) return cudaErrorLaunchOutOfResources;
-        if (const char* env = getenv("SIDCO_CTAS_PER_SM")) {
-            int want = atoi(env);
-            if (want >= 1 && want < occ) occ = want;
-        }
         di.sm_count = prop.multiProcessorCount;
         di.ctas_per_sm = occ;
+        di.grid = di.sm_count * occ;
+        // SIDCO_GRID=<n> runs with fewer CTAs (testing that results do not depend on the grid)
+        if (const char* env = getenv("SIDCO_GRID")) {
+            int want = atoi(env);
+            if (want >= 1 && want < di.grid) di.grid = want;
+        }
         di.ready = true;
     }
     *out = &di;
@@ -145,52 +149,59 @@ int check_args(const void* grad, const void* residual, const int64_t* off, int n
     return 0;
 }
 
-// Build the tile tables for a segment table and upload them together with fresh per-segment state.
+// Build the chunk tables for a segment table and upload them together with fresh per-segment state.
 // keep_state: the adaptation state of an existing context survives a change of nothing but the tables.
 cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t stream) {
     const int64_t d = off[S];
     DeviceInfo* di = nullptr;
     cudaError_t e = device_info(c->device, &di);
     if (e != cudaSuccess) return e;
-    const int G = di->sm_count * di->ctas_per_sm;
+    const int G = di->grid;
 
-    std::vector<int32_t> tile_start, tile_seg, seg_tile0(S + 1), seg_n(S + 1, 0);
+    std::vector<int32_t> chunk_start, chunk_seg, seg_chunk0(S + 1), seg_n(S + 1, 0), seg_runs(S + 1, 0);
     for (int s = 0; s < S; ++s) {
-        seg_tile0[s] = (int32_t)tile_start.size();
+        seg_chunk0[s] = (int32_t)chunk_start.size();
         seg_n[s] = (int32_t)(off[s + 1] - off[s]);
         int64_t at = off[s];
         while (at < off[s + 1]) {
-            int64_t end = (at / kTile + 1) * kTile;
+            int64_t end = (at / kChunk + 1) * kChunk;
             if (end > off[s + 1]) end = off[s + 1];
-            tile_start.push_back((int32_t)at);
-            tile_seg.push_back(s);
+            chunk_start.push_back((int32_t)at);
+            chunk_seg.push_back(s);
             at = end;
         }
     }
-    const int T = (int)tile_start.size();
-    seg_tile0[S] = T;
-    tile_start.push_back((int32_t)d);
-    tile_seg.push_back(0);
+    const int T = (int)chunk_start.size();
+    seg_chunk0[S] = T;
+    chunk_start.push_back((int32_t)d);
+    chunk_seg.push_back(0);
 
-    // Static partition of the tiles over the CTAs, balanced by elements plus a per-tile overhead.
-    std::vector<int32_t> cta_tile0(G + 1, T);
+    // Static partition of the chunks over the CTAs (contiguous runs), balanced by elements plus a
+    // per-chunk overhead.
+    std::vector<int32_t> cta_chunk0(G + 1, T);
     {
-        const double per_tile = 1024.0;
+        const double per_chunk = 128.0;
         double total = 0.0;
-        for (int t = 0; t < T; ++t) total += (tile_start[t + 1] - tile_start[t]) + per_tile;
+        for (int t = 0; t < T; ++t) total += (chunk_start[t + 1] - chunk_start[t]) + per_chunk;
         double acc = 0.0;
         int cta = 0;
-        cta_tile0[0] = 0;
+        cta_chunk0[0] = 0;
         for (int t = 0; t < T; ++t) {
-            // tile t goes to the CTA whose share contains the tile's midpoint
-            const double w = (tile_start[t + 1] - tile_start[t]) + per_tile;
+            // chunk t goes to the CTA whose share contains the chunk's midpoint
+            const double w = (chunk_start[t + 1] - chunk_start[t]) + per_chunk;
             const double mid = acc + 0.5 * w;
             int want = (int)(mid / total * G);
             if (want > G - 1) want = G - 1;
-            while (cta < want) cta_tile0[++cta] = t;
+            while (cta < want) cta_chunk0[++cta] = t;
             acc += w;
         }
-        while (cta < G) cta_tile0[++cta] = T;
+        while (cta < G) cta_chunk0[++cta] = T;
+    }
+    // number of CTA runs that hold chunks of each segment (arrivals expected per statistics phase)
+    for (int g = 0; g < G; ++g) {
+        int prev = -1;
+        for (int t = cta_chunk0[g]; t < cta_chunk0[g + 1]; ++t)
+            if (chunk_seg[t] != prev) { prev = chunk_seg[t]; ++seg_runs[prev]; }
     }
 
     const Layout L = make_layout(d, S, T, G);
@@ -214,7 +225,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
         if ((e = cudaMemcpy(seg_host.data(), (char*)c->ws + c->L.seg, sizeof(SegDev) * S, cudaMemcpyDeviceToHost)) !=
             cudaSuccess)
             return e;
-        for (auto& sg : seg_host) sg.arrived = 0;
+        for (auto& sg : seg_host) { sg.arrived = 0; sg.k_acc = 0; }
     } else {
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
         for (auto& sg : seg_host) {
@@ -226,15 +237,16 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     auto up = [&](size_t at, const void* src, size_t bytes) {
         return cudaMemcpy(base + at, src, bytes, cudaMemcpyHostToDevice);
     };
-    if ((e = up(L.tile_start, tile_start.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
-    if ((e = up(L.tile_seg, tile_seg.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
-    if ((e = up(L.seg_tile0, seg_tile0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = up(L.chunk_start, chunk_start.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = up(L.chunk_seg, chunk_seg.data(), sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg_chunk0, seg_chunk0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg_n, seg_n.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
-    if ((e = up(L.cta_tile0, cta_tile0.data(), sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg_runs, seg_runs.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = up(L.cta_chunk0, cta_chunk0.data(), sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
-    if ((e = cudaMemset(base + L.tile_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
 
     c->L = L;
     c->d = d;
@@ -263,15 +275,16 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.out_idx = out_idx;
     a.out_val = out_val;
     a.out_k = out_k;
-    a.tile_start = (const int32_t*)(base + L.tile_start);
-    a.tile_seg = (const int32_t*)(base + L.tile_seg);
-    a.seg_tile0 = (const int32_t*)(base + L.seg_tile0);
+    a.chunk_start = (const int32_t*)(base + L.chunk_start);
+    a.chunk_seg = (const int32_t*)(base + L.chunk_seg);
+    a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
     a.seg_n = (const int32_t*)(base + L.seg_n);
-    a.cta_tile0 = (const int32_t*)(base + L.cta_tile0);
+    a.seg_runs = (const int32_t*)(base + L.seg_runs);
+    a.cta_chunk0 = (const int32_t*)(base + L.cta_chunk0);
     a.part = (double*)(base + L.part);
     a.part_n = (int32_t*)(base + L.part_n);
     a.side_cnt = (int32_t*)(base + L.side_cnt);
-    a.tile_cnt = (int32_t*)(base + L.tile_cnt);
+    a.chunk_cnt = (int32_t*)(base + L.chunk_cnt);
     a.side_idx = (int32_t*)(base + L.side_idx);
     a.side_val = (float*)(base + L.side_val);
     a.stage_idx = (int32_t*)(base + L.stage_idx);
@@ -286,7 +299,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.Q = prm.Q;
     a.sid = sid;
     a.max_stages = max_stages;
-    a.T = c->T;
+    a.C = c->T;
     a.S = c->S;
     a.G = c->G;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
@@ -380,7 +393,7 @@ int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_o
 
 size_t sidco_workspace_bytes(int64_t d, int n_segs) {
     if (d < 0 || n_segs < 1) return 0;
-    return make_layout(d, n_segs, max_tiles(d, n_segs), kMaxGrid).total;
+    return make_layout(d, n_segs, max_chunks(d, n_segs), kMaxGrid).total;
 }
 
 int sidco_set_workspace(const float* residual, void* device_ptr, size_t bytes) {
@@ -458,6 +471,22 @@ int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs) {
             out[s].k_stage[m] = seg[s].k_stage[m];
         }
     }
+    return 0;
+}
+
+int sidco_get_phase_times(const float* residual, double* us_out) {
+    if (!us_out) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    Context* c = it->second;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    Control ctl;
+    if ((e = cudaMemcpy(&ctl, (char*)c->ws + c->L.ctl, sizeof(Control), cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return (int)e;
+    for (int i = 0; i < 5; ++i) us_out[i] = (double)(long long)(ctl.t_ns[i + 1] - ctl.t_ns[i]) * 1e-3;
+    us_out[5] = (double)(long long)(ctl.t_ns[5] - ctl.t_ns[0]) * 1e-3;
     return 0;
 }
 

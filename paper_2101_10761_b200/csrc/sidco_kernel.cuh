@@ -1,26 +1,30 @@
 // Device code of the SIDCo sparsifier for sm_100a.
 //
 // One persistent cooperative kernel runs the whole call.  The flat vector is cut
-// into tiles that never straddle a segment or an 8192-element window; every CTA
-// owns one contiguous run of tiles for the whole call, so data a CTA wrote in one
-// phase (acc, side buffers) is re-read by the same CTA in the next one.  Phases
-// are separated by grid-wide barriers with bounded waits:
+// into chunks that never straddle a segment or a 1024-element window.  Every CTA
+// (one per SM, 32 warps) owns one contiguous run of chunks for the whole call, so
+// what it wrote in one phase (acc, side buffers) it re-reads itself in the next.
+// Inside a run the warps pull chunks from a shared-memory queue and work on them
+// without any block-level synchronisation: a chunk is loaded, reduced with warp
+// shuffles, and compacted with ballots by one warp.  Phases are separated by
+// grid-wide barriers with bounded waits:
 //
-//   P1  acc = grad + residual (stored over residual) and stage-1 statistics per
-//       tile; the CTA that completes a segment's last tile sums the per-tile
-//       partials in tile order and fits eta_1 (Corollaries 1.1-1.3)
+//   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
+//       of every chunk; the CTA whose run completes a segment sums the per-chunk
+//       partials in chunk order and fits eta_1 (Corollaries 1.1-1.3)
 //   P3  (only if some segment uses M >= 2) exceedances |x| > eta_1 compacted, in
-//       order, into the segment's side buffer together with the statistics of the
-//       shifted peaks (Lemma 2 / Corollary 2.1); last arriver fits eta_2
-//   P4  (m = 3..M) statistics of side-buffer entries above eta_{m-1}; fit eta_m
-//   P5a survivors |x| >= eta_M staged per tile in ascending order (from acc for
-//       M = 1, from the side buffer otherwise), selected residual entries zeroed
-//   P5b CTA bases from the per-CTA totals, staged survivors copied to their final
-//       ascending positions, per-segment counts and stage adaptation
+//       order, into the chunk's side region together with the statistics of the
+//       shifted peaks (Lemma 2 / Corollary 2.1); fit of eta_2
+//   P4  (m = 3..M) statistics of side-region entries above eta_{m-1}; fit eta_m
+//   P5a survivors |x| >= eta_M staged per chunk in ascending order (from acc for
+//       M = 1, from the side region otherwise), selected residual entries zeroed
+//   P5b CTA bases from the per-CTA totals, chunk bases by a block scan, staged
+//       survivors copied to their final ascending positions, per-segment counts
+//       and stage adaptation (Algorithm 1, Adapt_Stages)
 //
-// Reductions are deterministic: per-thread sequential accumulation, a fixed
-// shuffle tree per tile, and a fixed-order sum of per-tile partials, so thresholds
-// do not depend on the grid size or on which CTA performs a fit.
+// Reductions are deterministic and independent of the grid: per-lane sequential
+// accumulation in a fixed order, a fixed shuffle tree per chunk, and a fixed-order
+// sum of the per-chunk partials of a segment.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -28,14 +32,15 @@
 
 namespace sidco {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
-constexpr int kTile = 8192;                       // window: elements per full tile
-constexpr int kSlots = kTile / 4 / kThreads;      // float4 slots per thread per tile (8)
-constexpr int kWarpElems = kTile / kWarps;        // contiguous elements per warp (1024)
+constexpr int kChunk = 1024;                      // window: elements per full chunk (one warp)
+constexpr int kSlots = kChunk / 128;              // float4 slots per lane per chunk (8)
+constexpr int kSmallSeg = 32;                     // segments of <= 32 chunks are summed by one warp
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr long long kSpinLimit = 1ll << 22;       // bounded waits: ~1 s with the back-off below
+static_assert(kWarps == 32, "block_tree and the scans assume 32 warps per CTA");
 
 enum { kSidExp = 0, kSidGamma = 1, kSidGpd = 2 };
 enum { kStNonFinite = 1, kStDegenerate = 2, kStAllZero = 4, kStTimeout = 8 };
@@ -47,10 +52,10 @@ struct SegDev {
     float thr_ge;        // smallest fp32 >= eta_M:                  (|x| >= thr_ge) == (|x| >= eta_M)
     int32_t M_eff;       // stages used by this call
     int32_t status;
-    int32_t arrived;     // tiles of this segment finished in the current phase (self-resetting)
+    int32_t arrived;     // CTA runs of this segment finished in the current phase (self-resetting)
+    int32_t k_acc;       // survivors counted so far in this call (integer atomics; self-resetting)
     int32_t M;           // adaptation state: stage count for the next adaptive call
     int32_t calls;
-    int32_t pad;
     long long k_sum;
 };
 
@@ -59,6 +64,7 @@ struct Control {
     unsigned finished;
     int timeout;         // set when a bounded wait ran out
     int M_max_eff;       // max over segments of M_eff for this call
+    unsigned long long t_ns[8];   // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
 };
 
 struct Args {
@@ -68,16 +74,17 @@ struct Args {
     float* out_val;
     int32_t* out_k;
     // tables (read only during the call)
-    const int32_t* tile_start;   // [T + 1]
-    const int32_t* tile_seg;     // [T]
-    const int32_t* seg_tile0;    // [S + 1]
+    const int32_t* chunk_start;  // [C + 1]
+    const int32_t* chunk_seg;    // [C]
+    const int32_t* seg_chunk0;   // [S + 1]
     const int32_t* seg_n;        // [S]
-    const int32_t* cta_tile0;    // [G + 1]
+    const int32_t* seg_runs;     // [S] number of CTA runs that hold chunks of the segment
+    const int32_t* cta_chunk0;   // [G + 1]
     // scratch
-    double* part;                // [T][3] per-tile partial sums
-    int32_t* part_n;             // [T] per-tile partial counts
-    int32_t* side_cnt;           // [T] stage-2 exceedances stored for the tile
-    int32_t* tile_cnt;           // [T] final survivors staged for the tile
+    double* part;                // [C][3] per-chunk partial sums
+    int32_t* part_n;             // [C] per-chunk partial counts
+    int32_t* side_cnt;           // [C] stage-2 exceedances stored for the chunk
+    int32_t* chunk_cnt;          // [C] final survivors staged for the chunk
     int32_t* side_idx;           // [d]
     float* side_val;             // [d]
     int32_t* stage_idx;          // [d]
@@ -88,7 +95,7 @@ struct Args {
     // scalars
     double delta, delta1, eps_H, eps_L;
     int Q, sid, max_stages;
-    int T, S, G;
+    int C, S, G;
     int vec_ok;                  // grad and residual are 16-byte aligned
 };
 
@@ -104,6 +111,12 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
 
 __device__ __forceinline__ int ld_volatile(const int* p) {
@@ -124,48 +137,49 @@ __device__ __forceinline__ void grid_barrier(Control* ctl, int G, int which) {
         while (ld_acquire(&ctl->bar) < target) {
             if (ld_volatile(&ctl->timeout)) break;
             if (++spins > kSpinLimit) { atomicExch(&ctl->timeout, 1); break; }
-            __nanosleep(spins < 64 ? 32 : 200);
+            __nanosleep(spins < 64 ? 20 : 200);
         }
         __threadfence();
     }
     __syncthreads();
 }
 
-struct RedOut { double a, b, c; int n; };
+struct Sums { double a, b; int n; };
 
-// Block-wide sums of three doubles and one int with a fixed tree; result valid in thread 0.
-__device__ __forceinline__ RedOut block_sum(double a, double b, double c, int n, double (*sm)[4]) {
+__device__ __forceinline__ Sums warp_tree(double a, double b, int n) {
     #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         a += __shfl_down_sync(kFull, a, o);
         b += __shfl_down_sync(kFull, b, o);
-        c += __shfl_down_sync(kFull, c, o);
         n += __shfl_down_sync(kFull, n, o);
     }
+    return Sums{a, b, n};
+}
+
+// Block-wide sums with a fixed tree (warp trees, then one warp over the 32 warp results);
+// result valid in thread 0.
+__device__ __forceinline__ Sums block_tree(double a, double b, int n, double (*sm)[3]) {
+    Sums w = warp_tree(a, b, n);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __syncthreads();                       // previous use of sm is over
-    if (lane == 0) { sm[warp][0] = a; sm[warp][1] = b; sm[warp][2] = c; sm[warp][3] = (double)n; }
+    if (lane == 0) { sm[warp][0] = w.a; sm[warp][1] = w.b; sm[warp][2] = (double)w.n; }
     __syncthreads();
-    RedOut r{0.0, 0.0, 0.0, 0};
+    Sums r{0.0, 0.0, 0};
     if (warp == 0) {
-        double x = lane < kWarps ? sm[lane][0] : 0.0;
-        double y = lane < kWarps ? sm[lane][1] : 0.0;
-        double z = lane < kWarps ? sm[lane][2] : 0.0;
-        double w = lane < kWarps ? sm[lane][3] : 0.0;
+        double x = sm[lane][0], y = sm[lane][1], z = sm[lane][2];
         #pragma unroll
-        for (int o = kWarps / 2; o > 0; o >>= 1) {
+        for (int o = 16; o > 0; o >>= 1) {
             x += __shfl_down_sync(kFull, x, o);
             y += __shfl_down_sync(kFull, y, o);
             z += __shfl_down_sync(kFull, z, o);
-            w += __shfl_down_sync(kFull, w, o);
         }
-        r.a = x; r.b = y; r.c = z; r.n = (int)w;
+        r.a = x; r.b = y; r.n = (int)z;
     }
     return r;
 }
 
 // ----------------------------------------------------------------------------
-// closed-form fits (thread 0 of the CTA that completed the segment)
+// closed-form fits (one thread)
 // ----------------------------------------------------------------------------
 
 // Largest M with delta1^(M-1) > delta: more stages would leave the last ratio >= 1.
@@ -209,8 +223,8 @@ __device__ inline void publish_eta(SegDev* sg, int m, double eta) {
     sg->thr_ge = __double2float_ru(eta);
 }
 
-// Stage 1 from the segment sums: S1 = sum|x|, S2 = sum x^2 (GPD), SL = sum log|x| over the n_nz
-// nonzero magnitudes (gamma).
+// Stage 1 from the segment sums: S1 = sum|x|, and S2 = sum x^2 (GPD) or SL = sum log|x| over the
+// n_nz nonzero magnitudes (gamma).
 __device__ inline void fit_stage1(const Args& A, SegDev* sg, int n, double S1, double S2_or_SL, int n_nz) {
     int M;
     if (A.max_stages > 0) {
@@ -263,7 +277,7 @@ __device__ inline void fit_stage1(const Args& A, SegDev* sg, int n, double S1, d
     atomicMax(&A.ctl->M_max_eff, M_eff);
 }
 
-// Stage m (1-based index m >= 1 means eta_{m+1}) from the shifted peaks over eta_m:
+// Stage index m >= 1 (eta_{m+1} in the paper's numbering) from the shifted peaks over eta_m:
 // n_e = #{|x| > eta_m}, Sy = sum(|x| - eta_m), Sy2 = sum(|x| - eta_m)^2.
 __device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, double Sy, double Sy2) {
     // fields another SM may have written during this call are read through L2
@@ -284,50 +298,49 @@ __device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, do
 }
 
 // ----------------------------------------------------------------------------
-// tile access
+// chunk access (one warp)
 // ----------------------------------------------------------------------------
 
-// Streaming load for data that is read exactly once (the gradient).
 __device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ float4 ld_l2_4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
-// Load the part [lo, hi) of the window starting at wb from `src` into registers in tile order
-// (warp-major, then slot, lane, component).  Returns the validity mask: bit 4*j + c.
-__device__ __forceinline__ unsigned load_tile(const float* __restrict__ src, int lo, int hi, int wb, bool vec_ok,
-                                              float (&v)[kSlots][4]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int e0 = wb + warp * kWarpElems + lane * 4;
-    unsigned valid = 0;
-    if (vec_ok && lo == wb && hi == wb + kTile) {
+// Load the part [lo, hi) of the window starting at wb from `src` into registers in chunk order
+// (slot, lane, component).  Returns the validity mask: bit 4*j + c.  Loads go through L2 only: the
+// data was written earlier in this kernel (by this SM) and is read once.
+__device__ __forceinline__ unsigned load_chunk(const float* __restrict__ src, int lo, int hi, int wb, bool vec_ok,
+                                               float (&v)[kSlots][4]) {
+    const int e0 = wb + (threadIdx.x & 31) * 4;
+    if (vec_ok && lo == wb && hi == wb + kChunk) {
         #pragma unroll
         for (int j = 0; j < kSlots; ++j) {
-            const float4 q = *reinterpret_cast<const float4*>(src + e0 + j * 128);
+            const float4 q = ld_l2_4(src + e0 + j * 128);
             v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
         }
         return kFull;
     }
+    unsigned valid = 0;
     #pragma unroll
     for (int j = 0; j < kSlots; ++j) {
         const int e = e0 + j * 128;
         v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0.0f;
         if (e + 4 <= lo || e >= hi) continue;
         if (vec_ok && e >= lo && e + 4 <= hi) {
-            const float4 q = *reinterpret_cast<const float4*>(src + e);
+            const float4 q = ld_l2_4(src + e);
             v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
             valid |= 0xFu << (4 * j);
         } else {
             #pragma unroll
             for (int c = 0; c < 4; ++c)
-                if (e + c >= lo && e + c < hi) { v[j][c] = src[e + c]; valid |= 1u << (4 * j + c); }
+                if (e + c >= lo && e + c < hi) { v[j][c] = __ldcg(src + e + c); valid |= 1u << (4 * j + c); }
         }
     }
     return valid;
 }
 
 // Warp-ordered emission: calls emit(position, j, c) for every set bit of `mask`, positions counted
-// in tile order starting at `base` for this warp.
+// in chunk order starting at `base`.  Returns the number of set bits in the warp.
 template <class Emit>
-__device__ __forceinline__ void ordered_emit(unsigned mask, int base, Emit emit) {
+__device__ __forceinline__ int ordered_emit(unsigned mask, int base, Emit emit) {
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
     int run = base;
     #pragma unroll
@@ -344,53 +357,111 @@ __device__ __forceinline__ void ordered_emit(unsigned mask, int base, Emit emit)
         for (int cc = 0; cc < 4; ++cc)
             if (nib & (1u << cc)) { emit(p, j, cc); ++p; }
     }
+    return run - base;
 }
 
-// Exclusive position of this warp among the CTA's warps and the CTA total, from per-warp counts.
-__device__ __forceinline__ int warp_bases(int warp_count, int* sm_cnt, int& total) {
+// Per-warp view of the segment a chunk belongs to, reloaded only when the segment changes.
+struct SegView {
+    int seg = -1;
+    int M_eff = 0;
+    float thr_gt = 0.f, thr_ge = 0.f;
+    double eta_prev = 0.0;
+    __device__ __forceinline__ void load(const Args& A, int s, int m_prev) {
+        if (s == seg) return;
+        seg = s;
+        const SegDev* sg = &A.seg[s];
+        M_eff = ld_cg(&sg->M_eff);
+        thr_gt = ld_cg(&sg->thr_gt);
+        thr_ge = ld_cg(&sg->thr_ge);
+        eta_prev = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
+    }
+};
+
+// Dynamic chunk queue of a CTA run: warps take the next chunk index (ascending or descending).
+struct ChunkQueue {
+    int* sm_next;
+    int c0, c1;
+    __device__ __forceinline__ int next(bool descending) const {
+        int k = 0;
+        if ((threadIdx.x & 31) == 0) k = atomicAdd(sm_next, 1);
+        k = __shfl_sync(kFull, k, 0);
+        if (k >= c1 - c0) return -1;
+        return descending ? c1 - 1 - k : c0 + k;
+    }
+};
+
+// ----------------------------------------------------------------------------
+// end of a statistics phase: arrivals and fits for the segments of this CTA's run
+// ----------------------------------------------------------------------------
+
+// `stage` = 0 for the first stage, m >= 1 for the refits.  Every CTA calls this after its warps
+// have written the partials of all chunks of its run.
+__device__ __forceinline__ void arrive_and_fit(const Args& A, int c0, int c1, int stage, int* sm_list, int* sm_count,
+                                               double (*sm_red)[3]) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *sm_count = 0;
+    __syncthreads();
+    if (c0 >= c1) return;
+    const int seg_lo = A.chunk_seg[c0], seg_hi = A.chunk_seg[c1 - 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();
-    if (lane == 0) sm_cnt[warp] = warp_count;
-    __syncthreads();
-    int base = 0, tot = 0;
-    #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        const int c = sm_cnt[w];
-        if (w < warp) base += c;
-        tot += c;
+    for (int base = seg_lo; base <= seg_hi; base += kThreads) {
+        const int s = base + (int)threadIdx.x;
+        if (s <= seg_hi && A.seg_chunk0[s + 1] > A.seg_chunk0[s]) {
+            SegDev* sg = &A.seg[s];
+            const bool takes_part = stage == 0 || ld_cg(&sg->M_eff) > stage;
+            if (takes_part) {
+                __threadfence();
+                const int old = atomicAdd(&sg->arrived, 1);
+                if (old == A.seg_runs[s] - 1) {
+                    sg->arrived = 0;
+                    __threadfence();
+                    sm_list[atomicAdd(sm_count, 1)] = s;
+                }
+            }
+        }
+        __syncthreads();
+        const int n_done = *sm_count;
+        // small segments: one warp each, lanes take one chunk partial each, fixed shuffle tree
+        for (int i = warp; i < n_done; i += kWarps) {
+            const int s2 = sm_list[i];
+            const int q0 = A.seg_chunk0[s2], q1 = A.seg_chunk0[s2 + 1];
+            if (q1 - q0 > kSmallSeg) continue;
+            double a = 0.0, b = 0.0;
+            int n = 0;
+            if (q0 + lane < q1) {
+                a = ld_cg(A.part + 3 * (size_t)(q0 + lane) + 0);
+                b = ld_cg(A.part + 3 * (size_t)(q0 + lane) + 1);
+                n = ld_cg(A.part_n + q0 + lane);
+            }
+            Sums r = warp_tree(a, b, n);
+            if (lane == 0) {
+                if (stage == 0) fit_stage1(A, &A.seg[s2], A.seg_n[s2], r.a, r.b, r.n);
+                else fit_stage_m(A, &A.seg[s2], stage, r.n, r.a, r.b);
+            }
+        }
+        // large segments: the whole CTA, threads stride over the chunk partials, fixed block tree
+        for (int i = 0; i < n_done; ++i) {
+            const int s2 = sm_list[i];
+            const int q0 = A.seg_chunk0[s2], q1 = A.seg_chunk0[s2 + 1];
+            if (q1 - q0 <= kSmallSeg) continue;
+            double a = 0.0, b = 0.0;
+            int n = 0;
+            for (int q = q0 + (int)threadIdx.x; q < q1; q += kThreads) {
+                a += ld_cg(A.part + 3 * (size_t)q + 0);
+                b += ld_cg(A.part + 3 * (size_t)q + 1);
+                n += ld_cg(A.part_n + q);
+            }
+            Sums r = block_tree(a, b, n, sm_red);
+            if (threadIdx.x == 0) {
+                if (stage == 0) fit_stage1(A, &A.seg[s2], A.seg_n[s2], r.a, r.b, r.n);
+                else fit_stage_m(A, &A.seg[s2], stage, r.n, r.a, r.b);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) *sm_count = 0;
+        __syncthreads();
     }
-    total = tot;
-    return base;
-}
-
-// Arrival of one tile of segment `seg`.  Returns true (to the whole CTA) when this was the segment's
-// last tile of the phase; the caller then reduces the segment's partials and fits.
-__device__ __forceinline__ bool segment_arrive(const Args& A, int seg, int* sm_flag) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const int ntiles = A.seg_tile0[seg + 1] - A.seg_tile0[seg];
-        const int old = atomicAdd(&A.seg[seg].arrived, 1);
-        const int last = (old == ntiles - 1);
-        if (last) { A.seg[seg].arrived = 0; __threadfence(); }
-        *sm_flag = last;
-    }
-    __syncthreads();
-    return *sm_flag != 0;
-}
-
-// Fixed-order sum of the per-tile partials of a segment (whole CTA); result in thread 0.
-__device__ __forceinline__ RedOut segment_sum(const Args& A, int seg, double (*sm)[4]) {
-    const int t0 = A.seg_tile0[seg], t1 = A.seg_tile0[seg + 1];
-    double a = 0.0, b = 0.0, c = 0.0;
-    int n = 0;
-    for (int t = t0 + (int)threadIdx.x; t < t1; t += kThreads) {
-        a += ld_cg(A.part + 3 * (size_t)t + 0);
-        b += ld_cg(A.part + 3 * (size_t)t + 1);
-        c += ld_cg(A.part + 3 * (size_t)t + 2);
-        n += ld_cg(A.part_n + t);
-    }
-    return block_sum(a, b, c, n, sm);
 }
 
 // ----------------------------------------------------------------------------
@@ -398,30 +469,37 @@ __device__ __forceinline__ RedOut segment_sum(const Args& A, int seg, double (*s
 // ----------------------------------------------------------------------------
 
 template <int SID>
-__global__ void __launch_bounds__(kThreads, 4) sidco_persistent_kernel(const Args A) {
-    __shared__ double sm_red[kWarps][4];
-    __shared__ int sm_cnt[kWarps];
-    __shared__ int sm_flag;
+__global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Args A) {
+    __shared__ double sm_red[kWarps][3];
+    __shared__ int sm_list[kThreads];
+    __shared__ int sm_scan[kThreads];
+    __shared__ int sm_warp[kWarps];
+    __shared__ int sm_count;
+    __shared__ int sm_next;
     __shared__ int sm_base;
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int t_begin = A.cta_tile0[cta], t_end = A.cta_tile0[cta + 1];
+    const int c0 = A.cta_chunk0[cta], c1 = A.cta_chunk0[cta + 1];
     const bool vec_ok = A.vec_ok != 0;
+    const ChunkQueue queue{&sm_next, c0, c1};
     int barrier_no = 0;
+    const bool stamper = (cta == 0 && threadIdx.x == 0);
+    if (stamper) A.ctl->t_ns[0] = global_ns();
+    if (threadIdx.x == 0) sm_next = 0;
 
-    // Segments without tiles (n = 0) never see an arrival: give them their defaults here.
-    for (int s = cta; s < A.S; s += A.G)
-        if (A.seg_tile0[s + 1] == A.seg_tile0[s] && threadIdx.x == 0) fit_stage1(A, &A.seg[s], 0, 0.0, 0.0, 0);
+    // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
+    for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
+        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], 0, 0.0, 0.0, 0);
+    __syncthreads();
 
     // ------------------------------------------------------------------ P1
-    // Descending tile order: the tiles touched last are the ones P3/P5a read first, which
+    // Descending chunk order: the chunks touched last are the ones P3/P5a read first, which
     // raises the share of acc that is still in L2 when it is read again.
-    for (int t = t_end - 1; t >= t_begin; --t) {
-        const int lo = A.tile_start[t], hi = A.tile_start[t + 1];
-        const int wb = lo & ~(kTile - 1);
-        const int seg = A.tile_seg[t];
-        const int e0 = wb + warp * kWarpElems + lane * 4;
+    for (int c = queue.next(true); c >= 0; c = queue.next(true)) {
+        const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
+        const int wb = lo & ~(kChunk - 1);
+        const int e0 = wb + lane * 4;
 
         double s1 = 0.0, s2 = 0.0, prod = 1.0;
         int esum = 0, nnz = 0;
@@ -433,7 +511,7 @@ __global__ void __launch_bounds__(kThreads, 4) sidco_persistent_kernel(const Arg
             if (SID == kSidGamma) {
                 if (a > 0.0f) {
                     // log|x| = exponent * ln 2 + log(mantissa): exponents are summed as integers,
-                    // mantissas multiplied in fp64, one log per tile.
+                    // mantissas multiplied in fp64, one log per chunk.
                     const long long bits = __double_as_longlong(ad);
                     esum += (int)(bits >> 52) - 1023;
                     prod *= __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
@@ -442,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 4) sidco_persistent_kernel(const Arg
             }
         };
 
-        if (vec_ok && lo == wb && hi == wb + kTile) {
+        if (vec_ok && lo == wb && hi == wb + kChunk) {
             #pragma unroll
             for (int b = 0; b < kSlots; b += 4) {
                 float4 g4[4], r4[4];
@@ -473,10 +551,10 @@ __global__ void __launch_bounds__(kThreads, 4) sidco_persistent_kernel(const Arg
                     *reinterpret_cast<float4*>(A.residual + e) = a4;
                     accumulate(a4.x); accumulate(a4.y); accumulate(a4.z); accumulate(a4.w);
                 } else {
-                    for (int c = 0; c < 4; ++c) {
-                        if (e + c >= lo && e + c < hi) {
-                            const float a = ld_stream1(A.grad + e + c) + A.residual[e + c];
-                            A.residual[e + c] = a;
+                    for (int cc = 0; cc < 4; ++cc) {
+                        if (e + cc >= lo && e + cc < hi) {
+                            const float a = __ldcs(A.grad + e + cc) + A.residual[e + cc];
+                            A.residual[e + cc] = a;
                             accumulate(a);
                         }
                     }
@@ -484,226 +562,256 @@ __global__ void __launch_bounds__(kThreads, 4) sidco_persistent_kernel(const Arg
             }
         }
 
-        // per-tile partials
-        double pb = s2;
+        // per-chunk partials with a fixed shuffle tree
+        double second = s2;
         if (SID == kSidGamma) {
-            // normalise the per-thread product, multiply mantissas across the CTA (fixed tree),
-            // then one log: SL_tile = esum * ln2 + log(product)
-            long long bits = __double_as_longlong(prod);
+            // normalise the per-lane product, multiply the mantissas across the warp, one log:
+            // SL_chunk = (sum of exponents) * ln 2 + log(product of mantissas)
+            const long long bits = __double_as_longlong(prod);
             esum += (int)(bits >> 52) - 1023;
             double m = __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
             #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m *= __shfl_down_sync(kFull, m, o);
-            __syncthreads();
-            if (lane == 0) sm_red[warp][0] = m;
-            __syncthreads();
-            double mm = 1.0;
-            if (threadIdx.x == 0) {
-                #pragma unroll
-                for (int w = 0; w < kWarps; ++w) mm *= sm_red[w][0];
+            for (int o = 16; o > 0; o >>= 1) {
+                m *= __shfl_down_sync(kFull, m, o);
+                esum += __shfl_down_sync(kFull, esum, o);
             }
-            pb = mm;     // thread 0 only; converted after the integer sum below
+            second = (double)esum * 0.693147180559945309417232121458 + log(m);   // used from lane 0 only
         }
-        RedOut r = block_sum(s1, SID == kSidGamma ? 0.0 : pb, (double)esum, nnz, sm_red);
-        if (threadIdx.x == 0) {
-            double second = r.b;
-            if (SID == kSidGamma) second = r.c * 0.693147180559945309417232121458 + log(pb);
-            A.part[3 * (size_t)t + 0] = r.a;
-            A.part[3 * (size_t)t + 1] = second;
-            A.part[3 * (size_t)t + 2] = 0.0;
-            A.part_n[t] = r.n;
-        }
-        if (segment_arrive(A, seg, &sm_flag)) {
-            RedOut sres = segment_sum(A, seg, sm_red);
-            if (threadIdx.x == 0) fit_stage1(A, &A.seg[seg], A.seg_n[seg], sres.a, sres.b, sres.n);
+        Sums r = warp_tree(s1, SID == kSidGamma ? 0.0 : second, nnz);
+        if (lane == 0) {
+            A.part[3 * (size_t)c + 0] = r.a;
+            A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
+            A.part_n[c] = r.n;
         }
     }
+    arrive_and_fit(A, c0, c1, 0, sm_list, &sm_count, sm_red);
+    if (threadIdx.x == 0) sm_next = 0;
     grid_barrier(A.ctl, A.G, ++barrier_no);
     const int M_max_eff = ld_volatile(&A.ctl->M_max_eff);
+    if (stamper) A.ctl->t_ns[1] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
 
     // ------------------------------------------------------------------ P3: stage 2 from acc
     if (M_max_eff >= 2) {
-        for (int t = t_begin; t < t_end; ++t) {
-            const int seg = A.tile_seg[t];
-            const SegDev* sg = &A.seg[seg];
-            if (ld_cg(&sg->M_eff) < 2) continue;
-            const int lo = A.tile_start[t], hi = A.tile_start[t + 1];
-            const int wb = lo & ~(kTile - 1);
-            const float thr = ld_cg(&sg->thr_gt);
-            const double eta_prev = ld_cg(&sg->eta[0]);
+        SegView sv;
+        for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
+            sv.load(A, __ldg(A.chunk_seg + c), 0);
+            if (sv.M_eff < 2) continue;
+            const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
+            const int wb = lo & ~(kChunk - 1);
             float v[kSlots][4];
-            const unsigned valid = load_tile(A.residual, lo, hi, wb, vec_ok, v);
+            const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, v);
             unsigned mask = 0;
+            #pragma unroll
+            for (int j = 0; j < kSlots; ++j)
+                #pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (4 * j + cc);
+            mask &= valid;
             double sy = 0.0, sy2 = 0.0;
             #pragma unroll
             for (int j = 0; j < kSlots; ++j)
                 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (fabsf(v[j][c]) > thr) mask |= 1u << (4 * j + c);
-            mask &= valid;
-            #pragma unroll
-            for (int j = 0; j < kSlots; ++j)
-                #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (mask & (1u << (4 * j + c))) {
-                        const double y = (double)fabsf(v[j][c]) - eta_prev;
+                for (int cc = 0; cc < 4; ++cc)
+                    if (mask & (1u << (4 * j + cc))) {
+                        const double y = (double)fabsf(v[j][cc]) - sv.eta_prev;
                         sy += y;
                         if (SID != kSidExp) sy2 = fma(y, y, sy2);
                     }
-            const int wcnt = __reduce_add_sync(kFull, __popc(mask));
-            int total;
-            const int wbase = warp_bases(wcnt, sm_cnt, total);
-            const int e0 = wb + warp * kWarpElems + lane * 4;
-            ordered_emit(mask, lo + wbase, [&](int p, int j, int c) {
-                A.side_idx[p] = e0 + j * 128 + c;
-                A.side_val[p] = v[j][c];
+            const int e0 = wb + lane * 4;
+            const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                A.side_idx[p] = e0 + j * 128 + cc;
+                A.side_val[p] = v[j][cc];
             });
-            RedOut r = block_sum(sy, sy2, 0.0, 0, sm_red);
-            if (threadIdx.x == 0) {
-                A.part[3 * (size_t)t + 0] = r.a;
-                A.part[3 * (size_t)t + 1] = r.b;
-                A.part_n[t] = total;
-                A.side_cnt[t] = total;
-            }
-            if (segment_arrive(A, seg, &sm_flag)) {
-                RedOut sres = segment_sum(A, seg, sm_red);
-                if (threadIdx.x == 0) fit_stage_m(A, &A.seg[seg], 1, sres.n, sres.a, sres.b);
+            Sums r = warp_tree(sy, sy2, 0);
+            if (lane == 0) {
+                A.part[3 * (size_t)c + 0] = r.a;
+                A.part[3 * (size_t)c + 1] = r.b;
+                A.part_n[c] = cnt;
+                A.side_cnt[c] = cnt;
             }
         }
+        arrive_and_fit(A, c0, c1, 1, sm_list, &sm_count, sm_red);
+        if (threadIdx.x == 0) sm_next = 0;
         grid_barrier(A.ctl, A.G, ++barrier_no);
+        if (stamper) A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
 
-        // -------------------------------------------------------------- P4: stages 3..M from the side buffer
+        // -------------------------------------------------------------- P4: stages 3..M from the side regions
         for (int m = 2; m < M_max_eff; ++m) {
-            for (int t = t_begin; t < t_end; ++t) {
-                const int seg = A.tile_seg[t];
-                const SegDev* sg = &A.seg[seg];
-                if (ld_cg(&sg->M_eff) <= m) continue;
-                const int lo = A.tile_start[t];
-                const int wb = lo & ~(kTile - 1);
-                const int hi = lo + A.side_cnt[t];
-                const float thr = ld_cg(&sg->thr_gt);
-                const double eta_prev = ld_cg(&sg->eta[m - 1]);
+            SegView sw;
+            for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
+                sw.load(A, __ldg(A.chunk_seg + c), m - 1);
+                if (sw.M_eff <= m) continue;
+                const int lo = __ldg(A.chunk_start + c);
+                const int wb = lo & ~(kChunk - 1);
+                const int hi = lo + ld_cg(A.side_cnt + c);
                 float v[kSlots][4];
-                const unsigned valid = load_tile(A.side_val, lo, hi, wb, vec_ok, v);
+                const unsigned valid = load_chunk(A.side_val, lo, hi, wb, true, v);
                 double sy = 0.0, sy2 = 0.0;
                 int cnt = 0;
                 #pragma unroll
                 for (int j = 0; j < kSlots; ++j)
                     #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if ((valid & (1u << (4 * j + c))) && fabsf(v[j][c]) > thr) {
-                            const double y = (double)fabsf(v[j][c]) - eta_prev;
+                    for (int cc = 0; cc < 4; ++cc)
+                        if ((valid & (1u << (4 * j + cc))) && fabsf(v[j][cc]) > sw.thr_gt) {
+                            const double y = (double)fabsf(v[j][cc]) - sw.eta_prev;
                             sy += y;
                             if (SID != kSidExp) sy2 = fma(y, y, sy2);
                             ++cnt;
                         }
-                RedOut r = block_sum(sy, sy2, 0.0, cnt, sm_red);
-                if (threadIdx.x == 0) {
-                    A.part[3 * (size_t)t + 0] = r.a;
-                    A.part[3 * (size_t)t + 1] = r.b;
-                    A.part_n[t] = r.n;
-                }
-                if (segment_arrive(A, seg, &sm_flag)) {
-                    RedOut sres = segment_sum(A, seg, sm_red);
-                    if (threadIdx.x == 0) fit_stage_m(A, &A.seg[seg], m, sres.n, sres.a, sres.b);
+                Sums r = warp_tree(sy, sy2, cnt);
+                if (lane == 0) {
+                    A.part[3 * (size_t)c + 0] = r.a;
+                    A.part[3 * (size_t)c + 1] = r.b;
+                    A.part_n[c] = r.n;
                 }
             }
+            arrive_and_fit(A, c0, c1, m, sm_list, &sm_count, sm_red);
+            if (threadIdx.x == 0) sm_next = 0;
             grid_barrier(A.ctl, A.G, ++barrier_no);
+            if (stamper) A.ctl->t_ns[3] = global_ns();
         }
     }
 
-    // ------------------------------------------------------------------ P5a: stage survivors per tile
-    int cta_count = 0;
-    for (int t = t_begin; t < t_end; ++t) {
-        const int seg = A.tile_seg[t];
-        const SegDev* sg = &A.seg[seg];
-        const bool from_side = ld_cg(&sg->M_eff) >= 2;
-        const int lo = A.tile_start[t];
-        const int wb = lo & ~(kTile - 1);
-        const int hi = from_side ? lo + A.side_cnt[t] : A.tile_start[t + 1];
-        const float thr = ld_cg(&sg->thr_ge);
-        float v[kSlots][4];
-        const unsigned valid = load_tile(from_side ? A.side_val : A.residual, lo, hi, wb, vec_ok, v);
-        unsigned mask = 0;
-        #pragma unroll
-        for (int j = 0; j < kSlots; ++j)
+    // ------------------------------------------------------------------ P5a: stage survivors per chunk
+    int warp_total = 0;
+    {
+        SegView sv;
+        int seg_count = 0;       // survivors of sv.seg not yet added to its counter
+        for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
+            const int s = __ldg(A.chunk_seg + c);
+            if (s != sv.seg) {
+                if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
+                seg_count = 0;
+            }
+            sv.load(A, s, -1);
+            const bool from_side = sv.M_eff >= 2;
+            const int lo = __ldg(A.chunk_start + c);
+            const int wb = lo & ~(kChunk - 1);
+            const int hi = from_side ? lo + ld_cg(A.side_cnt + c) : __ldg(A.chunk_start + c + 1);
+            float v[kSlots][4];
+            const unsigned valid = load_chunk(from_side ? A.side_val : A.residual, lo, hi, wb, from_side || vec_ok, v);
+            unsigned mask = 0;
             #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (fabsf(v[j][c]) >= thr) mask |= 1u << (4 * j + c);
-        mask &= valid;
-        const int wcnt = __reduce_add_sync(kFull, __popc(mask));
-        int total;
-        const int wbase = warp_bases(wcnt, sm_cnt, total);
-        if (total > 0) {
-            const int e0 = wb + warp * kWarpElems + lane * 4;
-            ordered_emit(mask, lo + wbase, [&](int p, int j, int c) {
-                const int e = e0 + j * 128 + c;
-                const int idx = from_side ? A.side_idx[e] : e;
-                A.stage_idx[p] = idx;
-                A.stage_val[p] = v[j][c];
-                A.residual[idx] = 0.0f;
-            });
+            for (int j = 0; j < kSlots; ++j)
+                #pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
+            mask &= valid;
+            int cnt = 0;
+            if (__ballot_sync(kFull, mask != 0)) {
+                const int e0 = wb + lane * 4;
+                cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                    const int e = e0 + j * 128 + cc;
+                    const int idx = from_side ? ld_cg(A.side_idx + e) : e;
+                    A.stage_idx[p] = idx;
+                    A.stage_val[p] = v[j][cc];
+                    A.residual[idx] = 0.0f;
+                });
+            }
+            if (lane == 0) A.chunk_cnt[c] = cnt;
+            seg_count += cnt;
+            warp_total += cnt;
         }
-        if (threadIdx.x == 0) A.tile_cnt[t] = total;
-        cta_count += total;
+        if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
     }
-    if (threadIdx.x == 0) A.cta_total[cta] = cta_count;
+    if (lane == 0) sm_warp[warp] = warp_total;
+    __threadfence();
+    __syncthreads();
+    int cta_count = 0;
+    if (warp == 0) {
+        int x = sm_warp[lane];
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(kFull, x, o);
+        if (lane == 0) { A.cta_total[cta] = x; sm_base = x; }
+    }
+    __syncthreads();
+    cta_count = sm_base;
     grid_barrier(A.ctl, A.G, ++barrier_no);
+    if (stamper) A.ctl->t_ns[4] = global_ns();
 
     // ------------------------------------------------------------------ P5b: final positions
     {
         int below = 0;
         for (int c = threadIdx.x; c < cta; c += kThreads) below += ld_cg(A.cta_total + c);
-        RedOut r = block_sum(0.0, 0.0, 0.0, below, sm_red);
+        Sums r = block_tree(0.0, 0.0, below, sm_red);
         if (threadIdx.x == 0) sm_base = r.n;
         __syncthreads();
-        int pos = sm_base;
-        if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = pos + cta_count;
-        for (int t = t_begin; t < t_end; ++t) {
-            const int cnt = A.tile_cnt[t];
-            const int lo = A.tile_start[t];
-            for (int i = threadIdx.x; i < cnt; i += kThreads) {
-                A.out_idx[pos + i] = A.stage_idx[lo + i];
-                A.out_val[pos + i] = A.stage_val[lo + i];
+        int run_base = sm_base;
+        if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
+        // chunk bases by a block-wide exclusive scan, kThreads chunks at a time
+        for (int pass = c0; pass < c1; pass += kThreads) {
+            const int c = pass + (int)threadIdx.x;
+            const int cnt = c < c1 ? ld_cg(A.chunk_cnt + c) : 0;
+            int incl = cnt;
+            #pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += t;
             }
-            pos += cnt;
+            __syncthreads();
+            if (lane == 31) sm_warp[warp] = incl;
+            __syncthreads();
+            if (warp == 0) {
+                int w = sm_warp[lane];
+                #pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(kFull, w, o);
+                    if (lane >= o) w += t;
+                }
+                sm_warp[lane] = w;          // inclusive over warps
+            }
+            __syncthreads();
+            const int warp_off = warp ? sm_warp[warp - 1] : 0;
+            const int pass_total = sm_warp[kWarps - 1];
+            sm_scan[threadIdx.x] = run_base + warp_off + incl - cnt;     // exclusive base of chunk c
+            sm_list[threadIdx.x] = cnt;
+            __syncthreads();
+            const int n_here = min(kThreads, c1 - pass);
+            for (int i = warp; i < n_here; i += kWarps) {
+                const int n = sm_list[i];
+                if (n == 0) continue;
+                const int src = __ldg(A.chunk_start + pass + i);
+                const int dst = sm_scan[i];
+                for (int t = lane; t < n; t += 32) {
+                    A.out_idx[dst + t] = ld_cg(A.stage_idx + src + t);
+                    A.out_val[dst + t] = ld_cg(A.stage_val + src + t);
+                }
+            }
+            run_base += pass_total;
+            __syncthreads();
         }
     }
     // per-segment counts, last stage count, adaptation (Algorithm 1, Adapt_Stages)
-    for (int s = cta; s < A.S; s += A.G) {
-        const int t0 = A.seg_tile0[s], t1 = A.seg_tile0[s + 1];
-        int k = 0;
-        for (int t = t0 + (int)threadIdx.x; t < t1; t += kThreads) k += ld_cg(A.tile_cnt + t);
-        RedOut r = block_sum(0.0, 0.0, 0.0, k, sm_red);
-        if (threadIdx.x == 0) {
-            SegDev* sg = &A.seg[s];
-            const int k_hat = r.n;
-            A.out_k[s] = k_hat;
-            sg->k_stage[ld_cg(&sg->M_eff) - 1] = k_hat;
-            if (ld_volatile(&A.ctl->timeout)) sg->status = ld_cg(&sg->status) | kStTimeout;
-            if (A.max_stages > 0) {
-                int calls = sg->calls + 1;
-                long long k_sum = sg->k_sum + k_hat;
-                if (calls % A.Q == 0) {
-                    const double k_avg = (double)k_sum / (double)A.Q;
-                    const double k_target = A.delta * (double)A.seg_n[s];
-                    int M = sg->M;
-                    if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
-                    if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
-                    if (M < 1) M = 1;
-                    if (M > A.max_stages) M = A.max_stages;
-                    sg->M = M;
-                    k_sum = 0;
-                }
-                sg->calls = calls;
-                sg->k_sum = k_sum;
+    for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads) {
+        SegDev* sg = &A.seg[s];
+        const int k_hat = ld_cg(&sg->k_acc);
+        sg->k_acc = 0;
+        A.out_k[s] = k_hat;
+        sg->k_stage[ld_cg(&sg->M_eff) - 1] = k_hat;
+        if (ld_volatile(&A.ctl->timeout)) sg->status = ld_cg(&sg->status) | kStTimeout;
+        if (A.max_stages > 0) {
+            const int calls = sg->calls + 1;
+            long long k_sum = sg->k_sum + k_hat;
+            if (calls % A.Q == 0) {
+                const double k_avg = (double)k_sum / (double)A.Q;
+                const double k_target = A.delta * (double)A.seg_n[s];
+                int M = sg->M;
+                if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
+                if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
+                if (M < 1) M = 1;
+                if (M > A.max_stages) M = A.max_stages;
+                sg->M = M;
+                k_sum = 0;
             }
+            sg->calls = calls;
+            sg->k_sum = k_sum;
         }
     }
 
     // last CTA out resets the control block for the next call
     __syncthreads();
     if (threadIdx.x == 0) {
+        if (stamper) A.ctl->t_ns[5] = global_ns();
         __threadfence();
         const unsigned done = atomicAdd(&A.ctl->finished, 1u);
         if (done == (unsigned)A.G - 1u) {

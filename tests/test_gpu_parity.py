@@ -156,7 +156,7 @@ def test_nan_and_inf_segments_select_nothing(sid):
 
 def test_thresholds_independent_of_grid_size():
     """Deterministic two-level combine: the same input gives bit-identical thresholds whatever the
-    number of CTAs (checked by running in a child process with fewer CTAs per SM)."""
+    number of CTAs (checked by running child processes with smaller grids)."""
     import json
     import os
     import subprocess
@@ -172,8 +172,8 @@ out = run.step(wl.draw(0), f32(0.001), 1, -3)
 print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [out["idx"][:50].tolist(), int(out["out_k"][-1])]))
 ''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
     outs = []
-    for ctas in ("1", "3", "8"):
-        env = dict(os.environ, SIDCO_CTAS_PER_SM=ctas)
+    for grid in ("100000", "37", "5"):
+        env = dict(os.environ, SIDCO_GRID=grid)
         r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
         assert r.returncode == 0, r.stderr[-2000:]
         outs.append(json.loads(r.stdout.strip().splitlines()[-1]))
