@@ -37,7 +37,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_chunk0;
-    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, cand, cta_dir, seg, ctl;
     size_t total;
 };
 
@@ -60,6 +60,8 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
     L.stage_val = take(sizeof(float) * (size_t)(d + 4));
     L.cta_total = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.cand = take(32 * (size_t)(T + 1));
+    L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
     L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
     L.ctl = take(sizeof(Control));
     L.total = o;
@@ -245,6 +247,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.cta_chunk0, cta_chunk0.data(), sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
 
@@ -290,6 +293,8 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.stage_idx = (int32_t*)(base + L.stage_idx);
     a.stage_val = (float*)(base + L.stage_val);
     a.cta_total = (int32_t*)(base + L.cta_total);
+    a.cand = (unsigned char*)(base + L.cand);
+    a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.seg = (SegDev*)(base + L.seg);
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;
@@ -303,6 +308,9 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.S = c->S;
     a.G = c->G;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
+    // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
+    static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
+    a.spec_enable = spec_on ? 1 : 0;
 
     void* kargs[] = {(void*)&a};
     const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>

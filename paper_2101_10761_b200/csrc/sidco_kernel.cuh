@@ -11,7 +11,12 @@
 //
 //   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
 //       of every chunk; the CTA whose run completes a segment sums the per-chunk
-//       partials in chunk order and fits eta_1 (Corollaries 1.1-1.3)
+//       partials in chunk order and fits eta_1 (Corollaries 1.1-1.3).  For
+//       single-stage segments the sweep also records, per lane and 4-element
+//       slot, whether some |x| >= tau, tau being 0.8 times the segment's threshold
+//       of the previous call: if the new eta turns out >= tau (checked per segment)
+//       P5a fetches only the flagged slots of acc instead of all of it; otherwise
+//       it reads all of acc, so the result never depends on tau
 //   P3  (only if some segment uses M >= 2) exceedances |x| > eta_1 compacted, in
 //       order, into the chunk's side region together with the statistics of the
 //       shifted peaks (Lemma 2 / Corollary 2.1); fit of eta_2
@@ -37,6 +42,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 1024;                      // window: elements per full chunk (one warp)
 constexpr int kSlots = kChunk / 128;              // float4 slots per lane per chunk (8)
 constexpr int kSmallSeg = 32;                     // segments of <= 32 chunks are summed by one warp
+constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr long long kSpinLimit = 1ll << 22;       // bounded waits: ~1 s with the back-off below
@@ -57,6 +63,8 @@ struct SegDev {
     int32_t M;           // adaptation state: stage count for the next adaptive call
     int32_t calls;
     long long k_sum;
+    float spec_thr;      // candidate threshold for the next call's first sweep (<= 0: none), see P1
+    int32_t pad;
 };
 
 struct Control {
@@ -90,6 +98,8 @@ struct Args {
     int32_t* stage_idx;          // [d]
     float* stage_val;            // [d]
     int32_t* cta_total;          // [G]
+    unsigned char* cand;         // [C][32] per-lane slot flags of full chunks: slot may hold a survivor
+    int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
     SegDev* seg;                 // [S]
     Control* ctl;
     // scalars
@@ -97,6 +107,7 @@ struct Args {
     int Q, sid, max_stages;
     int C, S, G;
     int vec_ok;                  // grad and residual are 16-byte aligned
+    int spec_enable;             // candidate pre-selection in the first sweep (see P1)
 };
 
 // ----------------------------------------------------------------------------
@@ -339,12 +350,12 @@ __device__ __forceinline__ unsigned load_chunk(const float* __restrict__ src, in
 
 // Warp-ordered emission: calls emit(position, j, c) for every set bit of `mask`, positions counted
 // in chunk order starting at `base`.  Returns the number of set bits in the warp.
-template <class Emit>
+template <int NS = kSlots, class Emit>
 __device__ __forceinline__ int ordered_emit(unsigned mask, int base, Emit emit) {
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
     int run = base;
     #pragma unroll
-    for (int j = 0; j < kSlots; ++j) {
+    for (int j = 0; j < NS; ++j) {
         const unsigned nib = (mask >> (4 * j)) & 0xFu;
         if (__ballot_sync(kFull, nib != 0) == 0) continue;
         const int c = __popc(nib);
@@ -389,6 +400,41 @@ struct ChunkQueue {
         return descending ? c1 - 1 - k : c0 + k;
     }
 };
+
+// Chunk descriptor, fetched one chunk ahead so that its loads overlap the current chunk's work.
+struct Desc {
+    int c, seg, lo, hi, side_n;
+    unsigned flags;      // this lane's candidate slot flags (P5a only)
+};
+
+__device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side, bool with_flags = false) {
+    Desc d{c, 0, 0, 0, 0, 0u};
+    if (c >= 0) {
+        d.seg = __ldg(A.chunk_seg + c);
+        d.lo = __ldg(A.chunk_start + c);
+        d.hi = __ldg(A.chunk_start + c + 1);
+        if (with_side) d.side_n = ld_cg(A.side_cnt + c);
+        if (with_flags) d.flags = __ldcg(A.cand + (size_t)c * 32 + (threadIdx.x & 31));
+    }
+    return d;
+}
+
+// Load only the flagged float4 slots of a full chunk of acc; the others read as zero.
+__device__ __forceinline__ unsigned load_flagged(const float* __restrict__ src, int wb, unsigned flags,
+                                                 float (&v)[kSlots][4]) {
+    const int e0 = wb + (threadIdx.x & 31) * 4;
+    unsigned valid = 0;
+    #pragma unroll
+    for (int j = 0; j < kSlots; ++j) {
+        v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0.0f;
+        if (flags & (1u << j)) {
+            const float4 q = ld_l2_4(src + e0 + j * 128);
+            v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
+            valid |= 0xFu << (4 * j);
+        }
+    }
+    return valid;
+}
 
 // ----------------------------------------------------------------------------
 // end of a statistics phase: arrivals and fits for the segments of this CTA's run
@@ -477,111 +523,142 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ int sm_count;
     __shared__ int sm_next;
     __shared__ int sm_base;
+    __shared__ int sm_resweep;
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c0 = A.cta_chunk0[cta], c1 = A.cta_chunk0[cta + 1];
     const bool vec_ok = A.vec_ok != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
+    const int cap = stage_cap(A.delta, A.delta1);
     int barrier_no = 0;
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
-    if (threadIdx.x == 0) sm_next = 0;
+    if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; }
+    // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
+    // of the last call) ended, so that it begins on the lines most recently left in L2.
+    const bool p1_desc = A.cta_dir[cta] != 0;
+    int resweep = 0;             // chunks of acc this warp read a second time in full
 
     // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
         if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], 0, 0.0, 0.0, 0);
     __syncthreads();
 
-    // ------------------------------------------------------------------ P1
-    // Descending chunk order: the chunks touched last are the ones P3/P5a read first, which
-    // raises the share of acc that is still in L2 when it is read again.
-    for (int c = queue.next(true); c >= 0; c = queue.next(true)) {
-        const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
-        const int wb = lo & ~(kChunk - 1);
-        const int e0 = wb + lane * 4;
-
-        double s1 = 0.0, s2 = 0.0, prod = 1.0;
-        int esum = 0, nnz = 0;
-        auto accumulate = [&](float x) {
-            const float a = fabsf(x);
-            const double ad = (double)a;
-            s1 += ad;
-            if (SID == kSidGpd) s2 = fma(ad, ad, s2);
-            if (SID == kSidGamma) {
-                if (a > 0.0f) {
-                    // log|x| = exponent * ln 2 + log(mantissa): exponents are summed as integers,
-                    // mantissas multiplied in fp64, one log per chunk.
-                    const long long bits = __double_as_longlong(ad);
-                    esum += (int)(bits >> 52) - 1023;
-                    prod *= __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
-                    ++nnz;
-                }
-            }
-        };
-
-        if (vec_ok && lo == wb && hi == wb + kChunk) {
-            #pragma unroll
-            for (int b = 0; b < kSlots; b += 4) {
-                float4 g4[4], r4[4];
-                #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    g4[j] = ld_stream4(A.grad + e0 + (b + j) * 128);
-                    r4[j] = *reinterpret_cast<const float4*>(A.residual + e0 + (b + j) * 128);
-                }
-                #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    float4 a4;
-                    a4.x = g4[j].x + r4[j].x; a4.y = g4[j].y + r4[j].y;
-                    a4.z = g4[j].z + r4[j].z; a4.w = g4[j].w + r4[j].w;
-                    *reinterpret_cast<float4*>(A.residual + e0 + (b + j) * 128) = a4;
-                    accumulate(a4.x); accumulate(a4.y); accumulate(a4.z); accumulate(a4.w);
-                }
-            }
+    // Candidate threshold of a segment for this call: only single-stage segments use one.  It depends
+    // on state the previous call left behind, so every warp and every phase derives the same value.
+    auto spec_tau = [&](int seg) -> float {
+        if (!A.spec_enable) return -1.0f;
+        const SegDev* sg = &A.seg[seg];
+        int M;
+        if (A.max_stages > 0) {
+            M = sg->M < 1 ? 1 : sg->M;
+            if (M > A.max_stages) M = A.max_stages;
         } else {
-            #pragma unroll 1
-            for (int j = 0; j < kSlots; ++j) {
-                const int e = e0 + j * 128;
-                if (e + 4 <= lo || e >= hi) continue;
-                if (vec_ok && e >= lo && e + 4 <= hi) {
-                    const float4 g = ld_stream4(A.grad + e);
-                    const float4 r = *reinterpret_cast<const float4*>(A.residual + e);
-                    float4 a4;
-                    a4.x = g.x + r.x; a4.y = g.y + r.y; a4.z = g.z + r.z; a4.w = g.w + r.w;
-                    *reinterpret_cast<float4*>(A.residual + e) = a4;
-                    accumulate(a4.x); accumulate(a4.y); accumulate(a4.z); accumulate(a4.w);
-                } else {
-                    for (int cc = 0; cc < 4; ++cc) {
-                        if (e + cc >= lo && e + cc < hi) {
-                            const float a = __ldcs(A.grad + e + cc) + A.residual[e + cc];
-                            A.residual[e + cc] = a;
-                            accumulate(a);
+            M = -A.max_stages;
+        }
+        if ((M < cap ? M : cap) != 1) return -1.0f;
+        const float tau = sg->spec_thr;
+        return tau > 0.0f ? tau : -1.0f;
+    };
+
+    // ------------------------------------------------------------------ P1
+    {
+        int tau_seg = -1;
+        float tau = -1.0f;
+        Desc cur = fetch_desc(A, queue.next(p1_desc), false);
+        while (cur.c >= 0) {
+            const Desc nxt = fetch_desc(A, queue.next(p1_desc), false);
+            const int c = cur.c, lo = cur.lo, hi = cur.hi;
+            const int wb = lo & ~(kChunk - 1);
+            const int e0 = wb + lane * 4;
+            if (cur.seg != tau_seg) { tau_seg = cur.seg; tau = spec_tau(cur.seg); }
+            unsigned flags = 0;
+
+            double s1 = 0.0, s2 = 0.0, prod = 1.0;
+            int esum = 0, nnz = 0;
+            auto accumulate = [&](float x) {
+                const float a = fabsf(x);
+                const double ad = (double)a;
+                s1 += ad;
+                if (SID == kSidGpd) s2 = fma(ad, ad, s2);
+                if (SID == kSidGamma) {
+                    if (a > 0.0f) {
+                        // log|x| = exponent * ln 2 + log(mantissa): exponents are summed as integers,
+                        // mantissas multiplied in fp64, one log per chunk.
+                        const long long bits = __double_as_longlong(ad);
+                        esum += (int)(bits >> 52) - 1023;
+                        prod *= __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
+                        ++nnz;
+                    }
+                }
+            };
+
+            if (vec_ok && lo == wb && hi == wb + kChunk) {
+                #pragma unroll
+                for (int b = 0; b < kSlots; b += 4) {
+                    float4 g4[4], r4[4];
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        g4[j] = ld_stream4(A.grad + e0 + (b + j) * 128);
+                        r4[j] = *reinterpret_cast<const float4*>(A.residual + e0 + (b + j) * 128);
+                    }
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        r4[j].x += g4[j].x; r4[j].y += g4[j].y; r4[j].z += g4[j].z; r4[j].w += g4[j].w;
+                        *reinterpret_cast<float4*>(A.residual + e0 + (b + j) * 128) = r4[j];
+                        accumulate(r4[j].x); accumulate(r4[j].y); accumulate(r4[j].z); accumulate(r4[j].w);
+                        const float big = fmaxf(fmaxf(fabsf(r4[j].x), fabsf(r4[j].y)),
+                                                fmaxf(fabsf(r4[j].z), fabsf(r4[j].w)));
+                        flags |= (unsigned)(big >= tau) << (b + j);
+                    }
+                }
+                if (tau > 0.0f) A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
+            } else {
+                #pragma unroll 1
+                for (int j = 0; j < kSlots; ++j) {
+                    const int e = e0 + j * 128;
+                    if (e + 4 <= lo || e >= hi) continue;
+                    if (vec_ok && e >= lo && e + 4 <= hi) {
+                        const float4 g = ld_stream4(A.grad + e);
+                        float4 r = *reinterpret_cast<const float4*>(A.residual + e);
+                        r.x += g.x; r.y += g.y; r.z += g.z; r.w += g.w;
+                        *reinterpret_cast<float4*>(A.residual + e) = r;
+                        accumulate(r.x); accumulate(r.y); accumulate(r.z); accumulate(r.w);
+                    } else {
+                        for (int cc = 0; cc < 4; ++cc) {
+                            if (e + cc >= lo && e + cc < hi) {
+                                const float a = __ldcs(A.grad + e + cc) + A.residual[e + cc];
+                                A.residual[e + cc] = a;
+                                accumulate(a);
+                            }
                         }
                     }
                 }
             }
-        }
 
-        // per-chunk partials with a fixed shuffle tree
-        double second = s2;
-        if (SID == kSidGamma) {
-            // normalise the per-lane product, multiply the mantissas across the warp, one log:
-            // SL_chunk = (sum of exponents) * ln 2 + log(product of mantissas)
-            const long long bits = __double_as_longlong(prod);
-            esum += (int)(bits >> 52) - 1023;
-            double m = __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
-            #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                m *= __shfl_down_sync(kFull, m, o);
-                esum += __shfl_down_sync(kFull, esum, o);
+            // per-chunk partials with a fixed shuffle tree
+            double second = s2;
+            if (SID == kSidGamma) {
+                // normalise the per-lane product, multiply the mantissas across the warp, one log:
+                // SL_chunk = (sum of exponents) * ln 2 + log(product of mantissas)
+                const long long bits = __double_as_longlong(prod);
+                esum += (int)(bits >> 52) - 1023;
+                double m = __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
+                #pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    m *= __shfl_down_sync(kFull, m, o);
+                    esum += __shfl_down_sync(kFull, esum, o);
+                }
+                second = (double)esum * 0.693147180559945309417232121458 + log(m);   // used from lane 0 only
             }
-            second = (double)esum * 0.693147180559945309417232121458 + log(m);   // used from lane 0 only
-        }
-        Sums r = warp_tree(s1, SID == kSidGamma ? 0.0 : second, nnz);
-        if (lane == 0) {
-            A.part[3 * (size_t)c + 0] = r.a;
-            A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
-            A.part_n[c] = r.n;
+            Sums r = warp_tree(s1, SID == kSidGamma ? 0.0 : second, nnz);
+            if (lane == 0) {
+                A.part[3 * (size_t)c + 0] = r.a;
+                A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
+                A.part_n[c] = r.n;
+            }
+            cur = nxt;
         }
     }
     arrive_and_fit(A, c0, c1, 0, sm_list, &sm_count, sm_red);
@@ -592,42 +669,49 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // ------------------------------------------------------------------ P3: stage 2 from acc
     if (M_max_eff >= 2) {
-        SegView sv;
-        for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
-            sv.load(A, __ldg(A.chunk_seg + c), 0);
-            if (sv.M_eff < 2) continue;
-            const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
-            const int wb = lo & ~(kChunk - 1);
-            float v[kSlots][4];
-            const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, v);
-            unsigned mask = 0;
-            #pragma unroll
-            for (int j = 0; j < kSlots; ++j)
-                #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (4 * j + cc);
-            mask &= valid;
-            double sy = 0.0, sy2 = 0.0;
-            #pragma unroll
-            for (int j = 0; j < kSlots; ++j)
-                #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    if (mask & (1u << (4 * j + cc))) {
-                        const double y = (double)fabsf(v[j][cc]) - sv.eta_prev;
-                        sy += y;
-                        if (SID != kSidExp) sy2 = fma(y, y, sy2);
+        {
+            SegView sv;
+            Desc cur = fetch_desc(A, queue.next(!p1_desc), false);
+            while (cur.c >= 0) {
+                const Desc nxt = fetch_desc(A, queue.next(!p1_desc), false);
+                sv.load(A, cur.seg, 0);
+                if (sv.M_eff >= 2) {
+                    ++resweep;
+                    const int c = cur.c, lo = cur.lo, hi = cur.hi;
+                    const int wb = lo & ~(kChunk - 1);
+                    float v[kSlots][4];
+                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, v);
+                    unsigned mask = 0;
+                    #pragma unroll
+                    for (int j = 0; j < kSlots; ++j)
+                        #pragma unroll
+                        for (int cc = 0; cc < 4; ++cc)
+                            if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (4 * j + cc);
+                    mask &= valid;
+                    double sy = 0.0, sy2 = 0.0;
+                    #pragma unroll
+                    for (int j = 0; j < kSlots; ++j)
+                        #pragma unroll
+                        for (int cc = 0; cc < 4; ++cc)
+                            if (mask & (1u << (4 * j + cc))) {
+                                const double y = (double)fabsf(v[j][cc]) - sv.eta_prev;
+                                sy += y;
+                                if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                            }
+                    const int e0 = wb + lane * 4;
+                    const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                        A.side_idx[p] = e0 + j * 128 + cc;
+                        A.side_val[p] = v[j][cc];
+                    });
+                    Sums r = warp_tree(sy, sy2, 0);
+                    if (lane == 0) {
+                        A.part[3 * (size_t)c + 0] = r.a;
+                        A.part[3 * (size_t)c + 1] = r.b;
+                        A.part_n[c] = cnt;
+                        A.side_cnt[c] = cnt;
                     }
-            const int e0 = wb + lane * 4;
-            const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                A.side_idx[p] = e0 + j * 128 + cc;
-                A.side_val[p] = v[j][cc];
-            });
-            Sums r = warp_tree(sy, sy2, 0);
-            if (lane == 0) {
-                A.part[3 * (size_t)c + 0] = r.a;
-                A.part[3 * (size_t)c + 1] = r.b;
-                A.part_n[c] = cnt;
-                A.side_cnt[c] = cnt;
+                }
+                cur = nxt;
             }
         }
         arrive_and_fit(A, c0, c1, 1, sm_list, &sm_count, sm_red);
@@ -637,32 +721,38 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
         // -------------------------------------------------------------- P4: stages 3..M from the side regions
         for (int m = 2; m < M_max_eff; ++m) {
-            SegView sw;
-            for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
-                sw.load(A, __ldg(A.chunk_seg + c), m - 1);
-                if (sw.M_eff <= m) continue;
-                const int lo = __ldg(A.chunk_start + c);
-                const int wb = lo & ~(kChunk - 1);
-                const int hi = lo + ld_cg(A.side_cnt + c);
-                float v[kSlots][4];
-                const unsigned valid = load_chunk(A.side_val, lo, hi, wb, true, v);
-                double sy = 0.0, sy2 = 0.0;
-                int cnt = 0;
-                #pragma unroll
-                for (int j = 0; j < kSlots; ++j)
-                    #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc)
-                        if ((valid & (1u << (4 * j + cc))) && fabsf(v[j][cc]) > sw.thr_gt) {
-                            const double y = (double)fabsf(v[j][cc]) - sw.eta_prev;
-                            sy += y;
-                            if (SID != kSidExp) sy2 = fma(y, y, sy2);
-                            ++cnt;
+            {
+                SegView sw;
+                Desc cur = fetch_desc(A, queue.next(false), true);
+                while (cur.c >= 0) {
+                    const Desc nxt = fetch_desc(A, queue.next(false), true);
+                    sw.load(A, cur.seg, m - 1);
+                    if (sw.M_eff > m) {
+                        const int c = cur.c, lo = cur.lo;
+                        const int wb = lo & ~(kChunk - 1);
+                        const int hi = lo + cur.side_n;
+                        float v[kSlots][4];
+                        const unsigned valid = load_chunk(A.side_val, lo, hi, wb, true, v);
+                        double sy = 0.0, sy2 = 0.0;
+                        int cnt = 0;
+                        #pragma unroll
+                        for (int j = 0; j < kSlots; ++j)
+                            #pragma unroll
+                            for (int cc = 0; cc < 4; ++cc)
+                                if ((valid & (1u << (4 * j + cc))) && fabsf(v[j][cc]) > sw.thr_gt) {
+                                    const double y = (double)fabsf(v[j][cc]) - sw.eta_prev;
+                                    sy += y;
+                                    if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                                    ++cnt;
+                                }
+                        Sums r = warp_tree(sy, sy2, cnt);
+                        if (lane == 0) {
+                            A.part[3 * (size_t)c + 0] = r.a;
+                            A.part[3 * (size_t)c + 1] = r.b;
+                            A.part_n[c] = r.n;
                         }
-                Sums r = warp_tree(sy, sy2, cnt);
-                if (lane == 0) {
-                    A.part[3 * (size_t)c + 0] = r.a;
-                    A.part[3 * (size_t)c + 1] = r.b;
-                    A.part_n[c] = r.n;
+                    }
+                    cur = nxt;
                 }
             }
             arrive_and_fit(A, c0, c1, m, sm_list, &sm_count, sm_red);
@@ -676,47 +766,63 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     int warp_total = 0;
     {
         SegView sv;
+        bool seg_from_side = false, seg_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
-        for (int c = queue.next(false); c >= 0; c = queue.next(false)) {
-            const int s = __ldg(A.chunk_seg + c);
-            if (s != sv.seg) {
+        Desc cur = fetch_desc(A, queue.next(!p1_desc), true, true);
+        while (cur.c >= 0) {
+            const Desc nxt = fetch_desc(A, queue.next(!p1_desc), true, true);
+            if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
                 seg_count = 0;
+                sv.load(A, cur.seg, -1);
+                // multi-stage segments keep their exceedances in the side region; single-stage ones
+                // have valid candidate flags if the candidate threshold proved low enough
+                const float tau = spec_tau(cur.seg);
+                seg_from_side = sv.M_eff >= 2;
+                seg_flagged = !seg_from_side && tau > 0.0f && sv.thr_ge >= tau;
             }
-            sv.load(A, s, -1);
-            const bool from_side = sv.M_eff >= 2;
-            const int lo = __ldg(A.chunk_start + c);
+            const bool from_side = seg_from_side;
+            const int c = cur.c, lo = cur.lo;
             const int wb = lo & ~(kChunk - 1);
-            const int hi = from_side ? lo + ld_cg(A.side_cnt + c) : __ldg(A.chunk_start + c + 1);
-            float v[kSlots][4];
-            const unsigned valid = load_chunk(from_side ? A.side_val : A.residual, lo, hi, wb, from_side || vec_ok, v);
-            unsigned mask = 0;
-            #pragma unroll
-            for (int j = 0; j < kSlots; ++j)
-                #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
-            mask &= valid;
+            const int hi = from_side ? lo + cur.side_n : cur.hi;
+            const bool flagged = seg_flagged && vec_ok && lo == wb && hi == wb + kChunk;
             int cnt = 0;
-            if (__ballot_sync(kFull, mask != 0)) {
-                const int e0 = wb + lane * 4;
-                cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                    const int e = e0 + j * 128 + cc;
-                    const int idx = from_side ? ld_cg(A.side_idx + e) : e;
-                    A.stage_idx[p] = idx;
-                    A.stage_val[p] = v[j][cc];
-                    A.residual[idx] = 0.0f;
-                });
+            if (!from_side && !flagged) ++resweep;
+            if (hi > lo && !(flagged && __ballot_sync(kFull, cur.flags != 0) == 0)) {
+                float v[kSlots][4];
+                const unsigned valid = flagged ? load_flagged(A.residual, wb, cur.flags, v)
+                                               : load_chunk(from_side ? A.side_val : A.residual, lo, hi, wb,
+                                                            from_side || vec_ok, v);
+                unsigned mask = 0;
+                #pragma unroll
+                for (int j = 0; j < kSlots; ++j)
+                    #pragma unroll
+                    for (int cc = 0; cc < 4; ++cc)
+                        if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
+                mask &= valid;
+                if (__ballot_sync(kFull, mask != 0)) {
+                    const int e0 = wb + lane * 4;
+                    cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                        const int e = e0 + j * 128 + cc;
+                        const int idx = from_side ? ld_cg(A.side_idx + e) : e;
+                        A.stage_idx[p] = idx;
+                        A.stage_val[p] = v[j][cc];
+                        A.residual[idx] = 0.0f;
+                    });
+                }
             }
             if (lane == 0) A.chunk_cnt[c] = cnt;
             seg_count += cnt;
             warp_total += cnt;
+            cur = nxt;
         }
         if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
     }
-    if (lane == 0) sm_warp[warp] = warp_total;
+    if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
     __threadfence();
     __syncthreads();
+    // next call: start the first sweep where this call's last full sweep over acc ended
+    if (threadIdx.x == 0) A.cta_dir[cta] = (2 * sm_resweep >= c1 - c0) ? (p1_desc ? 1 : 0) : (p1_desc ? 0 : 1);
     int cta_count = 0;
     if (warp == 0) {
         int x = sm_warp[lane];
@@ -739,7 +845,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
         // chunk bases by a block-wide exclusive scan, kThreads chunks at a time
-        for (int pass = c0; pass < c1; pass += kThreads) {
+        for (int pass = c0; pass < c1 && cta_count > 0; pass += kThreads) {
             const int c = pass + (int)threadIdx.x;
             const int cnt = c < c1 ? ld_cg(A.chunk_cnt + c) : 0;
             int incl = cnt;
@@ -764,18 +870,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             const int warp_off = warp ? sm_warp[warp - 1] : 0;
             const int pass_total = sm_warp[kWarps - 1];
             sm_scan[threadIdx.x] = run_base + warp_off + incl - cnt;     // exclusive base of chunk c
-            sm_list[threadIdx.x] = cnt;
             __syncthreads();
+            // one thread per survivor: the owning chunk is the last one whose base is <= the position
             const int n_here = min(kThreads, c1 - pass);
-            for (int i = warp; i < n_here; i += kWarps) {
-                const int n = sm_list[i];
-                if (n == 0) continue;
-                const int src = __ldg(A.chunk_start + pass + i);
-                const int dst = sm_scan[i];
-                for (int t = lane; t < n; t += 32) {
-                    A.out_idx[dst + t] = ld_cg(A.stage_idx + src + t);
-                    A.out_val[dst + t] = ld_cg(A.stage_val + src + t);
+            for (int p = threadIdx.x; p < pass_total; p += kThreads) {
+                const int pos = run_base + p;
+                int a = 0, b = n_here;
+                while (a < b) {
+                    const int mid = (a + b) >> 1;
+                    if (sm_scan[mid] <= pos) a = mid + 1; else b = mid;
                 }
+                const int i = a - 1;
+                const int src = __ldg(A.chunk_start + pass + i) + (pos - sm_scan[i]);
+                A.out_idx[pos] = ld_cg(A.stage_idx + src);
+                A.out_val[pos] = ld_cg(A.stage_val + src);
             }
             run_base += pass_total;
             __syncthreads();
@@ -806,6 +914,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             sg->calls = calls;
             sg->k_sum = k_sum;
         }
+        // candidate threshold for the next call's first sweep
+        const float thr = ld_cg(&sg->thr_ge);
+        sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
     }
 
     // last CTA out resets the control block for the next call

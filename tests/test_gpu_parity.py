@@ -117,6 +117,33 @@ def test_unaligned_offsets_and_pointers(sid, base_shift):
 
 
 @pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("max_stages", [-1, 2])
+def test_threshold_jumps_between_calls(sid, max_stages):
+    """Single-stage segments pre-select candidates against a fraction of the previous call's threshold.
+    Gradients that cancel the residual and shrink (or blow up) the scale by 1000x make the new
+    threshold fall far below (or above) that guess; the output must not depend on it."""
+    sizes = [30000, 5, 70001, 12000]
+    off = W.offsets_from_sizes(sizes)
+    d = int(off[-1])
+    delta = f32(0.01)
+    run = GpuRun(off)
+    res_o = np.zeros(d, np.float32)
+    state = O.new_state(len(sizes)) if max_stages > 0 else None
+    scales = [1.0, 1e-3, 1e-3, 1.0, 1e3, 1e-3, 1.0]
+    try:
+        for call, sc in enumerate(scales):
+            g = (sc * W.ragged_case(700 + call, sizes, 1e-2)).astype(np.float32)
+            if call in (1, 5):
+                g = (g - res_o).astype(np.float32)      # acc becomes the small fresh draw alone
+            ora = O.sidco_compress(g, res_o, off, delta, sid, max_stages, state=state)
+            gpu = run.step(g, delta, sid, max_stages)
+            assert check_parity(gpu, ora, off, state) == 0
+            res_o = ora.residual
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("sid", SIDS)
 @pytest.mark.parametrize("M", [1, 2, 3])
 def test_degenerate_segments(sid, M):
     sizes = [0, 5000, 7000, 1, 6, 3000]
