@@ -44,9 +44,12 @@ def schedule():
     from paper_2101_10761_b200 import workloads as W
     return [k if sgn > 0 else N_DRAWS + k for k, sgn in W.signed_walk(N_DRAWS, WALK_LEN)]
 
-# DRAM bytes per launch of the persistent kernel on this workload, from the ncu capture
-# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes per launch of the persistent kernel on this workload (dram__bytes_read.sum +
+# dram__bytes_write.sum of one ncu capture, summarised under profiles/), keyed by (sid, max_stages).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    (0, 4): 380.4e6,     # EXP, adaptive: every segment at M = 4 in steady state
+    (0, -1): 261.0e6,    # EXP, single stage
+}
 
 
 def measured_peaks():
@@ -217,6 +220,19 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def reduce_over_ranks(dist, device, times_ms, totals):
+    """Replicas only: every rank ran the same work on its own GPU.  The job's time is the MAX over
+    ranks of each entry of times_ms, the job's work the SUM over ranks of each entry of totals."""
+    if dist is None:
+        return list(times_ms), list(totals)
+    import torch
+    tmax = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    tsum = torch.tensor(list(totals), dtype=torch.float64, device=device)
+    dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+    return [float(x) for x in tmax], [float(x) for x in tsum]
+
+
 def run_gpu(args):
     import torch
     from paper_2101_10761_b200 import binding as B
@@ -296,6 +312,34 @@ def run_gpu(args):
         status_or |= sd.status
     i += args.steps
 
+    # ---- context: other SID / stage settings on the same workload (rank 0, short runs) -------
+    variants = {}
+    if rank == 0 and not args.no_variants:
+        res_v = torch.zeros(d, dtype=torch.float32, device=dev)
+        for v_sid, v_ms in ((0, -1), (1, -1), (2, -1), (0, -2), (1, 4), (2, 4)):
+            if (v_sid, v_ms) == (args.sid, args.max_stages):
+                continue
+            res_v.zero_()
+            for w in range(60):
+                B.sidco_compress(grads[SCHED[w % WALK_LEN]], res_v, off, DELTA, v_sid, v_ms, out_idx, out_val, out_k)
+            v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_v = 200
+            torch.cuda.synchronize()
+            v0.record()
+            for w in range(n_v):
+                B.sidco_compress(grads[SCHED[(60 + w) % WALK_LEN]], res_v, off, DELTA, v_sid, v_ms,
+                                 out_idx, out_val, out_k)
+            v1.record()
+            torch.cuda.synchronize()
+            us = v0.elapsed_time(v1) / n_v * 1e3
+            kh = int(out_k[S].item())
+            name = f"{SID_NAMES[v_sid]}_{'adaptive' + str(v_ms) if v_ms > 0 else 'M' + str(-v_ms)}"
+            variants[name] = {"us_per_step": round(us, 2), "GBps_min_bytes": round((12 * d + 8 * kh) / us / 1e3, 1),
+                              "frac_of_peak": round((12 * d + 8 * kh) / us / 1e3 / measured_peaks()[0], 4),
+                              "k_hat_last": kh}
+            B.sidco_release(res_v)
+        del res_v
+
     # ---- end to end: pinned host buffers through sidco_compress_host ----------------------
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     h_grads = [torch.from_numpy(g).pin_memory() for g in grads_h]
@@ -322,15 +366,8 @@ def run_gpu(args):
     sampler.stop()
 
     # ---- max over ranks, totals over ranks -------------------------------------------------
-    t_dev, t_e2e = total_ms, e2e_ms
-    tot_bytes, tot_e2e_bytes, tot_elems = bytes_min, e2e_bytes_min, d * args.steps
-    if dist is not None:
-        tmax = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        t_dev, t_e2e = float(tmax[0]), float(tmax[1])
-        tsum = torch.tensor([bytes_min, e2e_bytes_min, tot_elems], dtype=torch.float64, device=dev)
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        tot_bytes, tot_e2e_bytes, tot_elems = float(tsum[0]), float(tsum[1]), float(tsum[2])
+    (t_dev, t_e2e), (tot_bytes, tot_e2e_bytes, tot_elems) = reduce_over_ranks(
+        dist, dev, [total_ms, e2e_ms], [bytes_min, e2e_bytes_min, d * args.steps])
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
@@ -355,7 +392,8 @@ def run_gpu(args):
             "pct_of_8TBs_on_min_bytes": 100.0 * value / world / 8000.0,
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "peak_kind": "of " + peak_kind,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.sid, args.max_stages)),
                 "kernel": "sidco_persistent_kernel", "kernel_avg_ms": kern_avg_ms,
                 "kernel_min_ms": min(kern_ms), "algorithmic_bytes_per_launch": alg_bytes,
             },
@@ -368,6 +406,7 @@ def run_gpu(args):
                 "h2d_bytes_per_step": 8 * d, "d2h_bytes_per_step": d2h // e2e_steps, "steps": e2e_steps,
                 "ms_per_step": t_e2e / e2e_steps,
             },
+            "variants": variants,
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
         }
@@ -387,6 +426,7 @@ def main():
     ap.add_argument("--max-stages", type=int, default=4, help=">0 adaptive up to this many stages, <0 fixed")
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--no-variants", action="store_true", help="skip the short runs of other SID/stage settings")
     ap.add_argument("--prewarm-ms", type=float, default=300.0,
                     help="untimed steps run for this long before the warm-up to bring the clocks up")
     args = ap.parse_args()

@@ -139,8 +139,17 @@ int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);
 /* Phase breakdown of the last call in microseconds, from device timestamps taken by one CTA at the
  * grid-wide barriers: us_out[0] error compensation + stage-1 statistics and fit, [1] stage-2 side-buffer
  * compaction and fit, [2] stages 3..M, [3] survivor staging + residual zeroing, [4] final placement and
- * adaptation, [5] whole kernel.  Synchronises the device; for profiling. */
+ * adaptation, [5] whole kernel; then finer marks of that CTA alone: [6] its first sweep, [7] its arrivals
+ * and fits after it, [8] its stage-2 sweep, [9] arrivals and fits after it, [10] arrivals and fits of the
+ * last refit stage, [11] its survivor staging sweep.  us_out has room for 12 values.  Entries of phases
+ * the call did not run are meaningless.  Synchronises the device; for profiling. */
 int sidco_get_phase_times(const float* residual, double* us_out);
+
+/* Per-CTA view of the last call, for load-balance studies: us_out[4*i + p] is the time (microseconds
+ * after the kernel's first CTA started) at which CTA i finished its sweep of phase p (0 first sweep,
+ * 1 stage-2 sweep, 2 last refit sweep, 3 survivor staging).  Writes at most max_ctas rows and returns
+ * the number of rows written (>= 0) or an error code (< 0).  Synchronises the device. */
+int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_ctas);
 
 /* Checkpointing of the adaptation state (Algorithm 1 keeps M and the running k_hat sum across
  * iterations): host blobs of 3 int64 per segment (M, calls, k_sum).  Both synchronise the device. */

@@ -38,7 +38,7 @@ EXPORTS = [
     "sidco_compress", "sidco_compress_host", "sidco_workspace_bytes", "sidco_set_workspace",
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
-    "sidco_get_phase_times",
+    "sidco_get_phase_times", "sidco_get_cta_sweep_times",
 ]
 
 _lib = None
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
     L.sidco_get_debug.restype = i32
     L.sidco_get_phase_times.argtypes = [vp, C.POINTER(dbl)]
     L.sidco_get_phase_times.restype = i32
+    L.sidco_get_cta_sweep_times.argtypes = [vp, C.POINTER(dbl), i32]
+    L.sidco_get_cta_sweep_times.restype = i32
     L.sidco_state_save.argtypes = [vp, C.POINTER(i64), i32]
     L.sidco_state_save.restype = i32
     L.sidco_state_load.argtypes = [vp, C.POINTER(i64), i32]
@@ -212,9 +214,19 @@ def sidco_error_string(code: int) -> str:
 
 
 def sidco_get_phase_times(residual):
-    """Microseconds of the last call: [P1, stage 2, stages 3..M, staging, placement, total]."""
-    buf = (C.c_double * 6)()
+    """Microseconds of the last call: [P1, stage 2, stages 3..M, staging, placement, total] followed by
+    six finer marks of CTA 0 (see sidco.h)."""
+    buf = (C.c_double * 12)()
     rc = lib().sidco_get_phase_times(_ptr(residual), buf)
     if rc:
         raise SidcoError(rc, "sidco_get_phase_times")
     return list(buf)
+
+
+def sidco_get_cta_sweep_times(residual, max_ctas: int = 1024) -> np.ndarray:
+    """(n_ctas, 4) array: microseconds after kernel start at which each CTA finished its sweeps."""
+    buf = (C.c_double * (4 * max_ctas))()
+    rc = lib().sidco_get_cta_sweep_times(_ptr(residual), buf, max_ctas)
+    if rc < 0:
+        raise SidcoError(rc, "sidco_get_cta_sweep_times")
+    return np.ctypeslib.as_array(buf)[: 4 * rc].reshape(rc, 4).copy()

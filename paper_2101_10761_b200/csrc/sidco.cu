@@ -37,7 +37,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_chunk0;
-    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, cand, cta_dir, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, cand, cta_dir, cta_ns, seg, ctl;
     size_t total;
 };
 
@@ -62,6 +62,7 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.cta_total = take(sizeof(int32_t) * (size_t)(G + 1));
     L.cand = take(32 * (size_t)(T + 1));
     L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.cta_ns = take(sizeof(unsigned long long) * 4 * (size_t)(G + 1));
     L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
     L.ctl = take(sizeof(Control));
     L.total = o;
@@ -295,6 +296,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.cta_total = (int32_t*)(base + L.cta_total);
     a.cand = (unsigned char*)(base + L.cand);
     a.cta_dir = (int32_t*)(base + L.cta_dir);
+    a.cta_ns = (unsigned long long*)(base + L.cta_ns);
     a.seg = (SegDev*)(base + L.seg);
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;
@@ -493,9 +495,35 @@ int sidco_get_phase_times(const float* residual, double* us_out) {
     Control ctl;
     if ((e = cudaMemcpy(&ctl, (char*)c->ws + c->L.ctl, sizeof(Control), cudaMemcpyDeviceToHost)) != cudaSuccess)
         return (int)e;
-    for (int i = 0; i < 5; ++i) us_out[i] = (double)(long long)(ctl.t_ns[i + 1] - ctl.t_ns[i]) * 1e-3;
-    us_out[5] = (double)(long long)(ctl.t_ns[5] - ctl.t_ns[0]) * 1e-3;
+    auto us = [&](int a, int b) { return (double)(long long)(ctl.t_ns[b] - ctl.t_ns[a]) * 1e-3; };
+    for (int i = 0; i < 5; ++i) us_out[i] = us(i, i + 1);
+    us_out[5] = us(0, 5);
+    us_out[6] = us(0, 6);      // first sweep of CTA 0 alone
+    us_out[7] = us(6, 7);      // its arrivals and fits
+    us_out[8] = us(1, 8);      // stage-2 sweep of CTA 0 alone (meaningless if no segment used M >= 2)
+    us_out[9] = us(8, 9);
+    us_out[10] = us(10, 11);   // arrivals and fits of the last refit stage
+    us_out[11] = us(4, 12) < 0 ? us(3, 12) : us(3, 12);   // survivor staging sweep of CTA 0 alone
     return 0;
+}
+
+int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_ctas) {
+    if (!us_out) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    Context* c = it->second;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    Control ctl;
+    std::vector<unsigned long long> ns(4 * (size_t)c->G);
+    if ((e = cudaMemcpy(&ctl, (char*)c->ws + c->L.ctl, sizeof(Control), cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return (int)e;
+    if ((e = cudaMemcpy(ns.data(), (char*)c->ws + c->L.cta_ns, ns.size() * 8, cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return (int)e;
+    const int n = c->G < max_ctas ? c->G : max_ctas;
+    for (int i = 0; i < 4 * n; ++i) us_out[i] = (double)(long long)(ns[i] - ctl.t_ns[0]) * 1e-3;
+    return n;
 }
 
 int sidco_state_save(const float* residual, int64_t* blob, int n_segs) {

@@ -41,7 +41,8 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 1024;                      // window: elements per full chunk (one warp)
 constexpr int kSlots = kChunk / 128;              // float4 slots per lane per chunk (8)
-constexpr int kSmallSeg = 32;                     // segments of <= 32 chunks are summed by one warp
+constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
+constexpr int kSegCache = 512;                    // segments of a CTA run whose table entries sit in shared memory
 constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
@@ -72,7 +73,7 @@ struct Control {
     unsigned finished;
     int timeout;         // set when a bounded wait ran out
     int M_max_eff;       // max over segments of M_eff for this call
-    unsigned long long t_ns[8];   // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
+    unsigned long long t_ns[16];  // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
 };
 
 struct Args {
@@ -100,6 +101,7 @@ struct Args {
     int32_t* cta_total;          // [G]
     unsigned char* cand;         // [C][32] per-lane slot flags of full chunks: slot may hold a survivor
     int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
+    unsigned long long* cta_ns;  // [G][4] globaltimer when the CTA finished its P1, P3, last P4, P5a sweep
     SegDev* seg;                 // [S]
     Control* ctl;
     // scalars
@@ -236,10 +238,11 @@ __device__ inline void publish_eta(SegDev* sg, int m, double eta) {
 
 // Stage 1 from the segment sums: S1 = sum|x|, and S2 = sum x^2 (GPD) or SL = sum log|x| over the
 // n_nz nonzero magnitudes (gamma).
-__device__ inline void fit_stage1(const Args& A, SegDev* sg, int n, double S1, double S2_or_SL, int n_nz) {
+__device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n, double S1, double S2_or_SL,
+                                  int n_nz) {
     int M;
     if (A.max_stages > 0) {
-        M = sg->M < 1 ? 1 : sg->M;
+        M = M_state < 1 ? 1 : M_state;
         if (M > A.max_stages) M = A.max_stages;
     } else {
         M = -A.max_stages;
@@ -440,72 +443,104 @@ __device__ __forceinline__ unsigned load_flagged(const float* __restrict__ src, 
 // end of a statistics phase: arrivals and fits for the segments of this CTA's run
 // ----------------------------------------------------------------------------
 
+// Sum of the per-chunk partials q = first, first + stride, ... < q1, added in that order.  Loads are
+// issued eight chunks at a time so that a long segment costs few memory round trips.
+__device__ __forceinline__ Sums strided_partials(const Args& A, int first, int q1, int stride) {
+    double a = 0.0, b = 0.0;
+    int n = 0;
+    for (int q = first; q < q1; q += 8 * stride) {
+        double xa[8], xb[8];
+        int xn[8];
+        #pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int qq = q + u * stride;
+            const bool ok = qq < q1;
+            xa[u] = ok ? ld_cg(A.part + 3 * (size_t)qq + 0) : 0.0;
+            xb[u] = ok ? ld_cg(A.part + 3 * (size_t)qq + 1) : 0.0;
+            xn[u] = ok ? ld_cg(A.part_n + qq) : 0;
+        }
+        #pragma unroll
+        for (int u = 0; u < 8; ++u) { a += xa[u]; b += xb[u]; n += xn[u]; }
+    }
+    return Sums{a, b, n};
+}
+
+// Table entries of the segments of a CTA run, cached in shared memory at kernel start.
+struct RunSegs {
+    int seg_lo, n_seg;          // segments seg_lo .. seg_lo + n_seg - 1 have chunks in (or between) this run
+    int* q0;                    // [kSegCache] first chunk
+    int* q1;                    // [kSegCache] one past the last chunk
+    int* runs;                  // [kSegCache] CTA runs holding chunks of the segment
+    __device__ __forceinline__ void get(const Args& A, int i, int& a, int& b, int& r) const {
+        if (i < kSegCache) { a = q0[i]; b = q1[i]; r = runs[i]; }
+        else { a = A.seg_chunk0[seg_lo + i]; b = A.seg_chunk0[seg_lo + i + 1]; r = A.seg_runs[seg_lo + i]; }
+    }
+};
+
 // `stage` = 0 for the first stage, m >= 1 for the refits.  Every CTA calls this after its warps
-// have written the partials of all chunks of its run.
-__device__ __forceinline__ void arrive_and_fit(const Args& A, int c0, int c1, int stage, int* sm_list, int* sm_count,
-                                               double (*sm_red)[3]) {
+// have written the partials of all chunks of its run.  A segment that lies inside this run alone is
+// fitted at once; one shared with other runs is fitted by the run that arrives last.
+__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int* sm_small,
+                                               int* sm_large, int* sm_count, double (*sm_red)[3], int stamp_slot) {
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) *sm_count = 0;
-    __syncthreads();
-    if (c0 >= c1) return;
-    const int seg_lo = A.chunk_seg[c0], seg_hi = A.chunk_seg[c1 - 1];
+    if (threadIdx.x == 0) {                                   // this CTA's sweep is over
+        const unsigned long long now = global_ns();
+        A.cta_ns[4 * blockIdx.x + (stage < 2 ? stage : 2)] = now;
+        if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
+    }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int base = seg_lo; base <= seg_hi; base += kThreads) {
-        const int s = base + (int)threadIdx.x;
-        if (s <= seg_hi && A.seg_chunk0[s + 1] > A.seg_chunk0[s]) {
-            SegDev* sg = &A.seg[s];
-            const bool takes_part = stage == 0 || ld_cg(&sg->M_eff) > stage;
-            if (takes_part) {
-                __threadfence();
-                const int old = atomicAdd(&sg->arrived, 1);
-                if (old == A.seg_runs[s] - 1) {
-                    sg->arrived = 0;
-                    __threadfence();
-                    sm_list[atomicAdd(sm_count, 1)] = s;
+    for (int base = 0; base < R.n_seg; base += kThreads) {
+        const int i = base + (int)threadIdx.x;
+        if (i < R.n_seg) {
+            int q0, q1, runs;
+            R.get(A, i, q0, q1, runs);
+            if (q1 > q0) {
+                SegDev* sg = &A.seg[R.seg_lo + i];
+                const bool takes_part = stage == 0 || ld_cg(&sg->M_eff) > stage;
+                bool complete = takes_part && runs == 1;
+                if (takes_part && runs > 1) {
+                    complete = atomicAdd(&sg->arrived, 1) == runs - 1;
+                    if (complete) sg->arrived = 0;
+                }
+                if (complete) {
+                    if (q1 - q0 <= kSmallSeg) sm_small[atomicAdd(&sm_count[0], 1)] = i;
+                    else sm_large[atomicAdd(&sm_count[1], 1)] = i;
                 }
             }
         }
         __syncthreads();
-        const int n_done = *sm_count;
-        // small segments: one warp each, lanes take one chunk partial each, fixed shuffle tree
-        for (int i = warp; i < n_done; i += kWarps) {
-            const int s2 = sm_list[i];
-            const int q0 = A.seg_chunk0[s2], q1 = A.seg_chunk0[s2 + 1];
-            if (q1 - q0 > kSmallSeg) continue;
-            double a = 0.0, b = 0.0;
-            int n = 0;
-            if (q0 + lane < q1) {
-                a = ld_cg(A.part + 3 * (size_t)(q0 + lane) + 0);
-                b = ld_cg(A.part + 3 * (size_t)(q0 + lane) + 1);
-                n = ld_cg(A.part_n + q0 + lane);
-            }
-            Sums r = warp_tree(a, b, n);
+        const int n_small = sm_count[0], n_large = sm_count[1];
+        // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
+        for (int k = warp; k < n_small; k += kWarps) {
+            const int i2 = sm_small[k];
+            int q0, q1, runs;
+            R.get(A, i2, q0, q1, runs);
+            SegDev* sg = &A.seg[R.seg_lo + i2];
+            const int M_state = (stage == 0 && lane == 0) ? sg->M : 0;     // in flight with the partials
+            const Sums t = strided_partials(A, q0 + lane, q1, 32);
+            Sums r = warp_tree(t.a, t.b, t.n);
             if (lane == 0) {
-                if (stage == 0) fit_stage1(A, &A.seg[s2], A.seg_n[s2], r.a, r.b, r.n);
-                else fit_stage_m(A, &A.seg[s2], stage, r.n, r.a, r.b);
+                if (stage == 0) fit_stage1(A, sg, M_state, A.seg_n[R.seg_lo + i2], r.a, r.b, r.n);
+                else fit_stage_m(A, sg, stage, r.n, r.a, r.b);
             }
         }
         // large segments: the whole CTA, threads stride over the chunk partials, fixed block tree
-        for (int i = 0; i < n_done; ++i) {
-            const int s2 = sm_list[i];
-            const int q0 = A.seg_chunk0[s2], q1 = A.seg_chunk0[s2 + 1];
-            if (q1 - q0 <= kSmallSeg) continue;
-            double a = 0.0, b = 0.0;
-            int n = 0;
-            for (int q = q0 + (int)threadIdx.x; q < q1; q += kThreads) {
-                a += ld_cg(A.part + 3 * (size_t)q + 0);
-                b += ld_cg(A.part + 3 * (size_t)q + 1);
-                n += ld_cg(A.part_n + q);
-            }
-            Sums r = block_tree(a, b, n, sm_red);
+        for (int k = 0; k < n_large; ++k) {
+            const int i2 = sm_large[k];
+            int q0, q1, runs;
+            R.get(A, i2, q0, q1, runs);
+            SegDev* sg = &A.seg[R.seg_lo + i2];
+            const int M_state = (stage == 0 && threadIdx.x == 0) ? sg->M : 0;
+            const Sums t = strided_partials(A, q0 + (int)threadIdx.x, q1, kThreads);
+            Sums r = block_tree(t.a, t.b, t.n, sm_red);
             if (threadIdx.x == 0) {
-                if (stage == 0) fit_stage1(A, &A.seg[s2], A.seg_n[s2], r.a, r.b, r.n);
-                else fit_stage_m(A, &A.seg[s2], stage, r.n, r.a, r.b);
+                if (stage == 0) fit_stage1(A, sg, M_state, A.seg_n[R.seg_lo + i2], r.a, r.b, r.n);
+                else fit_stage_m(A, sg, stage, r.n, r.a, r.b);
             }
         }
         __syncthreads();
-        if (threadIdx.x == 0) *sm_count = 0;
+        if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
         __syncthreads();
     }
 }
@@ -520,10 +555,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ int sm_list[kThreads];
     __shared__ int sm_scan[kThreads];
     __shared__ int sm_warp[kWarps];
-    __shared__ int sm_count;
+    __shared__ int sm_count[2];
     __shared__ int sm_next;
     __shared__ int sm_base;
     __shared__ int sm_resweep;
+    __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache];
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -534,7 +570,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     int barrier_no = 0;
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
+#ifdef SIDCO_DIAG_SPAN
+    if (threadIdx.x == 0) A.cta_ns[4 * cta + 1] = global_ns();
+#endif
     if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; }
+    if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
+    RunSegs R{0, 0, sm_q0, sm_q1, sm_runs};
+    if (c0 < c1) {
+        R.seg_lo = A.chunk_seg[c0];
+        R.n_seg = A.chunk_seg[c1 - 1] - R.seg_lo + 1;
+        for (int i = threadIdx.x; i < R.n_seg && i < kSegCache; i += kThreads) {
+            sm_q0[i] = A.seg_chunk0[R.seg_lo + i];
+            sm_q1[i] = A.seg_chunk0[R.seg_lo + i + 1];
+            sm_runs[i] = A.seg_runs[R.seg_lo + i];
+        }
+    }
     // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
     // of the last call) ended, so that it begins on the lines most recently left in L2.
     const bool p1_desc = A.cta_dir[cta] != 0;
@@ -542,7 +592,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
-        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], 0, 0.0, 0.0, 0);
+        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0);
     __syncthreads();
 
     // Candidate threshold of a segment for this call: only single-stage segments use one.  It depends
@@ -661,7 +711,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             cur = nxt;
         }
     }
-    arrive_and_fit(A, c0, c1, 0, sm_list, &sm_count, sm_red);
+    arrive_and_fit(A, R, 0, sm_list, sm_scan, sm_count, sm_red, 6);
+    if (stamper) A.ctl->t_ns[7] = global_ns();
+#ifdef SIDCO_DIAG_BARRIER
+    if (threadIdx.x == 0) A.cta_ns[4 * cta + 1] = global_ns();
+#endif
     if (threadIdx.x == 0) sm_next = 0;
     grid_barrier(A.ctl, A.G, ++barrier_no);
     const int M_max_eff = ld_volatile(&A.ctl->M_max_eff);
@@ -714,7 +768,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 cur = nxt;
             }
         }
-        arrive_and_fit(A, c0, c1, 1, sm_list, &sm_count, sm_red);
+        arrive_and_fit(A, R, 1, sm_list, sm_scan, sm_count, sm_red, 8);
+        if (stamper) A.ctl->t_ns[9] = global_ns();
         if (threadIdx.x == 0) sm_next = 0;
         grid_barrier(A.ctl, A.G, ++barrier_no);
         if (stamper) A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
@@ -728,23 +783,27 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     const Desc nxt = fetch_desc(A, queue.next(false), true);
                     sw.load(A, cur.seg, m - 1);
                     if (sw.M_eff > m) {
-                        const int c = cur.c, lo = cur.lo;
-                        const int wb = lo & ~(kChunk - 1);
-                        const int hi = lo + cur.side_n;
-                        float v[kSlots][4];
-                        const unsigned valid = load_chunk(A.side_val, lo, hi, wb, true, v);
+                        // the side region is a compact list: lanes stride over its entries
+                        const int c = cur.c, n = cur.side_n;
+                        const float* list = A.side_val + cur.lo;
                         double sy = 0.0, sy2 = 0.0;
                         int cnt = 0;
-                        #pragma unroll
-                        for (int j = 0; j < kSlots; ++j)
+                        for (int i0 = 0; i0 < n; i0 += 128) {
+                            float a[4];
                             #pragma unroll
-                            for (int cc = 0; cc < 4; ++cc)
-                                if ((valid & (1u << (4 * j + cc))) && fabsf(v[j][cc]) > sw.thr_gt) {
-                                    const double y = (double)fabsf(v[j][cc]) - sw.eta_prev;
+                            for (int u = 0; u < 4; ++u) {
+                                const int i = i0 + u * 32 + lane;
+                                a[u] = i < n ? fabsf(ld_cg(list + i)) : 0.0f;
+                            }
+                            #pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (a[u] > sw.thr_gt) {        // thr_gt >= 0, so padding zeros never pass
+                                    const double y = (double)a[u] - sw.eta_prev;
                                     sy += y;
                                     if (SID != kSidExp) sy2 = fma(y, y, sy2);
                                     ++cnt;
                                 }
+                        }
                         Sums r = warp_tree(sy, sy2, cnt);
                         if (lane == 0) {
                             A.part[3 * (size_t)c + 0] = r.a;
@@ -755,7 +814,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     cur = nxt;
                 }
             }
-            arrive_and_fit(A, c0, c1, m, sm_list, &sm_count, sm_red);
+            arrive_and_fit(A, R, m, sm_list, sm_scan, sm_count, sm_red, 10);
+            if (stamper) A.ctl->t_ns[11] = global_ns();
             if (threadIdx.x == 0) sm_next = 0;
             grid_barrier(A.ctl, A.G, ++barrier_no);
             if (stamper) A.ctl->t_ns[3] = global_ns();
@@ -784,31 +844,57 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             const bool from_side = seg_from_side;
             const int c = cur.c, lo = cur.lo;
             const int wb = lo & ~(kChunk - 1);
-            const int hi = from_side ? lo + cur.side_n : cur.hi;
-            const bool flagged = seg_flagged && vec_ok && lo == wb && hi == wb + kChunk;
             int cnt = 0;
-            if (!from_side && !flagged) ++resweep;
-            if (hi > lo && !(flagged && __ballot_sync(kFull, cur.flags != 0) == 0)) {
-                float v[kSlots][4];
-                const unsigned valid = flagged ? load_flagged(A.residual, wb, cur.flags, v)
-                                               : load_chunk(from_side ? A.side_val : A.residual, lo, hi, wb,
-                                                            from_side || vec_ok, v);
-                unsigned mask = 0;
-                #pragma unroll
-                for (int j = 0; j < kSlots; ++j)
+            if (from_side) {
+                // compact list of stage-2 exceedances: lanes stride over it, one ballot per 32 entries
+                const int n = cur.side_n;
+                const unsigned lt = (1u << lane) - 1u;
+                for (int i0 = 0; i0 < n; i0 += 128) {
+                    float x[4];
                     #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc)
-                        if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
-                mask &= valid;
-                if (__ballot_sync(kFull, mask != 0)) {
-                    const int e0 = wb + lane * 4;
-                    cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                        const int e = e0 + j * 128 + cc;
-                        const int idx = from_side ? ld_cg(A.side_idx + e) : e;
-                        A.stage_idx[p] = idx;
-                        A.stage_val[p] = v[j][cc];
-                        A.residual[idx] = 0.0f;
-                    });
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        x[u] = i < n ? ld_cg(A.side_val + lo + i) : 0.0f;
+                    }
+                    #pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * 32 + lane;
+                        const bool hit = i < n && fabsf(x[u]) >= sv.thr_ge;
+                        const unsigned b = __ballot_sync(kFull, hit);
+                        if (hit) {
+                            const int p = lo + cnt + __popc(b & lt);
+                            const int idx = ld_cg(A.side_idx + lo + i);
+                            A.stage_idx[p] = idx;
+                            A.stage_val[p] = x[u];
+                            A.residual[idx] = 0.0f;
+                        }
+                        cnt += __popc(b);
+                    }
+                }
+            } else {
+                const int hi = cur.hi;
+                const bool flagged = seg_flagged && vec_ok && lo == wb && hi == wb + kChunk;
+                if (!flagged) ++resweep;
+                if (!(flagged && __ballot_sync(kFull, cur.flags != 0) == 0)) {
+                    float v[kSlots][4];
+                    const unsigned valid = flagged ? load_flagged(A.residual, wb, cur.flags, v)
+                                                   : load_chunk(A.residual, lo, hi, wb, vec_ok, v);
+                    unsigned mask = 0;
+                    #pragma unroll
+                    for (int j = 0; j < kSlots; ++j)
+                        #pragma unroll
+                        for (int cc = 0; cc < 4; ++cc)
+                            if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
+                    mask &= valid;
+                    if (__ballot_sync(kFull, mask != 0)) {
+                        const int e0 = wb + lane * 4;
+                        cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                            const int e = e0 + j * 128 + cc;
+                            A.stage_idx[p] = e;
+                            A.stage_val[p] = v[j][cc];
+                            A.residual[e] = 0.0f;
+                        });
+                    }
                 }
             }
             if (lane == 0) A.chunk_cnt[c] = cnt;
@@ -821,6 +907,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
     __threadfence();
     __syncthreads();
+    if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns();
+    if (stamper) A.ctl->t_ns[12] = global_ns();
     // next call: start the first sweep where this call's last full sweep over acc ended
     if (threadIdx.x == 0) A.cta_dir[cta] = (2 * sm_resweep >= c1 - c0) ? (p1_desc ? 1 : 0) : (p1_desc ? 0 : 1);
     int cta_count = 0;
@@ -923,6 +1011,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __syncthreads();
     if (threadIdx.x == 0) {
         if (stamper) A.ctl->t_ns[5] = global_ns();
+#ifdef SIDCO_DIAG_SPAN
+        A.cta_ns[4 * cta + 2] = global_ns();
+#endif
         __threadfence();
         const unsigned done = atomicAdd(&A.ctl->finished, 1u);
         if (done == (unsigned)A.G - 1u) {
