@@ -117,6 +117,38 @@ int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_o
                         float delta, int sid_type, int max_stages,
                         int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
 
+/*
+ * sidco_compress_static - sidco_compress for callers that must not allocate device memory.
+ *
+ * (The paper has no counterpart to this entry point; it exists for integration reasons only.)
+ *
+ * Some callers cannot tolerate a cudaMalloc: code running while a CUDA graph is being captured, code inside
+ * a framework whose caching allocator owns all device memory and treats outside allocations as leaks or
+ * fragmentation, and latency-critical loops where an allocation's implicit device synchronisation is
+ * unacceptable.  sidco_compress allocates its scratch workspace on the first call for a residual pointer.
+ * This variant never calls cudaMalloc, cudaFree or any allocating routine: its workspace is a fixed
+ * 18 MiB array in device memory that is part of the library image, so every GPU on which the library is
+ * loaded holds those 18 MiB until the process exits, whether or not this function is ever called.
+ *
+ * Same arguments, results and error codes as sidco_compress, with these differences:
+ *   - limits: d = seg_offsets[n_segs] <= SIDCO_STATIC_MAX_ELEMS and n_segs <= SIDCO_STATIC_MAX_SEGS;
+ *     larger inputs are rejected with SIDCO_E_SIZE before anything is enqueued;
+ *   - there is one workspace per device, shared by every call: two calls that overlap on the GPU (for
+ *     example on different streams) race on it and corrupt each other; serialise them;
+ *   - the workspace keeps the contents the previous call left.  The counters that must start at zero are
+ *     cleared on `stream` before each launch.  The stage-adaptation state lives in the workspace too and
+ *     belongs to the last (residual pointer, segment table) pair: calling with a different pair rebuilds
+ *     the tables, resets M to 1 and synchronises `stream` once;
+ *   - the first call on a device looks up the device address of the array (cudaGetSymbolAddress) and
+ *     uploads tables; make that first call before any stream capture begins;
+ *   - the debug, state and workspace helpers below do not see this workspace.
+ */
+#define SIDCO_STATIC_MAX_ELEMS 1048576
+#define SIDCO_STATIC_MAX_SEGS  256
+int sidco_compress_static(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs,
+                          float delta, int sid_type, int max_stages,
+                          int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
+
 /* Bytes of device scratch one residual key needs for a vector of d elements in n_segs segments. */
 size_t sidco_workspace_bytes(int64_t d, int n_segs);
 

@@ -38,7 +38,7 @@ EXPORTS = [
     "sidco_compress", "sidco_compress_host", "sidco_workspace_bytes", "sidco_set_workspace",
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
-    "sidco_get_phase_times", "sidco_get_cta_sweep_times",
+    "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
 ]
 
 _lib = None
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
     L.sidco_compress.restype = i32
     L.sidco_compress_host.argtypes = compress_sig
     L.sidco_compress_host.restype = i32
+    L.sidco_compress_static.argtypes = compress_sig
+    L.sidco_compress_static.restype = i32
     L.sidco_workspace_bytes.argtypes = [i64, i32]
     L.sidco_workspace_bytes.restype = C.c_size_t
     L.sidco_set_workspace.argtypes = [vp, vp, C.c_size_t]
@@ -230,3 +232,20 @@ def sidco_get_cta_sweep_times(residual, max_ctas: int = 1024) -> np.ndarray:
     if rc < 0:
         raise SidcoError(rc, "sidco_get_cta_sweep_times")
     return np.ctypeslib.as_array(buf)[: 4 * rc].reshape(rc, 4).copy()
+
+
+STATIC_MAX_ELEMS = 1048576
+STATIC_MAX_SEGS = 256
+
+
+def sidco_compress_static(grad, residual, seg_offsets, delta: float, sid_type: int, max_stages: int,
+                          out_idx, out_val, out_k, stream=None) -> None:
+    """sidco_compress without any device allocation: the workspace is a fixed 18 MiB array inside the
+    library, one per GPU, shared by all calls (do not overlap calls on one GPU).  For callers that
+    cannot call cudaMalloc, e.g. under stream capture or inside a pool-managed allocator.  Limits:
+    STATIC_MAX_ELEMS elements, STATIC_MAX_SEGS segments."""
+    arr, p, n = _offsets(seg_offsets)
+    rc = lib().sidco_compress_static(_ptr(grad), _ptr(residual), p, n, delta, sid_type, max_stages,
+                                     _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_compress_static")

@@ -356,6 +356,196 @@ int sidco_compress(const float* grad, float* residual, const int64_t* seg_offset
                          (cudaStream_t)stream, g_params);
 }
 
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Entry point that allocates nothing: its workspace is a fixed array in device memory.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxElems = SIDCO_STATIC_MAX_ELEMS;
+constexpr int kStaticMaxSegs = SIDCO_STATIC_MAX_SEGS;
+constexpr int kStaticMaxChunks = kStaticMaxElems / kChunk + kStaticMaxSegs + 1;
+constexpr size_t kStaticBytes = 18u << 20;
+
+// The workspace itself.  Device code could name it directly; host code may only take its address
+// through cudaGetSymbolAddress, because on the host this name is a stand-in, not a device pointer.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+struct StaticContext {
+    bool ready = false;              // device address looked up
+    unsigned char* base = nullptr;   // device address of g_static_scratch on this device
+    bool tables_valid = false;
+    const void* key = nullptr;       // residual pointer the adaptation state belongs to
+    int S = 0, T = 0, G = 0;
+    Layout L{};
+    int64_t offsets[kStaticMaxSegs + 1];
+    int32_t chunk_start[kStaticMaxChunks + 1], chunk_seg[kStaticMaxChunks + 1];
+    int32_t seg_chunk0[kStaticMaxSegs + 1], seg_n[kStaticMaxSegs + 1], seg_runs[kStaticMaxSegs + 1];
+    int32_t cta_chunk0[kMaxGrid + 1];
+    SegDev seg_init[kStaticMaxSegs + 1];
+};
+
+constexpr int kMaxDevices = 64;
+StaticContext g_static[kMaxDevices];
+
+// Same tables as build_tables(), written into the fixed host arrays of the static context.
+void fill_static_tables(StaticContext& c, const int64_t* off, int S, int G) {
+    int T = 0;
+    for (int s = 0; s < S; ++s) {
+        c.seg_chunk0[s] = T;
+        c.seg_n[s] = (int32_t)(off[s + 1] - off[s]);
+        c.seg_runs[s] = 0;
+        int64_t at = off[s];
+        while (at < off[s + 1]) {
+            int64_t end = (at / kChunk + 1) * kChunk;
+            if (end > off[s + 1]) end = off[s + 1];
+            c.chunk_start[T] = (int32_t)at;
+            c.chunk_seg[T] = s;
+            ++T;
+            at = end;
+        }
+    }
+    c.seg_chunk0[S] = T;
+    c.seg_n[S] = 0;
+    c.seg_runs[S] = 0;
+    c.chunk_start[T] = (int32_t)off[S];
+    c.chunk_seg[T] = 0;
+    const double per_chunk = 128.0;
+    double total = 0.0;
+    for (int t = 0; t < T; ++t) total += (c.chunk_start[t + 1] - c.chunk_start[t]) + per_chunk;
+    double acc = 0.0;
+    int cta = 0;
+    c.cta_chunk0[0] = 0;
+    for (int t = 0; t < T; ++t) {
+        const double w = (c.chunk_start[t + 1] - c.chunk_start[t]) + per_chunk;
+        int want = (int)((acc + 0.5 * w) / total * G);
+        if (want > G - 1) want = G - 1;
+        while (cta < want) c.cta_chunk0[++cta] = t;
+        acc += w;
+    }
+    while (cta < G) c.cta_chunk0[++cta] = T;
+    for (int g = 0; g < G; ++g) {
+        int prev = -1;
+        for (int t = c.cta_chunk0[g]; t < c.cta_chunk0[g + 1]; ++t)
+            if (c.chunk_seg[t] != prev) { prev = c.chunk_seg[t]; ++c.seg_runs[prev]; }
+    }
+    c.T = T;
+    c.S = S;
+    c.G = G;
+    for (int s = 0; s <= S; ++s) c.offsets[s] = off[s];
+}
+
+}  // namespace
+
+extern "C" {
+
+int sidco_compress_static(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
+                          int sid_type, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k,
+                          void* stream_v) {
+    int rc = check_args(grad, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k);
+    if (rc) return rc;
+    const int64_t d = seg_offsets[n_segs];
+    if (d > kStaticMaxElems || n_segs > kStaticMaxSegs) return SIDCO_E_SIZE;
+    if ((grad < residual + d) && (residual < grad + d) && d > 0) return SIDCO_E_ALIAS;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= kMaxDevices) return SIDCO_E_SIZE;
+    std::lock_guard<std::mutex> lock(g_mu);
+    StaticContext& c = g_static[dev];
+    if (!c.ready) {
+        // Once per device, with that device current: ask the runtime where the array lives there.
+        void* p = nullptr;
+        if ((e = cudaGetSymbolAddress(&p, g_static_scratch)) != cudaSuccess) return (int)e;
+        c.base = (unsigned char*)p;
+        c.ready = true;
+    }
+    DeviceInfo* di = nullptr;
+    if ((e = device_info(dev, &di)) != cudaSuccess) return (int)e;
+    const bool same = c.tables_valid && c.key == residual && c.S == n_segs &&
+                      std::memcmp(c.offsets, seg_offsets, sizeof(int64_t) * (n_segs + 1)) == 0;
+    if (!same) {
+        // New residual or segment table: rebuild the tables and start the adaptation state afresh.
+        fill_static_tables(c, seg_offsets, n_segs, di->grid);
+        c.L = make_layout(d, n_segs, c.T, c.G);
+        if (c.L.total > kStaticBytes) return SIDCO_E_SIZE;
+        for (int s = 0; s <= n_segs; ++s) {
+            std::memset(&c.seg_init[s], 0, sizeof(SegDev));
+            c.seg_init[s].M = 1;
+        }
+        const Layout& L = c.L;
+        auto up = [&](size_t at, const void* src, size_t bytes) {
+            return cudaMemcpyAsync(c.base + at, src, bytes, cudaMemcpyHostToDevice, stream);
+        };
+        if ((e = up(L.chunk_start, c.chunk_start, sizeof(int32_t) * (c.T + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.chunk_seg, c.chunk_seg, sizeof(int32_t) * (c.T + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.seg_chunk0, c.seg_chunk0, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.seg_n, c.seg_n, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.seg_runs, c.seg_runs, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.cta_chunk0, c.cta_chunk0, sizeof(int32_t) * (c.G + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
+        // the uploads read the fixed host arrays: let them finish before those can change again
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
+        c.key = residual;
+        c.tables_valid = true;
+    }
+    const Layout& L = c.L;
+    // The array keeps whatever the last call left.  The barrier and completion counters must start at
+    // zero, so they are cleared on the stream before every launch; everything else is either rewritten
+    // before it is read or is state that is meant to persist.
+    if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
+    unsigned char* base = c.base;
+    Args a{};
+    a.grad = grad;
+    a.residual = residual;
+    a.out_idx = out_idx;
+    a.out_val = out_val;
+    a.out_k = out_k;
+    a.chunk_start = (const int32_t*)(base + L.chunk_start);
+    a.chunk_seg = (const int32_t*)(base + L.chunk_seg);
+    a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
+    a.seg_n = (const int32_t*)(base + L.seg_n);
+    a.seg_runs = (const int32_t*)(base + L.seg_runs);
+    a.cta_chunk0 = (const int32_t*)(base + L.cta_chunk0);
+    a.part = (double*)(base + L.part);
+    a.part_n = (int32_t*)(base + L.part_n);
+    a.side_cnt = (int32_t*)(base + L.side_cnt);
+    a.chunk_cnt = (int32_t*)(base + L.chunk_cnt);
+    a.side_idx = (int32_t*)(base + L.side_idx);
+    a.side_val = (float*)(base + L.side_val);
+    a.stage_idx = (int32_t*)(base + L.stage_idx);
+    a.stage_val = (float*)(base + L.stage_val);
+    a.cta_total = (int32_t*)(base + L.cta_total);
+    a.cand = base + L.cand;
+    a.cta_dir = (int32_t*)(base + L.cta_dir);
+    a.cta_ns = (unsigned long long*)(base + L.cta_ns);
+    a.seg = (SegDev*)(base + L.seg);
+    a.ctl = (Control*)(base + L.ctl);
+    a.delta = (double)delta;
+    a.delta1 = g_params.delta1;
+    a.eps_H = g_params.eps_H;
+    a.eps_L = g_params.eps_L;
+    a.Q = g_params.Q;
+    a.sid = sid_type;
+    a.max_stages = max_stages;
+    a.C = c.T;
+    a.S = c.S;
+    a.G = c.G;
+    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
+    a.spec_enable = 1;
+    void* kargs[] = {(void*)&a};
+    const void* fn = sid_type == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
+                     : sid_type == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
+                                     : (const void*)sidco::sidco_persistent_kernel<2>;
+    e = cudaLaunchCooperativeKernel(fn, dim3(c.G), dim3(kThreads), kargs, 0, stream);
+    if (e != cudaSuccess) return (int)e;
+    g_launches.fetch_add(1);
+    return 0;
+}
+
 int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
                         int sid_type, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k,
                         void* stream_v) {
