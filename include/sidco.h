@@ -164,6 +164,10 @@ int sidco_set_params(double delta1, double eps_H, double eps_L, int Q);
 /* Forget the adaptation state of `residual` (M back to 1, counters to 0).  Synchronises the device. */
 int sidco_reset_state(const float* residual);
 
+/* The same reset enqueued on `stream` (one tiny kernel, no synchronisation): for callers that restart a
+ * run - zero the residual, reset the stage adaptation - without stalling the stream. */
+int sidco_reset_state_async(const float* residual, void* stream);
+
 /* Copy per-segment thresholds, counts, stage counts and status of the last call to host memory
  * (`out` has room for n_segs entries).  Synchronises the device; meant for tests and logging. */
 int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);

@@ -39,6 +39,7 @@ EXPORTS = [
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
+    "sidco_reset_state_async",
 ]
 
 _lib = None
@@ -77,6 +78,8 @@ def lib() -> C.CDLL:
     L.sidco_set_params.restype = i32
     L.sidco_reset_state.argtypes = [vp]
     L.sidco_reset_state.restype = i32
+    L.sidco_reset_state_async.argtypes = [vp, vp]
+    L.sidco_reset_state_async.restype = i32
     L.sidco_get_debug.argtypes = [vp, C.POINTER(SegDebug), i32]
     L.sidco_get_debug.restype = i32
     L.sidco_get_phase_times.argtypes = [vp, C.POINTER(dbl)]
@@ -249,3 +252,10 @@ def sidco_compress_static(grad, residual, seg_offsets, delta: float, sid_type: i
                                      _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
     if rc:
         raise SidcoError(rc, "sidco_compress_static")
+
+
+def sidco_reset_state_async(residual, stream=None) -> None:
+    """Reset the stage adaptation of `residual` on `stream` without synchronising."""
+    rc = lib().sidco_reset_state_async(_ptr(residual), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_reset_state_async")

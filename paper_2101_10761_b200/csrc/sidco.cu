@@ -36,7 +36,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
-    size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_chunk0;
+    size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_desc;
     size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, cand, cta_dir, cta_ns, seg, ctl;
     size_t total;
 };
@@ -50,7 +50,7 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.seg_chunk0 = take(sizeof(int32_t) * (size_t)(S + 1));
     L.seg_n = take(sizeof(int32_t) * (size_t)(S + 1));
     L.seg_runs = take(sizeof(int32_t) * (size_t)(S + 1));
-    L.cta_chunk0 = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.cta_desc = take(sizeof(int4) * (size_t)(G + 1));
     L.part = take(sizeof(double) * 3 * (size_t)(T + 1));
     L.part_n = take(sizeof(int32_t) * (size_t)(T + 1));
     L.side_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
@@ -83,6 +83,7 @@ struct Context {
     size_t ws_bytes = 0;
     bool ws_owned = false;
     bool tables_valid = false;
+    unsigned call_id = 0;                  // tags the per-segment ready words
     Layout L{};
     // staging for sidco_compress_host
     float* h_grad = nullptr; float* h_res = nullptr;
@@ -200,11 +201,15 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
         }
         while (cta < G) cta_chunk0[++cta] = T;
     }
-    // number of CTA runs that hold chunks of each segment (arrivals expected per statistics phase)
+    // number of CTA runs that hold chunks of each segment (arrivals expected per statistics phase),
+    // and the per-CTA descriptor {first chunk, end chunk, first segment, number of segments spanned}
+    std::vector<int4> cta_desc(G + 1, make_int4(T, T, 0, 0));
     for (int g = 0; g < G; ++g) {
         int prev = -1;
         for (int t = cta_chunk0[g]; t < cta_chunk0[g + 1]; ++t)
             if (chunk_seg[t] != prev) { prev = chunk_seg[t]; ++seg_runs[prev]; }
+        const int a = cta_chunk0[g], b = cta_chunk0[g + 1];
+        cta_desc[g] = a < b ? make_int4(a, b, chunk_seg[a], chunk_seg[b - 1] - chunk_seg[a] + 1) : make_int4(a, a, 0, 0);
     }
 
     const Layout L = make_layout(d, S, T, G);
@@ -245,7 +250,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.seg_chunk0, seg_chunk0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg_n, seg_n.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg_runs, seg_runs.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
-    if ((e = up(L.cta_chunk0, cta_chunk0.data(), sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
+    if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
@@ -284,7 +289,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
     a.seg_n = (const int32_t*)(base + L.seg_n);
     a.seg_runs = (const int32_t*)(base + L.seg_runs);
-    a.cta_chunk0 = (const int32_t*)(base + L.cta_chunk0);
+    a.cta_desc = (const int4*)(base + L.cta_desc);
     a.part = (double*)(base + L.part);
     a.part_n = (int32_t*)(base + L.part_n);
     a.side_cnt = (int32_t*)(base + L.side_cnt);
@@ -309,6 +314,8 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.C = c->T;
     a.S = c->S;
     a.G = c->G;
+    c->call_id = (c->call_id + 1u) & 0x0fffffffu;
+    a.call_id = (int)c->call_id;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
     // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
     static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
@@ -318,7 +325,9 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
                      : sid == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
-    e = cudaLaunchCooperativeKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
+    static const bool plain = [] { const char* v = getenv("SIDCO_PLAIN_LAUNCH"); return v && v[0] == '1'; }();
+    if (plain) e = cudaLaunchKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
+    else e = cudaLaunchCooperativeKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
     return 0;
@@ -383,6 +392,8 @@ struct StaticContext {
     int32_t chunk_start[kStaticMaxChunks + 1], chunk_seg[kStaticMaxChunks + 1];
     int32_t seg_chunk0[kStaticMaxSegs + 1], seg_n[kStaticMaxSegs + 1], seg_runs[kStaticMaxSegs + 1];
     int32_t cta_chunk0[kMaxGrid + 1];
+    int4 cta_desc[kMaxGrid + 1];
+    unsigned call_id = 0;
     SegDev seg_init[kStaticMaxSegs + 1];
 };
 
@@ -429,6 +440,9 @@ void fill_static_tables(StaticContext& c, const int64_t* off, int S, int G) {
         int prev = -1;
         for (int t = c.cta_chunk0[g]; t < c.cta_chunk0[g + 1]; ++t)
             if (c.chunk_seg[t] != prev) { prev = c.chunk_seg[t]; ++c.seg_runs[prev]; }
+        const int a = c.cta_chunk0[g], b = c.cta_chunk0[g + 1];
+        c.cta_desc[g] = a < b ? make_int4(a, b, c.chunk_seg[a], c.chunk_seg[b - 1] - c.chunk_seg[a] + 1)
+                              : make_int4(a, a, 0, 0);
     }
     c.T = T;
     c.S = S;
@@ -484,7 +498,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = up(L.seg_chunk0, c.seg_chunk0, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg_n, c.seg_n, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg_runs, c.seg_runs, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
-        if ((e = up(L.cta_chunk0, c.cta_chunk0, sizeof(int32_t) * (c.G + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.cta_desc, c.cta_desc, sizeof(int4) * (c.G + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
         // the uploads read the fixed host arrays: let them finish before those can change again
@@ -509,7 +523,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
     a.seg_n = (const int32_t*)(base + L.seg_n);
     a.seg_runs = (const int32_t*)(base + L.seg_runs);
-    a.cta_chunk0 = (const int32_t*)(base + L.cta_chunk0);
+    a.cta_desc = (const int4*)(base + L.cta_desc);
     a.part = (double*)(base + L.part);
     a.part_n = (int32_t*)(base + L.part_n);
     a.side_cnt = (int32_t*)(base + L.side_cnt);
@@ -534,6 +548,8 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.C = c.T;
     a.S = c.S;
     a.G = c.G;
+    c.call_id = (c.call_id + 1u) & 0x0fffffffu;
+    a.call_id = (int)c.call_id;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
     a.spec_enable = 1;
     void* kargs[] = {(void*)&a};
@@ -643,6 +659,19 @@ int sidco_reset_state(const float* residual) {
     if ((e = cudaMemcpy(base + c->L.seg, seg.data(), sizeof(SegDev) * (c->S + 1), cudaMemcpyHostToDevice)) != cudaSuccess)
         return (int)e;
     if ((e = cudaMemset(base + c->L.ctl, 0, sizeof(Control))) != cudaSuccess) return (int)e;
+    return 0;
+}
+
+int sidco_reset_state_async(const float* residual, void* stream) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    Context* c = it->second;
+    sidco::sidco_reset_state_kernel<<<(c->S + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
+        (SegDev*)((char*)c->ws + c->L.seg), c->S);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+    g_launches.fetch_add(1);
     return 0;
 }
 

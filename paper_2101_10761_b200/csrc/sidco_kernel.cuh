@@ -6,8 +6,11 @@
 // what it wrote in one phase (acc, side buffers) it re-reads itself in the next.
 // Inside a run the warps pull chunks from a shared-memory queue and work on them
 // without any block-level synchronisation: a chunk is loaded, reduced with warp
-// shuffles, and compacted with ballots by one warp.  Phases are separated by
-// grid-wide barriers with bounded waits:
+// shuffles, and compacted with ballots by one warp.  A CTA moves from one phase to
+// the next on its own: a warp that needs a segment's threshold waits (bounded) on
+// that segment's "stages ready" word, which the run completing the segment's
+// statistics publishes with release semantics.  One grid-wide barrier remains,
+// before the final placement, which needs every CTA's survivor count:
 //
 //   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
 //       of every chunk; the CTA whose run completes a segment sums the per-chunk
@@ -65,14 +68,14 @@ struct SegDev {
     int32_t calls;
     long long k_sum;
     float spec_thr;      // candidate threshold for the next call's first sweep (<= 0: none), see P1
-    int32_t pad;
+    int32_t ready;       // call_id * 16 + number of stages fitted so far in that call (release/acquire)
 };
 
 struct Control {
-    unsigned bar;        // grid barrier arrivals (reset by the last CTA to finish)
-    unsigned finished;
+    unsigned count;      // grid barrier arrivals of the current generation (reset by the last arriver)
+    unsigned gen;        // grid barrier generation, never reset
     int timeout;         // set when a bounded wait ran out
-    int M_max_eff;       // max over segments of M_eff for this call
+    int pad;
     unsigned long long t_ns[16];  // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
 };
 
@@ -88,7 +91,7 @@ struct Args {
     const int32_t* seg_chunk0;   // [S + 1]
     const int32_t* seg_n;        // [S]
     const int32_t* seg_runs;     // [S] number of CTA runs that hold chunks of the segment
-    const int32_t* cta_chunk0;   // [G + 1]
+    const int4* cta_desc;        // [G] {first chunk, one past last chunk, first segment, segments} of the run
     // scratch
     double* part;                // [C][3] per-chunk partial sums
     int32_t* part_n;             // [C] per-chunk partial counts
@@ -108,6 +111,7 @@ struct Args {
     double delta, delta1, eps_H, eps_L;
     int Q, sid, max_stages;
     int C, S, G;
+    int call_id;                 // per-workspace call number, tags SegDev::ready
     int vec_ok;                  // grad and residual are 16-byte aligned
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
 };
@@ -136,25 +140,65 @@ __device__ __forceinline__ int ld_volatile(const int* p) {
     return *reinterpret_cast<const volatile int*>(p);
 }
 
-// Grid-wide barrier number `which` (1-based within the call).  All CTAs of the
-// cooperative launch are resident, so the wait normally ends within microseconds;
-// it is nevertheless bounded, and a time-out raises Control::timeout, after which
-// every later wait returns at once.
-__device__ __forceinline__ void grid_barrier(Control* ctl, int G, int which) {
+__device__ __forceinline__ void st_release(int* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ int ld_acquire_s32(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide barrier: the last CTA to arrive clears the arrival count and advances the generation;
+// the others wait for the generation to reach `target_gen`.  All CTAs of the cooperative launch are
+// resident, so the wait normally ends within microseconds; it is nevertheless bounded, and a
+// time-out raises Control::timeout, after which every later wait returns at once.
+__device__ __forceinline__ void grid_barrier(Control* ctl, int G, unsigned target_gen) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(&ctl->bar, 1u);
-        const unsigned target = (unsigned)which * (unsigned)G;
-        long long spins = 0;
-        while (ld_acquire(&ctl->bar) < target) {
-            if (ld_volatile(&ctl->timeout)) break;
-            if (++spins > kSpinLimit) { atomicExch(&ctl->timeout, 1); break; }
-            __nanosleep(spins < 64 ? 20 : 200);
+        const unsigned old = atomicAdd(&ctl->count, 1u);
+        if (old == (unsigned)G - 1u) {
+            ctl->count = 0u;
+            __threadfence();
+            atomicAdd(&ctl->gen, 1u);
+        } else {
+            long long spins = 0;
+            while ((int)(ld_acquire(&ctl->gen) - target_gen) < 0) {
+                if (ld_volatile(&ctl->timeout)) break;
+                if (++spins > kSpinLimit) { atomicExch(&ctl->timeout, 1); break; }
+                __nanosleep(spins < 64 ? 20 : 200);
+            }
         }
         __threadfence();
     }
     __syncthreads();
+}
+
+// Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).
+__device__ __forceinline__ void wait_ready_thread(const Args& A, const SegDev* sg, int need) {
+    const unsigned target = (unsigned)A.call_id * 16u + (unsigned)need;
+    long long spins = 0;
+    while ((int)((unsigned)ld_acquire_s32(&sg->ready) - target) < 0) {     // wrap-safe
+        if (ld_volatile(&A.ctl->timeout)) break;
+        if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+        __nanosleep(spins < 16 ? 20 : 100);
+    }
+}
+
+// Warp-level wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).
+__device__ __forceinline__ void wait_ready(const Args& A, const SegDev* sg, int need) {
+    if ((threadIdx.x & 31) == 0) {
+        const unsigned target = (unsigned)A.call_id * 16u + (unsigned)need;
+        long long spins = 0;
+        while ((int)((unsigned)ld_acquire_s32(&sg->ready) - target) < 0) {     // wrap-safe
+            if (ld_volatile(&A.ctl->timeout)) break;
+            if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+            __nanosleep(spins < 16 ? 20 : 100);
+        }
+    }
+    __syncwarp();
 }
 
 struct Sums { double a, b; int n; };
@@ -204,6 +248,19 @@ __device__ inline int stage_cap(double delta, double delta1) {
         if (!(p > delta) || M >= 64) return M;
         ++M;
     }
+}
+
+// Stage count of a segment for this call: from the adaptation state the previous call left (or the
+// fixed count), capped so that the last stage's ratio stays below one.  Stable during a call.
+__device__ __forceinline__ int seg_stages(const Args& A, int seg, int cap) {
+    int M;
+    if (A.max_stages > 0) {
+        M = A.seg[seg].M < 1 ? 1 : A.seg[seg].M;
+        if (M > A.max_stages) M = A.max_stages;
+    } else {
+        M = -A.max_stages;
+    }
+    return M < cap ? M : cap;
 }
 
 // Tail ratio of stage m (0-based) out of M: delta_1 for every non-final stage, the rest for the last.
@@ -288,7 +345,8 @@ __device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n,
     if (n == 0)
         for (int m = 1; m < M_eff; ++m) sg->eta[m] = eta;
     publish_eta(sg, 0, eta);
-    atomicMax(&A.ctl->M_max_eff, M_eff);
+    __threadfence();
+    st_release(&sg->ready, (int)((unsigned)A.call_id * 16u + (unsigned)(n == 0 ? M_eff : 1)));
 }
 
 // Stage index m >= 1 (eta_{m+1} in the paper's numbering) from the shifted peaks over eta_m:
@@ -309,6 +367,8 @@ __device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, do
         eta = prev + inc;
     }
     publish_eta(sg, m, eta);
+    __threadfence();
+    st_release(&sg->ready, (int)((unsigned)A.call_id * 16u + (unsigned)(m + 1)));
 }
 
 // ----------------------------------------------------------------------------
@@ -374,24 +434,17 @@ __device__ __forceinline__ int ordered_emit(unsigned mask, int base, Emit emit) 
     return run - base;
 }
 
-// Per-warp view of the segment a chunk belongs to, reloaded only when the segment changes.
+// Per-warp view of the segment a chunk belongs to, refreshed only when the segment changes.  The
+// values come from the run's shared-memory cache; a warp that gets there first waits (bounded) for
+// the thread that publishes them.
 struct SegView {
     int seg = -1;
     int M_eff = 0;
     float thr_gt = 0.f, thr_ge = 0.f;
     double eta_prev = 0.0;
-    __device__ __forceinline__ void load(const Args& A, int s, int m_prev) {
-        if (s == seg) return;
-        seg = s;
-        const SegDev* sg = &A.seg[s];
-        M_eff = ld_cg(&sg->M_eff);
-        thr_gt = ld_cg(&sg->thr_gt);
-        thr_ge = ld_cg(&sg->thr_ge);
-        eta_prev = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
-    }
 };
 
-// Dynamic chunk queue of a CTA run: warps take the next chunk index (ascending or descending).
+// Dynamic chunk queue of a CTA run// Dynamic chunk queue of a CTA run: warps take the next chunk index (ascending or descending).
 struct ChunkQueue {
     int* sm_next;
     int c0, c1;
@@ -471,16 +524,68 @@ struct RunSegs {
     int* q0;                    // [kSegCache] first chunk
     int* q1;                    // [kSegCache] one past the last chunk
     int* runs;                  // [kSegCache] CTA runs holding chunks of the segment
+    int* m_eff;                 // [kSegCache] stage count of the segment in this call
+    float* tau;                 // [kSegCache] candidate threshold for the first sweep (< 0: none)
+    // thresholds of the phase being swept, published by one thread per segment (see publish_params)
+    float* thr_gt;              // [kSegCache]
+    float* thr_ge;              // [kSegCache]
+    double* eta_prev;           // [kSegCache]
+    volatile int* ok;           // [kSegCache] == phase tag once the three values above are valid
     __device__ __forceinline__ void get(const Args& A, int i, int& a, int& b, int& r) const {
         if (i < kSegCache) { a = q0[i]; b = q1[i]; r = runs[i]; }
         else { a = A.seg_chunk0[seg_lo + i]; b = A.seg_chunk0[seg_lo + i + 1]; r = A.seg_runs[seg_lo + i]; }
     }
 };
 
+// One thread per segment of the run waits (bounded) until the segment has the stages this phase needs,
+// then copies its thresholds into the shared-memory cache and marks them valid with the phase tag.
+// need: stages that must be fitted (0: all of the segment's); m_prev: index of the eta the phase shifts by.
+__device__ __forceinline__ void publish_params(const Args& A, const RunSegs& R, int need, int m_prev, int tag) {
+    const int i = threadIdx.x;
+    if (i < R.n_seg && i < kSegCache && R.q1[i] > R.q0[i]) {
+        const SegDev* sg = &A.seg[R.seg_lo + i];
+        const int M_eff = R.m_eff[i];
+        wait_ready_thread(A, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
+        R.thr_gt[i] = ld_cg(&sg->thr_gt);
+        R.thr_ge[i] = ld_cg(&sg->thr_ge);
+        R.eta_prev[i] = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
+        __threadfence_block();
+        R.ok[i] = tag;
+    }
+}
+
+// Refresh a warp's segment view when the chunk's segment changed.
+__device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegView& v, int seg, int need, int m_prev,
+                                          int tag, int cap) {
+    if (seg == v.seg) return;
+    v.seg = seg;
+    const int i = seg - R.seg_lo;
+    if (i < kSegCache) {
+        v.M_eff = R.m_eff[i];
+        long long spins = 0;
+        while (R.ok[i] != tag) {                       // published by a thread of this CTA
+            if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+            __nanosleep(20);
+        }
+        __threadfence_block();
+        v.thr_gt = R.thr_gt[i];
+        v.thr_ge = R.thr_ge[i];
+        v.eta_prev = R.eta_prev[i];
+    } else {
+        // beyond the cache (a run spanning more than kSegCache segments): straight from global memory
+        const SegDev* sg = &A.seg[seg];
+        v.M_eff = seg_stages(A, seg, cap);
+        wait_ready(A, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
+        v.thr_gt = ld_cg(&sg->thr_gt);
+        v.thr_ge = ld_cg(&sg->thr_ge);
+        v.eta_prev = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
+    }
+}
+
 // `stage` = 0 for the first stage, m >= 1 for the refits.  Every CTA calls this after its warps
 // have written the partials of all chunks of its run.  A segment that lies inside this run alone is
 // fitted at once; one shared with other runs is fitted by the run that arrives last.
-__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int* sm_small,
+__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, int* sm_small,
                                                int* sm_large, int* sm_count, double (*sm_red)[3], int stamp_slot) {
     __threadfence();
     __syncthreads();
@@ -497,7 +602,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
             R.get(A, i, q0, q1, runs);
             if (q1 > q0) {
                 SegDev* sg = &A.seg[R.seg_lo + i];
-                const bool takes_part = stage == 0 || ld_cg(&sg->M_eff) > stage;
+                const bool takes_part = stage == 0 || seg_stages(A, R.seg_lo + i, cap) > stage;
                 bool complete = takes_part && runs == 1;
                 if (takes_part && runs > 1) {
                     complete = atomicAdd(&sg->arrived, 1) == runs - 1;
@@ -559,31 +664,44 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ int sm_next;
     __shared__ int sm_base;
     __shared__ int sm_resweep;
-    __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache];
+    __shared__ unsigned sm_gen;
+    __shared__ int sm_mloc;
+    __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache], sm_meff[kSegCache];
+    __shared__ float sm_tau[kSegCache], sm_thr_gt[kSegCache], sm_thr_ge[kSegCache];
+    __shared__ double sm_eta[kSegCache];
+    __shared__ int sm_ok[kSegCache];
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int c0 = A.cta_chunk0[cta], c1 = A.cta_chunk0[cta + 1];
+    const int4 run = __ldg(A.cta_desc + cta);          // {first chunk, end chunk, first segment, segments}
+    const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
     const int cap = stage_cap(A.delta, A.delta1);
-    int barrier_no = 0;
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
+    if (threadIdx.x == 0) { sm_gen = ld_acquire(&A.ctl->gen); sm_mloc = 1; }
 #ifdef SIDCO_DIAG_SPAN
     if (threadIdx.x == 0) A.cta_ns[4 * cta + 1] = global_ns();
 #endif
     if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
-    RunSegs R{0, 0, sm_q0, sm_q1, sm_runs};
-    if (c0 < c1) {
-        R.seg_lo = A.chunk_seg[c0];
-        R.n_seg = A.chunk_seg[c1 - 1] - R.seg_lo + 1;
-        for (int i = threadIdx.x; i < R.n_seg && i < kSegCache; i += kThreads) {
-            sm_q0[i] = A.seg_chunk0[R.seg_lo + i];
-            sm_q1[i] = A.seg_chunk0[R.seg_lo + i + 1];
-            sm_runs[i] = A.seg_runs[R.seg_lo + i];
+    RunSegs R{run.z, run.w, sm_q0, sm_q1, sm_runs, sm_meff, sm_tau, sm_thr_gt, sm_thr_ge, sm_eta, sm_ok};
+    __syncthreads();
+    auto stages_of = [&](int seg) -> int { return seg_stages(A, seg, cap); };
+    // cache the run's segment table; find the largest stage count among the run's segments, which
+    // is the number of statistics phases this CTA takes part in
+    for (int i = threadIdx.x; i < R.n_seg; i += kThreads) {
+        const int q0 = A.seg_chunk0[R.seg_lo + i], q1 = A.seg_chunk0[R.seg_lo + i + 1];
+        const int m = stages_of(R.seg_lo + i);
+        if (i < kSegCache) {
+            sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[R.seg_lo + i];
+            sm_meff[i] = m;
+            const float tau = A.seg[R.seg_lo + i].spec_thr;
+            sm_tau[i] = (A.spec_enable && m == 1 && tau > 0.0f) ? tau : -1.0f;
+            sm_ok[i] = 0;
         }
+        if (q1 > q0) atomicMax(&sm_mloc, m);
     }
     // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
     // of the last call) ended, so that it begins on the lines most recently left in L2.
@@ -598,17 +716,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     // Candidate threshold of a segment for this call: only single-stage segments use one.  It depends
     // on state the previous call left behind, so every warp and every phase derives the same value.
     auto spec_tau = [&](int seg) -> float {
-        if (!A.spec_enable) return -1.0f;
-        const SegDev* sg = &A.seg[seg];
-        int M;
-        if (A.max_stages > 0) {
-            M = sg->M < 1 ? 1 : sg->M;
-            if (M > A.max_stages) M = A.max_stages;
-        } else {
-            M = -A.max_stages;
-        }
-        if ((M < cap ? M : cap) != 1) return -1.0f;
-        const float tau = sg->spec_thr;
+        if (seg - R.seg_lo < kSegCache) return sm_tau[seg - R.seg_lo];
+        if (!A.spec_enable || stages_of(seg) != 1) return -1.0f;
+        const float tau = A.seg[seg].spec_thr;
         return tau > 0.0f ? tau : -1.0f;
     };
 
@@ -711,24 +821,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             cur = nxt;
         }
     }
-    arrive_and_fit(A, R, 0, sm_list, sm_scan, sm_count, sm_red, 6);
-    if (stamper) A.ctl->t_ns[7] = global_ns();
-#ifdef SIDCO_DIAG_BARRIER
-    if (threadIdx.x == 0) A.cta_ns[4 * cta + 1] = global_ns();
-#endif
+    arrive_and_fit(A, R, 0, cap, sm_list, sm_scan, sm_count, sm_red, 6);
     if (threadIdx.x == 0) sm_next = 0;
-    grid_barrier(A.ctl, A.G, ++barrier_no);
-    const int M_max_eff = ld_volatile(&A.ctl->M_max_eff);
-    if (stamper) A.ctl->t_ns[1] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
+    __syncthreads();
+    const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
+    if (stamper) A.ctl->t_ns[7] = A.ctl->t_ns[1] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
 
     // ------------------------------------------------------------------ P3: stage 2 from acc
     if (M_max_eff >= 2) {
+        publish_params(A, R, 1, 0, 1);
         {
             SegView sv;
             Desc cur = fetch_desc(A, queue.next(!p1_desc), false);
             while (cur.c >= 0) {
                 const Desc nxt = fetch_desc(A, queue.next(!p1_desc), false);
-                sv.load(A, cur.seg, 0);
+                view_load(A, R, sv, cur.seg, 1, 0, 1, cap);
                 if (sv.M_eff >= 2) {
                     ++resweep;
                     const int c = cur.c, lo = cur.lo, hi = cur.hi;
@@ -768,35 +875,35 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 cur = nxt;
             }
         }
-        arrive_and_fit(A, R, 1, sm_list, sm_scan, sm_count, sm_red, 8);
-        if (stamper) A.ctl->t_ns[9] = global_ns();
+        arrive_and_fit(A, R, 1, cap, sm_list, sm_scan, sm_count, sm_red, 8);
         if (threadIdx.x == 0) sm_next = 0;
-        grid_barrier(A.ctl, A.G, ++barrier_no);
-        if (stamper) A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
+        __syncthreads();
+        if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
 
         // -------------------------------------------------------------- P4: stages 3..M from the side regions
         for (int m = 2; m < M_max_eff; ++m) {
+            publish_params(A, R, m, m - 1, m);
             {
                 SegView sw;
                 Desc cur = fetch_desc(A, queue.next(false), true);
                 while (cur.c >= 0) {
                     const Desc nxt = fetch_desc(A, queue.next(false), true);
-                    sw.load(A, cur.seg, m - 1);
+                    view_load(A, R, sw, cur.seg, m, m - 1, m, cap);
                     if (sw.M_eff > m) {
                         // the side region is a compact list: lanes stride over its entries
                         const int c = cur.c, n = cur.side_n;
                         const float* list = A.side_val + cur.lo;
                         double sy = 0.0, sy2 = 0.0;
                         int cnt = 0;
-                        for (int i0 = 0; i0 < n; i0 += 128) {
-                            float a[4];
+                        for (int i0 = 0; i0 < n; i0 += 512) {
+                            float a[16];
                             #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < 16; ++u) {
                                 const int i = i0 + u * 32 + lane;
                                 a[u] = i < n ? fabsf(ld_cg(list + i)) : 0.0f;
                             }
                             #pragma unroll
-                            for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < 16; ++u)
                                 if (a[u] > sw.thr_gt) {        // thr_gt >= 0, so padding zeros never pass
                                     const double y = (double)a[u] - sw.eta_prev;
                                     sy += y;
@@ -814,16 +921,16 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     cur = nxt;
                 }
             }
-            arrive_and_fit(A, R, m, sm_list, sm_scan, sm_count, sm_red, 10);
-            if (stamper) A.ctl->t_ns[11] = global_ns();
+            arrive_and_fit(A, R, m, cap, sm_list, sm_scan, sm_count, sm_red, 10);
             if (threadIdx.x == 0) sm_next = 0;
-            grid_barrier(A.ctl, A.G, ++barrier_no);
-            if (stamper) A.ctl->t_ns[3] = global_ns();
+            __syncthreads();
+            if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns();
         }
     }
 
     // ------------------------------------------------------------------ P5a: stage survivors per chunk
     int warp_total = 0;
+    publish_params(A, R, 0, -1, 100);
     {
         SegView sv;
         bool seg_from_side = false, seg_flagged = false;
@@ -834,7 +941,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
                 seg_count = 0;
-                sv.load(A, cur.seg, -1);
+                view_load(A, R, sv, cur.seg, 0, -1, 100, cap);
                 // multi-stage segments keep their exceedances in the side region; single-stage ones
                 // have valid candidate flags if the candidate threshold proved low enough
                 const float tau = spec_tau(cur.seg);
@@ -849,15 +956,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 // compact list of stage-2 exceedances: lanes stride over it, one ballot per 32 entries
                 const int n = cur.side_n;
                 const unsigned lt = (1u << lane) - 1u;
-                for (int i0 = 0; i0 < n; i0 += 128) {
-                    float x[4];
+                for (int i0 = 0; i0 < n; i0 += 512) {
+                    float x[16];
                     #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 16; ++u) {
                         const int i = i0 + u * 32 + lane;
                         x[u] = i < n ? ld_cg(A.side_val + lo + i) : 0.0f;
                     }
                     #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 16; ++u) {
                         const int i = i0 + u * 32 + lane;
                         const bool hit = i < n && fabsf(x[u]) >= sv.thr_ge;
                         const unsigned b = __ballot_sync(kFull, hit);
@@ -920,7 +1027,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     }
     __syncthreads();
     cta_count = sm_base;
-    grid_barrier(A.ctl, A.G, ++barrier_no);
+    grid_barrier(A.ctl, A.G, sm_gen + 1u);
     if (stamper) A.ctl->t_ns[4] = global_ns();
 
     // ------------------------------------------------------------------ P5b: final positions
@@ -1007,21 +1114,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
     }
 
-    // last CTA out resets the control block for the next call
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        if (stamper) A.ctl->t_ns[5] = global_ns();
+    if (stamper) A.ctl->t_ns[5] = global_ns();
 #ifdef SIDCO_DIAG_SPAN
-        A.cta_ns[4 * cta + 2] = global_ns();
+    if (threadIdx.x == 0) A.cta_ns[4 * cta + 2] = global_ns();
 #endif
-        __threadfence();
-        const unsigned done = atomicAdd(&A.ctl->finished, 1u);
-        if (done == (unsigned)A.G - 1u) {
-            A.ctl->bar = 0u;
-            A.ctl->finished = 0u;
-            A.ctl->M_max_eff = 0;
-            __threadfence();
-        }
+}
+
+// Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared.  The ready
+// words keep their call tags.
+__global__ void sidco_reset_state_kernel(SegDev* seg, int S) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < S) {
+        seg[s].M = 1;
+        seg[s].calls = 0;
+        seg[s].k_sum = 0;
+        seg[s].spec_thr = -1.0f;
     }
 }
 
