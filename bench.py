@@ -9,8 +9,8 @@ stage adaptation) on the ResNet-50-shaped synthetic gradient (d = 25,557,032,
 161 segments, delta = 1e-3).  Steps follow the configuration's own protocol:
 runs of ten consecutive calls with the residual carried forward, a fresh
 gradient draw per call (ten distinct device buffers), each run starting from a
-zero residual and a fresh stage-adaptation state (M = 1); the resets sit inside
-the timed region.
+zero residual and a fresh stage-adaptation state (M = 1); the reset (one tiny
+kernel that also declares the residual empty) sits inside the timed region.
 
 Prints ONE JSON line.  `value` is GB/s on the minimal bytes the method must move
 (12 d + 8 k_hat per step), inputs resident in HBM; `e2e` is the same metric
@@ -259,8 +259,7 @@ def run_gpu(args):
     def step(i, k_buf=None, ev=None):
         """Call number i; every RUN_LEN-th call first zeroes the residual and resets the adaptation."""
         if i % RUN_LEN == 0 and i > 0:
-            res.zero_()
-            B.sidco_reset_state_async(res)
+            B.sidco_reset_state_async(res)      # also declares the residual empty: no memset needed
         if ev is not None:
             ev[0].record()
         B.sidco_compress(grads[i % RUN_LEN], res, off, DELTA, args.sid, args.max_stages, out_idx, out_val,
@@ -289,20 +288,28 @@ def run_gpu(args):
     i += (-i) % RUN_LEN          # the timed region starts at the beginning of a run
 
     # ---- timed region: device-resident inputs --------------------------------------------
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     region = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
     launches0 = B.sidco_launch_count()
     barrier()
     sampler.region = "device"
     region[0].record()
     for s in range(args.steps):
-        step(i + s, out_k_steps[s], ev[s])
+        step(i + s, out_k_steps[s])
     region[1].record()
     barrier()
-    sampler.region = None
     launches = B.sidco_launch_count() - launches0
     total_ms = region[0].elapsed_time(region[1])
+    # Second pass over the same steps with an event pair around every launch: the kernel's own average
+    # duration for the roofline figure.  (Event records between launches cost a few microseconds of
+    # stream time each, so they stay out of the region that `value` is computed from.)
+    n_ev = min(args.steps, 20 * RUN_LEN)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+    for s in range(n_ev):
+        step(i + args.steps + s, out_k, ev[s])
+    barrier()
+    sampler.region = None
     kern_ms = [a.elapsed_time(b) for a, b in ev]
+    i += n_ev
     k_hats = out_k_steps[:, S].cpu().numpy().astype(np.int64)
     bytes_min = int(12 * d * args.steps + 8 * k_hats.sum())
     dbg = B.sidco_get_debug(res, S)
@@ -321,11 +328,10 @@ def run_gpu(args):
         for v_sid, v_ms in ((0, 4), (1, 4), (2, 4), (0, -1), (1, -1), (2, -1), (0, -2), (0, -4)):
             if (v_sid, v_ms) == (args.sid, args.max_stages):
                 continue
+            res_v.zero_()
             def v_step(w):
-                if w % RUN_LEN == 0:
-                    res_v.zero_()
-                    if w:
-                        B.sidco_reset_state_async(res_v)
+                if w % RUN_LEN == 0 and w:
+                    B.sidco_reset_state_async(res_v)
                 B.sidco_compress(grads[w % RUN_LEN], res_v, off, DELTA, v_sid, v_ms, out_idx, out_val, out_k)
             for w in range(2 * RUN_LEN):
                 v_step(w)
@@ -391,8 +397,8 @@ def run_gpu(args):
                 "sid": SID_NAMES[args.sid], "max_stages": args.max_stages,
                 "M_used_hist_last_call": m_hist, "status_or": status_or,
                 "k_hat_mean": float(k_hats.mean()), "parallelism": "replicas only" if world > 1 else "1 GPU",
-                "protocol": "runs of 10 calls, residual carried, fresh draw per call; residual zeroed and adaptation "
-                            "reset before each run, inside the timed region",
+                "protocol": "runs of 10 calls, residual carried, fresh draw per call; before each run the adaptation is "
+                            "reset and the residual declared empty (sidco_reset_state_async), inside the timed region",
                 "l2": "inputs 204 MB per step exceed the 126 MB L2; 10 distinct gradient buffers",
                 "prewarm_steps": prewarm_steps,
             },

@@ -161,11 +161,14 @@ int sidco_set_workspace(const float* residual, void* device_ptr, size_t bytes);
  * delta_1 = 0.25, eps_H = eps_L = 0.2, Q = 5).  0 < delta1 < 1, 0 <= eps < 1, Q >= 1. */
 int sidco_set_params(double delta1, double eps_H, double eps_L, int Q);
 
-/* Forget the adaptation state of `residual` (M back to 1, counters to 0).  Synchronises the device. */
+/* Start over for `residual`: the adaptation state is forgotten (M back to 1, counters to 0) and the error
+ * compensation memory is declared empty - the next sidco_compress on it takes the residual as all zeros
+ * without reading it (and overwrites it), so the caller need not clear the buffer.  Synchronises the device. */
 int sidco_reset_state(const float* residual);
 
 /* The same reset enqueued on `stream` (one tiny kernel, no synchronisation): for callers that restart a
- * run - zero the residual, reset the stage adaptation - without stalling the stream. */
+ * run without stalling the stream.  The next sidco_compress for `residual` must be issued after this call
+ * returns (it is the host-side bookkeeping that tells it not to read the residual). */
 int sidco_reset_state_async(const float* residual, void* stream);
 
 /* Copy per-segment thresholds, counts, stage counts and status of the last call to host memory

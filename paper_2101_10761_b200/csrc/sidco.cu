@@ -84,6 +84,7 @@ struct Context {
     bool ws_owned = false;
     bool tables_valid = false;
     unsigned call_id = 0;                  // tags the per-segment ready words
+    bool residual_is_zero = false;         // set by a state reset: the next call does not read the residual
     Layout L{};
     // staging for sidco_compress_host
     float* h_grad = nullptr; float* h_res = nullptr;
@@ -267,6 +268,11 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     return cudaSuccess;
 }
 
+// Cooperative launch: all CTAs of the persistent kernel are co-resident.
+cudaError_t launch_persistent(const void* fn, int grid, void** kargs, cudaStream_t stream) {
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), kargs, 0, stream);
+}
+
 int compress_impl(Context* c, const float* grad, float* residual, const int64_t* off, int S, float delta, int sid,
                   int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
                   const Params& prm) {
@@ -316,6 +322,8 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.G = c->G;
     c->call_id = (c->call_id + 1u) & 0x0fffffffu;
     a.call_id = (int)c->call_id;
+    a.residual_is_zero = c->residual_is_zero ? 1 : 0;
+    c->residual_is_zero = false;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
     // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
     static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
@@ -325,9 +333,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
                      : sid == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
-    static const bool plain = [] { const char* v = getenv("SIDCO_PLAIN_LAUNCH"); return v && v[0] == '1'; }();
-    if (plain) e = cudaLaunchKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
-    else e = cudaLaunchCooperativeKernel(fn, dim3(c->G), dim3(kThreads), kargs, 0, stream);
+    e = launch_persistent(fn, c->G, kargs, stream);
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
     return 0;
@@ -556,7 +562,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     const void* fn = sid_type == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
                      : sid_type == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
                                      : (const void*)sidco::sidco_persistent_kernel<2>;
-    e = cudaLaunchCooperativeKernel(fn, dim3(c.G), dim3(kThreads), kargs, 0, stream);
+    e = launch_persistent(fn, c.G, kargs, stream);
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
     return 0;
@@ -659,6 +665,7 @@ int sidco_reset_state(const float* residual) {
     if ((e = cudaMemcpy(base + c->L.seg, seg.data(), sizeof(SegDev) * (c->S + 1), cudaMemcpyHostToDevice)) != cudaSuccess)
         return (int)e;
     if ((e = cudaMemset(base + c->L.ctl, 0, sizeof(Control))) != cudaSuccess) return (int)e;
+    c->residual_is_zero = true;
     return 0;
 }
 
@@ -672,6 +679,7 @@ int sidco_reset_state_async(const float* residual, void* stream) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
+    c->residual_is_zero = true;
     return 0;
 }
 

@@ -112,6 +112,7 @@ struct Args {
     int Q, sid, max_stages;
     int C, S, G;
     int call_id;                 // per-workspace call number, tags SegDev::ready
+    int residual_is_zero;        // the residual's contents are to be taken as zeros and not read
     int vec_ok;                  // grad and residual are 16-byte aligned
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
 };
@@ -676,6 +677,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const int4 run = __ldg(A.cta_desc + cta);          // {first chunk, end chunk, first segment, segments}
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
+    const bool res_zero = A.residual_is_zero != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
@@ -761,7 +763,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         g4[j] = ld_stream4(A.grad + e0 + (b + j) * 128);
-                        r4[j] = *reinterpret_cast<const float4*>(A.residual + e0 + (b + j) * 128);
+                        r4[j] = res_zero ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                         : *reinterpret_cast<const float4*>(A.residual + e0 + (b + j) * 128);
                     }
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -781,14 +784,14 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     if (e + 4 <= lo || e >= hi) continue;
                     if (vec_ok && e >= lo && e + 4 <= hi) {
                         const float4 g = ld_stream4(A.grad + e);
-                        float4 r = *reinterpret_cast<const float4*>(A.residual + e);
+                        float4 r = res_zero ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(A.residual + e);
                         r.x += g.x; r.y += g.y; r.z += g.z; r.w += g.w;
                         *reinterpret_cast<float4*>(A.residual + e) = r;
                         accumulate(r.x); accumulate(r.y); accumulate(r.z); accumulate(r.w);
                     } else {
                         for (int cc = 0; cc < 4; ++cc) {
                             if (e + cc >= lo && e + cc < hi) {
-                                const float a = __ldcs(A.grad + e + cc) + A.residual[e + cc];
+                                const float a = __ldcs(A.grad + e + cc) + (res_zero ? 0.0f : A.residual[e + cc]);
                                 A.residual[e + cc] = a;
                                 accumulate(a);
                             }

@@ -205,3 +205,37 @@ print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [o
         assert r.returncode == 0, r.stderr[-2000:]
         outs.append(json.loads(r.stdout.strip().splitlines()[-1]))
     assert outs[0] == outs[1] == outs[2]
+
+
+@pytest.mark.parametrize("use_async", [False, True])
+def test_reset_declares_the_residual_empty(use_async):
+    """After a reset the next call must behave as if the residual were all zeros, whatever it holds,
+    and the adaptation must start again from M = 1."""
+    import torch
+    from paper_2101_10761_b200 import binding as B
+    wl = W.config(2)
+    off = wl.seg_offsets
+    delta = f32(0.001)
+    run = GpuRun(off)
+    try:
+        state = O.new_state(wl.n_segs)
+        res_o = np.zeros(wl.d, np.float32)
+        for call in range(7):                      # past one adaptation point, residual now non-zero
+            ora = O.sidco_compress(wl.draw(call), res_o, off, delta, O.SID_GAMMA, 4, state=state)
+            gpu = run.step(wl.draw(call), delta, O.SID_GAMMA, 4)
+            check_parity(gpu, ora, off, state)
+            res_o = ora.residual
+        assert any(st.M > 1 for st in state)
+        if use_async:
+            B.sidco_reset_state_async(run.res)
+        else:
+            B.sidco_reset_state(run.res)
+        state = O.new_state(wl.n_segs)
+        res_o = np.zeros(wl.d, np.float32)         # the GPU buffer still holds the old residual
+        for call in range(3):
+            ora = O.sidco_compress(wl.draw(20 + call), res_o, off, delta, O.SID_GAMMA, 4, state=state)
+            gpu = run.step(wl.draw(20 + call), delta, O.SID_GAMMA, 4)
+            check_parity(gpu, ora, off, state)
+            res_o = ora.residual
+    finally:
+        run.close()
