@@ -700,7 +700,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[R.seg_lo + i];
             sm_meff[i] = m;
             const float tau = A.seg[R.seg_lo + i].spec_thr;
-            sm_tau[i] = (A.spec_enable && m == 1 && tau > 0.0f) ? tau : -1.0f;
+            sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
             sm_ok[i] = 0;
         }
         if (q1 > q0) atomicMax(&sm_mloc, m);
@@ -715,11 +715,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0);
     __syncthreads();
 
-    // Candidate threshold of a segment for this call: only single-stage segments use one.  It depends
-    // on state the previous call left behind, so every warp and every phase derives the same value.
+    // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
+    // that precedes their last fit records which slots may hold survivors).  It depends on state the
+    // previous call left behind, so every warp and every phase derives the same value.
     auto spec_tau = [&](int seg) -> float {
         if (seg - R.seg_lo < kSegCache) return sm_tau[seg - R.seg_lo];
-        if (!A.spec_enable || stages_of(seg) != 1) return -1.0f;
+        if (!A.spec_enable || stages_of(seg) > 2) return -1.0f;
         const float tau = A.seg[seg].spec_thr;
         return tau > 0.0f ? tau : -1.0f;
     };
@@ -734,7 +735,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             const int c = cur.c, lo = cur.lo, hi = cur.hi;
             const int wb = lo & ~(kChunk - 1);
             const int e0 = wb + lane * 4;
-            if (cur.seg != tau_seg) { tau_seg = cur.seg; tau = spec_tau(cur.seg); }
+            if (cur.seg != tau_seg) {
+                tau_seg = cur.seg;
+                tau = stages_of(cur.seg) == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments flag in P3
+            }
             unsigned flags = 0;
 
             double s1 = 0.0, s2 = 0.0, prod = 1.0;
@@ -862,17 +866,38 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                                 sy += y;
                                 if (SID != kSidExp) sy2 = fma(y, y, sy2);
                             }
-                    const int e0 = wb + lane * 4;
-                    const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                        A.side_idx[p] = e0 + j * 128 + cc;
-                        A.side_val[p] = v[j][cc];
-                    });
-                    Sums r = warp_tree(sy, sy2, 0);
-                    if (lane == 0) {
-                        A.part[3 * (size_t)c + 0] = r.a;
-                        A.part[3 * (size_t)c + 1] = r.b;
-                        A.part_n[c] = cnt;
-                        A.side_cnt[c] = cnt;
+                    const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
+                    const bool full = vec_ok && lo == wb && hi == wb + kChunk;
+                    if (tau2 > 0.0f && full) {
+                        // Stage 2 is this segment's last: nothing reads the exceedances again except the
+                        // final selection, which can work from slot flags (as after P1 for one stage).
+                        unsigned flags = 0;
+                        #pragma unroll
+                        for (int j = 0; j < kSlots; ++j) {
+                            const float big = fmaxf(fmaxf(fabsf(v[j][0]), fabsf(v[j][1])),
+                                                    fmaxf(fabsf(v[j][2]), fabsf(v[j][3])));
+                            flags |= (unsigned)(big >= tau2) << j;
+                        }
+                        A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
+                        Sums r = warp_tree(sy, sy2, __popc(mask));
+                        if (lane == 0) {
+                            A.part[3 * (size_t)c + 0] = r.a;
+                            A.part[3 * (size_t)c + 1] = r.b;
+                            A.part_n[c] = r.n;
+                        }
+                    } else {
+                        const int e0 = wb + lane * 4;
+                        const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                            A.side_idx[p] = e0 + j * 128 + cc;
+                            A.side_val[p] = v[j][cc];
+                        });
+                        Sums r = warp_tree(sy, sy2, 0);
+                        if (lane == 0) {
+                            A.part[3 * (size_t)c + 0] = r.a;
+                            A.part[3 * (size_t)c + 1] = r.b;
+                            A.part_n[c] = cnt;
+                            A.side_cnt[c] = cnt;
+                        }
                     }
                 }
                 cur = nxt;
@@ -936,7 +961,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     publish_params(A, R, 0, -1, 100);
     {
         SegView sv;
-        bool seg_from_side = false, seg_flagged = false;
+        bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
         Desc cur = fetch_desc(A, queue.next(!p1_desc), true, true);
         while (cur.c >= 0) {
@@ -948,12 +973,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 // multi-stage segments keep their exceedances in the side region; single-stage ones
                 // have valid candidate flags if the candidate threshold proved low enough
                 const float tau = spec_tau(cur.seg);
+                seg_two_flagged = sv.M_eff == 2 && tau > 0.0f;      // P3 wrote flags for its full chunks
                 seg_from_side = sv.M_eff >= 2;
-                seg_flagged = !seg_from_side && tau > 0.0f && sv.thr_ge >= tau;
+                seg_flagged = tau > 0.0f && sv.thr_ge >= tau;
             }
-            const bool from_side = seg_from_side;
             const int c = cur.c, lo = cur.lo;
             const int wb = lo & ~(kChunk - 1);
+            // a full chunk of a flag-carrying two-stage segment has no side region: it is read from acc,
+            // through its flags if they proved valid, in full otherwise
+            const bool from_side = seg_from_side && !(seg_two_flagged && vec_ok && lo == wb && cur.hi == wb + kChunk);
             int cnt = 0;
             if (from_side) {
                 // compact list of stage-2 exceedances: lanes stride over it, one ballot per 32 entries
