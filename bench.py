@@ -36,6 +36,22 @@ if ROOT not in sys.path:
 METRIC = "SIDCo compress GB/s on minimal bytes (12 d + 8 k_hat) at d=25.6M, delta=1e-3"
 UNIT = "GB/s"
 DELTA = float(np.float32(1e-3))
+
+
+def metric_name():
+    if CONFIG == 4 and abs(DELTA - 1e-3) < 1e-6:
+        return METRIC
+    return "SIDCo compress GB/s on minimal bytes (12 d + 8 k_hat)"
+
+
+CONFIG = 4                 # which of the five synthetic configurations (default: the one the metric is quoted on)
+WORKLOAD_NAMES = {
+    1: "laplace d=262144 1 segment (configs[0])",
+    2: "resnet20-shaped d=269722 20 segments (configs[1])",
+    3: "vgg16-shaped d=14719818 16 segments (configs[2])",
+    4: "resnet50-shaped d=25557032 161 segments delta=1e-3 (configs[3])",
+    5: "lstm-ptb-shaped d=66034000 6 segments (configs[4])",
+}
 SID_NAMES = {0: "EXP", 1: "GAMMA", 2: "GPD"}
 RUN_LEN = 10               # consecutive calls per run (residual carried), then residual and state reset
 N_GRADS = RUN_LEN          # one fresh draw per call of a run
@@ -135,7 +151,7 @@ class ClockSampler(threading.Thread):
 
 def make_inputs():
     from paper_2101_10761_b200 import workloads as W
-    wl = W.config(4)
+    wl = W.config(CONFIG)
     return wl, [wl.draw(c) for c in range(N_GRADS)]
 
 
@@ -170,7 +186,7 @@ def run_reference(args):
         return
     from oracle import sidco_oracle as O
     from paper_2101_10761_b200 import workloads as W
-    wl = W.config(4)
+    wl = W.config(CONFIG)
     # bounded sample: a prefix of whole segments sized so that K + W steps end within ~2 minutes
     probe = wl.draw(0)
     t0 = time.perf_counter()
@@ -200,10 +216,10 @@ def run_reference(args):
     value = bytes_min / dt / 1e9
     sample = f"first {n_seg} of {wl.n_segs} segments ({d_sub} of {wl.d} elements) per step"
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric_name(), "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "resnet50-shaped d=25557032 161 segments delta=1e-3", "sid": SID_NAMES[args.sid],
+        "config": {"workload": WORKLOAD_NAMES[CONFIG], "delta": DELTA, "sid": SID_NAMES[args.sid],
                    "max_stages": 4, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": used_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -389,11 +405,11 @@ def run_gpu(args):
         achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
         cpu_val, cpu_calls, cpu_dt = oracle_rate(wl, grads_h, args.cpu_budget, args.sid)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": metric_name(), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": t_dev / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 data, f64 statistics and fits", "data": "synthetic",
             "config": {
-                "workload": "resnet50-shaped d=25557032 161 segments delta=1e-3 (configs[3])",
+                "workload": WORKLOAD_NAMES[CONFIG], "delta": DELTA,
                 "sid": SID_NAMES[args.sid], "max_stages": args.max_stages,
                 "M_used_hist_last_call": m_hist, "status_or": status_or,
                 "k_hat_mean": float(k_hats.mean()), "parallelism": "replicas only" if world > 1 else "1 GPU",
@@ -407,7 +423,7 @@ def run_gpu(args):
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": "of " + peak_kind,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.sid, args.max_stages)),
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((args.sid, args.max_stages)) if CONFIG == 4 else None,
                 "kernel": "sidco_persistent_kernel", "kernel_avg_ms": kern_avg_ms,
                 "kernel_min_ms": min(kern_ms), "algorithmic_bytes_per_launch": alg_bytes,
             },
@@ -443,7 +459,13 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="skip the short runs of other SID/stage settings")
     ap.add_argument("--prewarm-ms", type=float, default=300.0,
                     help="untimed steps run for this long before the warm-up to bring the clocks up")
+    ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5],
+                    help="synthetic configuration (default 4, the one the metric is quoted on)")
+    ap.add_argument("--delta", type=float, default=None, help="target ratio (default 1e-3; 1e-2 for configs 1-2)")
     args = ap.parse_args()
+    global CONFIG, DELTA
+    CONFIG = args.config
+    DELTA = float(np.float32(args.delta if args.delta is not None else (1e-2 if CONFIG <= 2 else 1e-3)))
     if args.warmup < 3:
         args.warmup = 3
     if args.steps is None:
