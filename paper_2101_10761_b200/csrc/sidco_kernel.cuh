@@ -20,12 +20,15 @@
 //       of the previous call: if the new eta turns out >= tau (checked per segment)
 //       P5a fetches only the flagged slots of acc instead of all of it; otherwise
 //       it reads all of acc, so the result never depends on tau
-//   P3  (only if some segment uses M >= 2) exceedances |x| > eta_1 compacted, in
-//       order, into the chunk's side region together with the statistics of the
-//       shifted peaks (Lemma 2 / Corollary 2.1); fit of eta_2
+//   P3  (segments with M >= 2) statistics of the shifted peaks |x| - eta_1 over
+//       the exceedances |x| > eta_1 (Lemma 2 / Corollary 2.1) and fit of eta_2.
+//       Two-stage segments record slot flags here (as P1 does for one stage);
+//       segments with more stages compact their exceedances, in order, into the
+//       chunk's side region
 //   P4  (m = 3..M) statistics of side-region entries above eta_{m-1}; fit eta_m
-//   P5a survivors |x| >= eta_M staged per chunk in ascending order (from acc for
-//       M = 1, from the side region otherwise), selected residual entries zeroed
+//   P5a survivors |x| >= eta_M staged per chunk in ascending order (from the
+//       flagged slots of acc or all of acc for M <= 2, from the side region
+//       otherwise), selected residual entries zeroed
 //   P5b CTA bases from the per-CTA totals, chunk bases by a block scan, staged
 //       survivors copied to their final ascending positions, per-segment counts
 //       and stage adaptation (Algorithm 1, Adapt_Stages)
@@ -683,9 +686,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
     if (threadIdx.x == 0) { sm_gen = ld_acquire(&A.ctl->gen); sm_mloc = 1; }
-#ifdef SIDCO_DIAG_SPAN
-    if (threadIdx.x == 0) A.cta_ns[4 * cta + 1] = global_ns();
-#endif
     if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
     RunSegs R{run.z, run.w, sm_q0, sm_q1, sm_runs, sm_meff, sm_tau, sm_thr_gt, sm_thr_ge, sm_eta, sm_ok};
@@ -1146,9 +1146,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     }
 
     if (stamper) A.ctl->t_ns[5] = global_ns();
-#ifdef SIDCO_DIAG_SPAN
-    if (threadIdx.x == 0) A.cta_ns[4 * cta + 2] = global_ns();
-#endif
 }
 
 // Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared.  The ready
