@@ -380,6 +380,35 @@ __device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, do
 // ----------------------------------------------------------------------------
 
 __device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+
+// L2 residency hints.  The error-compensation memory is read and rewritten by every call, the gradient
+// is read once: acc lines are asked to stay in L2 (evict_last), gradient lines to leave first.
+__device__ __forceinline__ unsigned long long policy_evict_last() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 ld_hint4(const float* p, unsigned long long pol) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_hint4_nc(const float* p, unsigned long long pol) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ void st_hint4(float* p, float4 v, unsigned long long pol) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
+}
 __device__ __forceinline__ float4 ld_l2_4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 // Load the part [lo, hi) of the window starting at wb from `src` into registers in chunk order
@@ -681,6 +710,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
     const bool res_zero = A.residual_is_zero != 0;
+    const unsigned long long pol_last = policy_evict_last(), pol_first = policy_evict_first();
     const ChunkQueue queue{&sm_next, c0, c1};
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
@@ -766,14 +796,14 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     float4 g4[4], r4[4];
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        g4[j] = ld_stream4(A.grad + e0 + (b + j) * 128);
+                        g4[j] = ld_hint4_nc(A.grad + e0 + (b + j) * 128, pol_first);
                         r4[j] = res_zero ? make_float4(0.f, 0.f, 0.f, 0.f)
-                                         : *reinterpret_cast<const float4*>(A.residual + e0 + (b + j) * 128);
+                                         : ld_hint4(A.residual + e0 + (b + j) * 128, pol_last);
                     }
                     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         r4[j].x += g4[j].x; r4[j].y += g4[j].y; r4[j].z += g4[j].z; r4[j].w += g4[j].w;
-                        *reinterpret_cast<float4*>(A.residual + e0 + (b + j) * 128) = r4[j];
+                        st_hint4(A.residual + e0 + (b + j) * 128, r4[j], pol_last);
                         accumulate(r4[j].x); accumulate(r4[j].y); accumulate(r4[j].z); accumulate(r4[j].w);
                         const float big = fmaxf(fmaxf(fabsf(r4[j].x), fabsf(r4[j].y)),
                                                 fmaxf(fabsf(r4[j].z), fabsf(r4[j].w)));
