@@ -639,7 +639,10 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                 bool complete = takes_part && runs == 1;
                 if (takes_part && runs > 1) {
                     complete = atomicAdd(&sg->arrived, 1) == runs - 1;
-                    if (complete) sg->arrived = 0;
+                    if (complete) {
+                        sg->arrived = 0;
+                        __threadfence();     // acquire side: the other runs' partials are read next
+                    }
                 }
                 if (complete) {
                     if (q1 - q0 <= kSmallSeg) sm_small[atomicAdd(&sm_count[0], 1)] = i;
