@@ -99,7 +99,7 @@ typedef struct sidco_seg_debug {
  * stream      all device work is enqueued here; the call does not synchronise, except that the first
  *             call for a residual pointer (or for a new segment table) allocates and uploads tables.
  *
- * 16-byte aligned grad and residual take the vectorised path; other alignments are handled with scalar
+ * 32-byte aligned grad and residual take the vectorised path; other alignments are handled with scalar
  * accesses.
  */
 int sidco_compress(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs,

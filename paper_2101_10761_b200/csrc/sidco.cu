@@ -324,7 +324,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.call_id = (int)c->call_id;
     a.residual_is_zero = c->residual_is_zero ? 1 : 0;
     c->residual_is_zero = false;
-    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
+    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
     // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
     static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
     a.spec_enable = spec_on ? 1 : 0;
@@ -556,7 +556,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.G = c.G;
     c.call_id = (c.call_id + 1u) & 0x0fffffffu;
     a.call_id = (int)c.call_id;
-    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 15u) == 0;
+    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
     a.spec_enable = 1;
     void* kargs[] = {(void*)&a};
     const void* fn = sid_type == 0   ? (const void*)sidco::sidco_persistent_kernel<0>

@@ -15,7 +15,7 @@
 //   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
 //       of every chunk; the CTA whose run completes a segment sums the per-chunk
 //       partials in chunk order and fits eta_1 (Corollaries 1.1-1.3).  For
-//       single-stage segments the sweep also records, per lane and 4-element
+//       single-stage segments the sweep also records, per lane and 8-element
 //       slot, whether some |x| >= tau, tau being 0.8 times the segment's threshold
 //       of the previous call: if the new eta turns out >= tau (checked per segment)
 //       P5a fetches only the flagged slots of acc instead of all of it; otherwise
@@ -46,7 +46,8 @@ namespace sidco {
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 1024;                      // window: elements per full chunk (one warp)
-constexpr int kSlots = kChunk / 128;              // float4 slots per lane per chunk (8)
+constexpr int kComp = 8;                          // elements per slot: one 32-byte access per lane
+constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4)
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
 constexpr int kSegCache = 512;                    // segments of a CTA run whose table entries sit in shared memory
 constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
@@ -116,7 +117,7 @@ struct Args {
     int C, S, G;
     int call_id;                 // per-workspace call number, tags SegDev::ready
     int residual_is_zero;        // the residual's contents are to be taken as zeros and not read
-    int vec_ok;                  // grad and residual are 16-byte aligned
+    int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
 };
 
@@ -379,66 +380,80 @@ __device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, do
 // chunk access (one warp)
 // ----------------------------------------------------------------------------
 
-__device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+// 256-bit global accesses with an L2 eviction priority.  The error-compensation memory is read and
+// rewritten by every call and nearly fits in L2: its lines are asked to stay (evict_last).  The gradient
+// is read once: its lines are asked to leave first.  (Cache-policy operands on 128-bit accesses did not
+// change what stays resident; these qualified 256-bit forms do.)
+struct F8 { float v[kComp]; };
 
-// L2 residency hints.  The error-compensation memory is read and rewritten by every call, the gradient
-// is read once: acc lines are asked to stay in L2 (evict_last), gradient lines to leave first.
-__device__ __forceinline__ unsigned long long policy_evict_last() {
-    unsigned long long pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
+__device__ __forceinline__ F8 ld8_evict_first(const float* p) {
+    F8 r;
+    asm volatile("ld.global.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p));
+    return r;
 }
-__device__ __forceinline__ unsigned long long policy_evict_first() {
-    unsigned long long pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
+__device__ __forceinline__ F8 ld8_evict_last(const float* p) {
+    F8 r;
+    asm volatile("ld.global.L2::evict_last.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+                 : "l"(p) : "memory");
+    return r;
 }
-__device__ __forceinline__ float4 ld_hint4(const float* p, unsigned long long pol) {
-    float4 v;
-    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol) : "memory");
-    return v;
+__device__ __forceinline__ void st8_evict_last(float* p, const F8& r) {
+    asm volatile("st.global.L2::evict_last.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(r.v[0]), "f"(r.v[1]), "f"(r.v[2]), "f"(r.v[3]), "f"(r.v[4]), "f"(r.v[5]), "f"(r.v[6]), "f"(r.v[7])
+                 : "memory");
 }
-__device__ __forceinline__ float4 ld_hint4_nc(const float* p, unsigned long long pol) {
-    float4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
-    return v;
-}
-__device__ __forceinline__ void st_hint4(float* p, float4 v, unsigned long long pol) {
-    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
-                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
-}
-__device__ __forceinline__ float4 ld_l2_4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
-// Load the part [lo, hi) of the window starting at wb from `src` into registers in chunk order
-// (slot, lane, component).  Returns the validity mask: bit 4*j + c.  Loads go through L2 only: the
-// data was written earlier in this kernel (by this SM) and is read once.
+// Error-compensation memory accesses: `keep` asks for L2 residency.  Segments with three or more stages
+// go without it, because their side regions (re-read by every later stage) need the L2 more.
+__device__ __forceinline__ F8 ld8_res(const float* p, bool keep) {
+    if (keep) return ld8_evict_last(p);
+    F8 r;
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(p)), b = __ldcg(reinterpret_cast<const float4*>(p) + 1);
+    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w; r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+    return r;
+}
+__device__ __forceinline__ void st8_res(float* p, const F8& r, bool keep) {
+    if (keep) { st8_evict_last(p, r); return; }
+    reinterpret_cast<float4*>(p)[0] = make_float4(r.v[0], r.v[1], r.v[2], r.v[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(r.v[4], r.v[5], r.v[6], r.v[7]);
+}
+
+// A chunk in registers: lane l holds, for slot j, the 8 elements at window offset 256 j + 8 l.
+// Chunk order (= ascending index) is slot, lane, component; mask bit 8 j + c stands for v[j][c].
+
+// Load the part [lo, hi) of the window starting at wb from `src` (the error-compensation memory).
+// Returns the validity mask.
 __device__ __forceinline__ unsigned load_chunk(const float* __restrict__ src, int lo, int hi, int wb, bool vec_ok,
-                                               float (&v)[kSlots][4]) {
-    const int e0 = wb + (threadIdx.x & 31) * 4;
+                                               bool keep, float (&v)[kSlots][kComp]) {
+    const int e0 = wb + (threadIdx.x & 31) * kComp;
     if (vec_ok && lo == wb && hi == wb + kChunk) {
         #pragma unroll
         for (int j = 0; j < kSlots; ++j) {
-            const float4 q = ld_l2_4(src + e0 + j * 128);
-            v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
+            const F8 q = ld8_res(src + e0 + j * 256, keep);
+            #pragma unroll
+            for (int c = 0; c < kComp; ++c) v[j][c] = q.v[c];
         }
         return kFull;
     }
     unsigned valid = 0;
     #pragma unroll
     for (int j = 0; j < kSlots; ++j) {
-        const int e = e0 + j * 128;
-        v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0.0f;
-        if (e + 4 <= lo || e >= hi) continue;
-        if (vec_ok && e >= lo && e + 4 <= hi) {
-            const float4 q = ld_l2_4(src + e);
-            v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
-            valid |= 0xFu << (4 * j);
+        const int e = e0 + j * 256;
+        #pragma unroll
+        for (int c = 0; c < kComp; ++c) v[j][c] = 0.0f;
+        if (e + kComp <= lo || e >= hi) continue;
+        if (vec_ok && e >= lo && e + kComp <= hi) {
+            const F8 q = ld8_res(src + e, keep);
+            #pragma unroll
+            for (int c = 0; c < kComp; ++c) v[j][c] = q.v[c];
+            valid |= 0xFFu << (8 * j);
         } else {
             #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (e + c >= lo && e + c < hi) { v[j][c] = __ldcg(src + e + c); valid |= 1u << (4 * j + c); }
+            for (int c = 0; c < kComp; ++c)
+                if (e + c >= lo && e + c < hi) { v[j][c] = __ldcg(src + e + c); valid |= 1u << (8 * j + c); }
         }
     }
     return valid;
@@ -446,23 +461,24 @@ __device__ __forceinline__ unsigned load_chunk(const float* __restrict__ src, in
 
 // Warp-ordered emission: calls emit(position, j, c) for every set bit of `mask`, positions counted
 // in chunk order starting at `base`.  Returns the number of set bits in the warp.
-template <int NS = kSlots, class Emit>
+template <class Emit>
 __device__ __forceinline__ int ordered_emit(unsigned mask, int base, Emit emit) {
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
     int run = base;
     #pragma unroll
-    for (int j = 0; j < NS; ++j) {
-        const unsigned nib = (mask >> (4 * j)) & 0xFu;
-        if (__ballot_sync(kFull, nib != 0) == 0) continue;
-        const int c = __popc(nib);
-        const unsigned b0 = __ballot_sync(kFull, c & 1);
-        const unsigned b1 = __ballot_sync(kFull, c & 2);
-        const unsigned b2 = __ballot_sync(kFull, c & 4);
-        int p = run + __popc(b0 & lt) + 2 * __popc(b1 & lt) + 4 * __popc(b2 & lt);
-        run += __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2);
+    for (int j = 0; j < kSlots; ++j) {
+        const unsigned byte = (mask >> (8 * j)) & 0xFFu;
+        if (__ballot_sync(kFull, byte != 0) == 0) continue;
+        const int n = __popc(byte);                       // 0..8 survivors of this lane in this slot
+        const unsigned b0 = __ballot_sync(kFull, n & 1);
+        const unsigned b1 = __ballot_sync(kFull, n & 2);
+        const unsigned b2 = __ballot_sync(kFull, n & 4);
+        const unsigned b3 = __ballot_sync(kFull, n & 8);
+        int p = run + __popc(b0 & lt) + 2 * __popc(b1 & lt) + 4 * __popc(b2 & lt) + 8 * __popc(b3 & lt);
+        run += __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2) + 8 * __popc(b3);
         #pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-            if (nib & (1u << cc)) { emit(p, j, cc); ++p; }
+        for (int cc = 0; cc < kComp; ++cc)
+            if (byte & (1u << cc)) { emit(p, j, cc); ++p; }
     }
     return run - base;
 }
@@ -508,26 +524,24 @@ __device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side,
     return d;
 }
 
-// Load only the flagged float4 slots of a full chunk of acc; the others read as zero.
+// Load only the flagged slots of a full chunk of acc; the others read as zero.
 __device__ __forceinline__ unsigned load_flagged(const float* __restrict__ src, int wb, unsigned flags,
-                                                 float (&v)[kSlots][4]) {
-    const int e0 = wb + (threadIdx.x & 31) * 4;
+                                                 float (&v)[kSlots][kComp]) {
+    const int e0 = wb + (threadIdx.x & 31) * kComp;
     unsigned valid = 0;
     #pragma unroll
     for (int j = 0; j < kSlots; ++j) {
-        v[j][0] = v[j][1] = v[j][2] = v[j][3] = 0.0f;
+        #pragma unroll
+        for (int c = 0; c < kComp; ++c) v[j][c] = 0.0f;
         if (flags & (1u << j)) {
-            const float4 q = ld_l2_4(src + e0 + j * 128);
-            v[j][0] = q.x; v[j][1] = q.y; v[j][2] = q.z; v[j][3] = q.w;
-            valid |= 0xFu << (4 * j);
+            const F8 q = ld8_evict_last(src + e0 + j * 256);
+            #pragma unroll
+            for (int c = 0; c < kComp; ++c) v[j][c] = q.v[c];
+            valid |= 0xFFu << (8 * j);
         }
     }
     return valid;
 }
-
-// ----------------------------------------------------------------------------
-// end of a statistics phase: arrivals and fits for the segments of this CTA's run
-// ----------------------------------------------------------------------------
 
 // Sum of the per-chunk partials q = first, first + stride, ... < q1, added in that order.  Loads are
 // issued eight chunks at a time so that a long segment costs few memory round trips.
@@ -713,7 +727,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
     const bool res_zero = A.residual_is_zero != 0;
-    const unsigned long long pol_last = policy_evict_last(), pol_first = policy_evict_first();
     const ChunkQueue queue{&sm_next, c0, c1};
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
@@ -762,15 +775,18 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     {
         int tau_seg = -1;
         float tau = -1.0f;
+        bool keep = true;          // ask for L2 residency of this segment's acc lines
         Desc cur = fetch_desc(A, queue.next(p1_desc), false);
         while (cur.c >= 0) {
             const Desc nxt = fetch_desc(A, queue.next(p1_desc), false);
             const int c = cur.c, lo = cur.lo, hi = cur.hi;
             const int wb = lo & ~(kChunk - 1);
-            const int e0 = wb + lane * 4;
+            const int e0 = wb + lane * kComp;
             if (cur.seg != tau_seg) {
                 tau_seg = cur.seg;
-                tau = stages_of(cur.seg) == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments flag in P3
+                const int m = stages_of(cur.seg);
+                tau = m == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments flag in P3
+                keep = m <= 2;
             }
             unsigned flags = 0;
 
@@ -795,21 +811,24 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
             if (vec_ok && lo == wb && hi == wb + kChunk) {
                 #pragma unroll
-                for (int b = 0; b < kSlots; b += 4) {
-                    float4 g4[4], r4[4];
+                for (int b = 0; b < kSlots; b += 2) {
+                    F8 g8[2], r8[2];
                     #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        g4[j] = ld_hint4_nc(A.grad + e0 + (b + j) * 128, pol_first);
-                        r4[j] = res_zero ? make_float4(0.f, 0.f, 0.f, 0.f)
-                                         : ld_hint4(A.residual + e0 + (b + j) * 128, pol_last);
+                    for (int j = 0; j < 2; ++j) {
+                        g8[j] = ld8_evict_first(A.grad + e0 + (b + j) * 256);
+                        if (!res_zero) r8[j] = ld8_res(A.residual + e0 + (b + j) * 256, keep);
                     }
                     #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        r4[j].x += g4[j].x; r4[j].y += g4[j].y; r4[j].z += g4[j].z; r4[j].w += g4[j].w;
-                        st_hint4(A.residual + e0 + (b + j) * 128, r4[j], pol_last);
-                        accumulate(r4[j].x); accumulate(r4[j].y); accumulate(r4[j].z); accumulate(r4[j].w);
-                        const float big = fmaxf(fmaxf(fabsf(r4[j].x), fabsf(r4[j].y)),
-                                                fmaxf(fabsf(r4[j].z), fabsf(r4[j].w)));
+                    for (int j = 0; j < 2; ++j) {
+                        float big = 0.0f;
+                        #pragma unroll
+                        for (int cc = 0; cc < kComp; ++cc) {
+                            const float a = res_zero ? g8[j].v[cc] : g8[j].v[cc] + r8[j].v[cc];
+                            r8[j].v[cc] = a;
+                            accumulate(a);
+                            big = fmaxf(big, fabsf(a));
+                        }
+                        st8_res(A.residual + e0 + (b + j) * 256, r8[j], keep);
                         flags |= (unsigned)(big >= tau) << (b + j);
                     }
                 }
@@ -817,16 +836,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             } else {
                 #pragma unroll 1
                 for (int j = 0; j < kSlots; ++j) {
-                    const int e = e0 + j * 128;
-                    if (e + 4 <= lo || e >= hi) continue;
-                    if (vec_ok && e >= lo && e + 4 <= hi) {
-                        const float4 g = ld_stream4(A.grad + e);
-                        float4 r = res_zero ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(A.residual + e);
-                        r.x += g.x; r.y += g.y; r.z += g.z; r.w += g.w;
-                        *reinterpret_cast<float4*>(A.residual + e) = r;
-                        accumulate(r.x); accumulate(r.y); accumulate(r.z); accumulate(r.w);
+                    const int e = e0 + j * 256;
+                    if (e + kComp <= lo || e >= hi) continue;
+                    if (vec_ok && e >= lo && e + kComp <= hi) {
+                        const F8 g = ld8_evict_first(A.grad + e);
+                        F8 r;
+                        if (!res_zero) r = ld8_res(A.residual + e, keep);
+                        #pragma unroll
+                        for (int cc = 0; cc < kComp; ++cc) {
+                            r.v[cc] = res_zero ? g.v[cc] : g.v[cc] + r.v[cc];
+                            accumulate(r.v[cc]);
+                        }
+                        st8_res(A.residual + e, r, keep);
                     } else {
-                        for (int cc = 0; cc < 4; ++cc) {
+                        for (int cc = 0; cc < kComp; ++cc) {
                             if (e + cc >= lo && e + cc < hi) {
                                 const float a = __ldcs(A.grad + e + cc) + (res_zero ? 0.0f : A.residual[e + cc]);
                                 A.residual[e + cc] = a;
@@ -880,21 +903,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     ++resweep;
                     const int c = cur.c, lo = cur.lo, hi = cur.hi;
                     const int wb = lo & ~(kChunk - 1);
-                    float v[kSlots][4];
-                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, v);
+                    float v[kSlots][kComp];
+                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, sv.M_eff <= 2, v);
                     unsigned mask = 0;
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j)
                         #pragma unroll
-                        for (int cc = 0; cc < 4; ++cc)
-                            if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (4 * j + cc);
+                        for (int cc = 0; cc < kComp; ++cc)
+                            if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (8 * j + cc);
                     mask &= valid;
                     double sy = 0.0, sy2 = 0.0;
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j)
                         #pragma unroll
-                        for (int cc = 0; cc < 4; ++cc)
-                            if (mask & (1u << (4 * j + cc))) {
+                        for (int cc = 0; cc < kComp; ++cc)
+                            if (mask & (1u << (8 * j + cc))) {
                                 const double y = (double)fabsf(v[j][cc]) - sv.eta_prev;
                                 sy += y;
                                 if (SID != kSidExp) sy2 = fma(y, y, sy2);
@@ -907,8 +930,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                         unsigned flags = 0;
                         #pragma unroll
                         for (int j = 0; j < kSlots; ++j) {
-                            const float big = fmaxf(fmaxf(fabsf(v[j][0]), fabsf(v[j][1])),
-                                                    fmaxf(fabsf(v[j][2]), fabsf(v[j][3])));
+                            float big = 0.0f;
+                            #pragma unroll
+                            for (int cc = 0; cc < kComp; ++cc) big = fmaxf(big, fabsf(v[j][cc]));
                             flags |= (unsigned)(big >= tau2) << j;
                         }
                         A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
@@ -919,9 +943,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                             A.part_n[c] = r.n;
                         }
                     } else {
-                        const int e0 = wb + lane * 4;
+                        const int e0 = wb + lane * kComp;
                         const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                            A.side_idx[p] = e0 + j * 128 + cc;
+                            A.side_idx[p] = e0 + j * 256 + cc;
                             A.side_val[p] = v[j][cc];
                         });
                         Sums r = warp_tree(sy, sy2, 0);
@@ -1047,20 +1071,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 const bool flagged = seg_flagged && vec_ok && lo == wb && hi == wb + kChunk;
                 if (!flagged) ++resweep;
                 if (!(flagged && __ballot_sync(kFull, cur.flags != 0) == 0)) {
-                    float v[kSlots][4];
+                    float v[kSlots][kComp];
                     const unsigned valid = flagged ? load_flagged(A.residual, wb, cur.flags, v)
-                                                   : load_chunk(A.residual, lo, hi, wb, vec_ok, v);
+                                                   : load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
                     unsigned mask = 0;
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j)
                         #pragma unroll
-                        for (int cc = 0; cc < 4; ++cc)
-                            if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (4 * j + cc);
+                        for (int cc = 0; cc < kComp; ++cc)
+                            if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (8 * j + cc);
                     mask &= valid;
                     if (__ballot_sync(kFull, mask != 0)) {
-                        const int e0 = wb + lane * 4;
+                        const int e0 = wb + lane * kComp;
                         cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
-                            const int e = e0 + j * 128 + cc;
+                            const int e = e0 + j * 256 + cc;
                             A.stage_idx[p] = e;
                             A.stage_val[p] = v[j][cc];
                             A.residual[e] = 0.0f;

@@ -107,7 +107,7 @@ def test_single_segment_sizes(n, sid, M):
 
 
 @pytest.mark.parametrize("sid", SIDS)
-@pytest.mark.parametrize("base_shift", [0, 1, 2, 3])
+@pytest.mark.parametrize("base_shift", [0, 1, 2, 3, 4])
 def test_unaligned_offsets_and_pointers(sid, base_shift):
     # offsets congruent to 1, 2, 3 (mod 4), empty segments, segments crossing tile windows
     sizes = [5, 0, 8190, 3, 0, 9001, 2, 16385, 1, 777, 0]
