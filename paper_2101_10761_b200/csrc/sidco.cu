@@ -155,7 +155,7 @@ int check_args(const void* grad, const void* residual, const int64_t* off, int n
 }
 
 // Build the chunk tables for a segment table and upload them together with fresh per-segment state.
-// keep_state: the adaptation state of an existing context survives a change of nothing but the tables.
+// The adaptation state of an existing context survives a table rebuild when the segment count is unchanged.
 cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t stream) {
     const int64_t d = off[S];
     DeviceInfo* di = nullptr;

@@ -57,7 +57,7 @@ constexpr long long kSpinLimit = 1ll << 22;       // bounded waits: ~1 s with th
 static_assert(kWarps == 32, "block_tree and the scans assume 32 warps per CTA");
 
 enum { kSidExp = 0, kSidGamma = 1, kSidGpd = 2 };
-enum { kStNonFinite = 1, kStDegenerate = 2, kStAllZero = 4, kStTimeout = 8 };
+enum { kStNonFinite = 1, kStDegenerate = 2, kStAllZero = 4, kStTimeout = 8, kStFlagsUsed = 16, kStFlagsMissed = 32 };
 
 struct SegDev {
     double eta[kMaxStages];
@@ -917,11 +917,13 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     for (int j = 0; j < kSlots; ++j)
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc)
-                            if (mask & (1u << (8 * j + cc))) {
-                                const double y = (double)fabsf(v[j][cc]) - sv.eta_prev;
-                                sy += y;
-                                if (SID != kSidExp) sy2 = fma(y, y, sy2);
-                            }
+                        {
+                            // branch-free: entries below the threshold contribute an exact zero
+                            const bool in = (mask >> (8 * j + cc)) & 1u;
+                            const double y = in ? (double)fabsf(v[j][cc]) - sv.eta_prev : 0.0;
+                            sy += y;
+                            if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                        }
                     const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
                     const bool full = vec_ok && lo == wb && hi == wb + kChunk;
                     if (tau2 > 0.0f && full) {
@@ -1197,8 +1199,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             sg->calls = calls;
             sg->k_sum = k_sum;
         }
-        // candidate threshold for the next call's first sweep
+        // candidate threshold for the next call's first sweep (and whether this call's guess held)
         const float thr = ld_cg(&sg->thr_ge);
+        {
+            const float tau_used = (A.spec_enable && seg_stages(A, s, cap) <= 2 && sg->spec_thr > 0.0f) ? sg->spec_thr : -1.0f;
+            if (tau_used > 0.0f) sg->status = ld_cg(&sg->status) | (thr >= tau_used ? kStFlagsUsed : kStFlagsMissed);
+        }
         sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
     }
 
