@@ -1,0 +1,68 @@
+"""Randomised GPU-vs-oracle parity: random segment tables (including very many tiny segments, so that
+one CTA's run spans more segments than its shared-memory cache holds), ratios, SIDs and stage counts."""
+import numpy as np
+import pytest
+
+from oracle import sidco_oracle as O
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, check_parity, f32
+
+pytestmark = pytest.mark.gpu
+
+
+def rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def run_case(sizes, scales, delta, sid, max_stages, calls, seed, zero_frac=0.0):
+    off = W.offsets_from_sizes(sizes)
+    d = int(off[-1])
+    r = rng(seed)
+    delta = f32(delta)
+    run = GpuRun(off)
+    res_o = np.zeros(d, np.float32)
+    state = O.new_state(len(sizes)) if max_stages > 0 else None
+    per_elem_scale = np.repeat(np.asarray(scales, np.float64), sizes)
+    try:
+        for call in range(calls):
+            g = (r.laplace(0.0, 1.0, d) * per_elem_scale).astype(np.float32)
+            if zero_frac:
+                g[r.random(d) < zero_frac] = 0.0
+            ora = O.sidco_compress(g, res_o, off, delta, sid, max_stages, state=state)
+            gpu = run.step(g, delta, sid, max_stages)
+            check_parity(gpu, ora, off, state)
+            res_o = ora.residual
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_segment_tables(seed):
+    r = rng(1000 + seed)
+    n_segs = int(r.integers(1, 60))
+    kinds = r.integers(0, 4, n_segs)
+    sizes = [int(x) for x in np.where(kinds == 0, r.integers(0, 8, n_segs),
+                              np.where(kinds == 1, r.integers(1, 300, n_segs),
+                              np.where(kinds == 2, r.integers(900, 5000, n_segs), r.integers(20000, 90000, n_segs))))]
+    scales = np.exp(r.uniform(np.log(1e-6), np.log(1e-1), n_segs))
+    delta = float(r.choice([0.3, 0.1, 0.03, 0.01, 0.003, 0.001]))
+    sid = int(r.integers(0, 3))
+    max_stages = int(r.choice([-1, -2, -3, -5, 2, 4, 6]))
+    run_case(sizes, scales, delta, sid, max_stages, calls=7 if max_stages > 0 else 2, seed=seed,
+             zero_frac=float(r.choice([0.0, 0.0, 0.5])))
+
+
+@pytest.mark.parametrize("sid,max_stages", [(0, -1), (1, 3), (2, -2)])
+def test_more_segments_per_run_than_the_cache_holds(sid, max_stages):
+    """~150,000 segments of 1-4 elements: every CTA run spans about a thousand segments, more than the
+    512 whose parameters are cached in shared memory and more than one 1024-thread pass of the arrival loop."""
+    r = rng(77)
+    sizes = [int(x) for x in r.integers(1, 5, 150000)]
+    scales = np.exp(r.uniform(np.log(1e-4), np.log(1e-2), len(sizes)))
+    run_case(sizes, scales, 0.3, sid, max_stages, calls=6 if max_stages > 0 else 2, seed=5)
+
+
+def test_mixed_giant_and_tiny_segments():
+    sizes = [3, 2_500_000, 1, 17, 1_200_000, 64, 64, 700_001, 5]
+    scales = [1e-3, 1e-4, 1.0, 1e-2, 1e-5, 1e-3, 1e-3, 1e-2, 1e-1]
+    run_case(sizes, scales, 0.001, O.SID_GPD, 4, calls=11, seed=9)

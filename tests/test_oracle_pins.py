@@ -402,3 +402,50 @@ def test_adaptive_compress_moves_M_on_misfit_data():
     assert used[5] == 2
     assert all(1 <= m <= 4 for m in used)
     assert all(abs(used[i + 1] - used[i]) <= 1 for i in range(9))
+
+
+# ------------------------------------------------------------------ invariants
+
+@pytest.mark.parametrize("sid", [O.SID_EXP, O.SID_GAMMA, O.SID_GPD])
+@pytest.mark.parametrize("M", [1, 2, 3])
+@pytest.mark.parametrize("k", [-20, 7])
+def test_scale_equivariance(sid, M, k):
+    # every fit is scale-equivariant: multiplying the data by 2^k (exact in floating point) multiplies
+    # every threshold by 2^k and selects the same positions
+    n = 50000
+    x = gamma_sample(n, 0.7, 1e-2, 900 + M)
+    r = laplace_acc(n, 1e-3, 901)
+    a = O.sidco_compress(x, r, [0, 20000, n], 0.01, sid, -M)
+    sc = np.float32(2.0 ** k)
+    b = O.sidco_compress(x * sc, r * sc, [0, 20000, n], 0.01, sid, -M)
+    assert np.array_equal(a.idx, b.idx)
+    assert np.array_equal(a.val * sc, b.val)
+    for ra, rb in zip(a.report, b.report):
+        for ea, eb in zip(ra.eta, rb.eta):
+            assert eb == pytest.approx(ea * 2.0 ** k, rel=1e-12)
+        assert ra.k_stage == rb.k_stage
+
+
+@pytest.mark.parametrize("sid", [O.SID_EXP, O.SID_GAMMA, O.SID_GPD])
+def test_permutation_invariance_within_a_segment(sid):
+    # thresholds depend on the multiset of magnitudes only; the selected values are the same multiset
+    n = 30000
+    x = gamma_sample(n, 0.5, 1.0, 950)
+    perm = rng(951).permutation(n)
+    a = O.sidco_compress(x, np.zeros_like(x), [0, n], 0.01, sid, -3)
+    b = O.sidco_compress(x[perm], np.zeros_like(x), [0, n], 0.01, sid, -3)
+    for ea, eb in zip(a.report[0].eta, b.report[0].eta):
+        assert eb == pytest.approx(ea, rel=1e-12)
+    assert a.report[0].k_stage == b.report[0].k_stage
+    assert np.array_equal(np.sort(a.val), np.sort(b.val))
+    assert np.array_equal(np.sort(perm[b.idx]), a.idx)
+
+
+def test_sign_symmetry():
+    # the model is symmetric around zero: flipping signs changes nothing but the signs of the values
+    n = 20000
+    x = laplace_acc(n, 1e-2, 960)
+    a = O.sidco_compress(x, np.zeros_like(x), [0, n], 0.01, O.SID_GPD, -2)
+    b = O.sidco_compress(-x, np.zeros_like(x), [0, n], 0.01, O.SID_GPD, -2)
+    assert np.array_equal(a.idx, b.idx) and np.array_equal(a.val, -b.val)
+    assert a.report[0].eta == b.report[0].eta
