@@ -59,7 +59,7 @@ N_GRADS = RUN_LEN          # one fresh draw per call of a run
 # DRAM bytes per launch of the persistent kernel on this workload (dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture, summarised under profiles/), keyed by (sid, max_stages).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    (0, 4): 257.9e6,     # EXP, adaptive: mean over the ten launches of one run
+    (0, 4): 236.8e6,     # EXP, adaptive: mean over the ten launches of one run
 }
 
 
