@@ -83,7 +83,8 @@ struct Context {
     size_t ws_bytes = 0;
     bool ws_owned = false;
     bool tables_valid = false;
-    unsigned call_id = 0;                  // tags the per-segment ready words
+    unsigned call_id = 0;                  // tags the per-segment published words
+    unsigned barrier_count = 0;            // grid-barrier arrivals recorded in the workspace's Control so far
     bool residual_is_zero = false;         // set by a state reset: the next call does not read the residual
     Layout L{};
     // staging for sidco_compress_host
@@ -254,6 +255,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
+    c->barrier_count = 0;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
@@ -322,6 +324,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.G = c->G;
     c->call_id = (c->call_id + 1u) & 0x0fffffffu;
     a.call_id = (int)c->call_id;
+    a.barrier_target = c->barrier_count + (unsigned)c->G;
     a.residual_is_zero = c->residual_is_zero ? 1 : 0;
     c->residual_is_zero = false;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
@@ -335,6 +338,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
     e = launch_persistent(fn, c->G, kargs, stream);
     if (e != cudaSuccess) return (int)e;
+    c->barrier_count += (unsigned)c->G;
     g_launches.fetch_add(1);
     return 0;
 }
@@ -556,6 +560,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.G = c.G;
     c.call_id = (c.call_id + 1u) & 0x0fffffffu;
     a.call_id = (int)c.call_id;
+    a.barrier_target = (unsigned)c.G;      // the Control block, arrival count included, was cleared above
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
     a.spec_enable = 1;
     void* kargs[] = {(void*)&a};
@@ -665,6 +670,7 @@ int sidco_reset_state(const float* residual) {
     if ((e = cudaMemcpy(base + c->L.seg, seg.data(), sizeof(SegDev) * (c->S + 1), cudaMemcpyHostToDevice)) != cudaSuccess)
         return (int)e;
     if ((e = cudaMemset(base + c->L.ctl, 0, sizeof(Control))) != cudaSuccess) return (int)e;
+    c->barrier_count = 0;
     c->residual_is_zero = true;
     return 0;
 }

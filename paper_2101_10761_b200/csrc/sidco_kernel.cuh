@@ -50,6 +50,9 @@ constexpr int kComp = 8;                          // elements per slot: one 32-b
 constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4)
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
 constexpr int kSegCache = 512;                    // segments of a CTA run whose table entries sit in shared memory
+constexpr int kCoopChunks = 4096;                 // chunks of a run the block-wide flagged-slot pass can cover
+constexpr int kCoopPass = kThreads / 2;           // chunks per pass of it (two threads per chunk)
+constexpr int kCoopItems = 4096;                  // flagged slots one pass can list
 constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
@@ -71,13 +74,18 @@ struct SegDev {
     int32_t M;           // adaptation state: stage count for the next adaptive call
     int32_t calls;
     long long k_sum;
+    // Published with release semantics by the thread that fits a stage and polled with acquire semantics by
+    // the runs that wait for it.  Low word: call_id * 16 + number of stages fitted so far in that call.  High
+    // word: the fp32 compare threshold of the newest stage, thr_ge if that stage is the segment's last,
+    // thr_gt otherwise, so that a waiting thread has it with the same load that tells it the stage is fitted.
+    unsigned long long pub;
     float spec_thr;      // candidate threshold for the next call's first sweep (<= 0: none), see P1
-    int32_t ready;       // call_id * 16 + number of stages fitted so far in that call (release/acquire)
+    int32_t pad;
 };
 
 struct Control {
-    unsigned count;      // grid barrier arrivals of the current generation (reset by the last arriver)
-    unsigned gen;        // grid barrier generation, never reset
+    unsigned count;      // grid barrier arrivals since the workspace was set up (never reset by the kernel)
+    unsigned unused;
     int timeout;         // set when a bounded wait ran out
     int pad;
     unsigned long long t_ns[16];  // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
@@ -115,7 +123,8 @@ struct Args {
     double delta, delta1, eps_H, eps_L;
     int Q, sid, max_stages;
     int C, S, G;
-    int call_id;                 // per-workspace call number, tags SegDev::ready
+    int call_id;                 // per-workspace call number, tags SegDev::pub
+    unsigned barrier_target;     // value of Control::count once every CTA of this call has arrived
     int residual_is_zero;        // the residual's contents are to be taken as zeros and not read
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
@@ -145,32 +154,33 @@ __device__ __forceinline__ int ld_volatile(const int* p) {
     return *reinterpret_cast<const volatile int*>(p);
 }
 
-__device__ __forceinline__ void st_release(int* p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-__device__ __forceinline__ int ld_acquire_s32(const int* p) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
 
-// Grid-wide barrier: the last CTA to arrive clears the arrival count and advances the generation;
-// the others wait for the generation to reach `target_gen`.  All CTAs of the cooperative launch are
-// resident, so the wait normally ends within microseconds; it is nevertheless bounded, and a
-// time-out raises Control::timeout, after which every later wait returns at once.
-__device__ __forceinline__ void grid_barrier(Control* ctl, int G, unsigned target_gen) {
+// Grid-wide barrier, used once per call: every CTA adds one arrival to a counter that is never reset and
+// waits until it reaches the value the host computed for this call (arrivals before the call + grid size),
+// so the last arrival releases the others with the same atomic that records it.  All CTAs of the
+// cooperative launch are resident, so the wait normally ends within microseconds; it is nevertheless
+// bounded, and a CTA whose wait runs out raises the timeout flag, which ends every other wait of the call.
+__device__ __forceinline__ void grid_barrier(Control* ctl, unsigned target) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         const unsigned old = atomicAdd(&ctl->count, 1u);
-        if (old == (unsigned)G - 1u) {
-            ctl->count = 0u;
-            __threadfence();
-            atomicAdd(&ctl->gen, 1u);
-        } else {
+        if ((int)(old + 1u - target) < 0) {
             long long spins = 0;
-            while ((int)(ld_acquire(&ctl->gen) - target_gen) < 0) {
+            while ((int)(ld_acquire(&ctl->count) - target) < 0) {       // wrap-safe
                 if (ld_volatile(&ctl->timeout)) break;
                 if (++spins > kSpinLimit) { atomicExch(&ctl->timeout, 1); break; }
                 __nanosleep(spins < 64 ? 20 : 200);
@@ -181,29 +191,26 @@ __device__ __forceinline__ void grid_barrier(Control* ctl, int G, unsigned targe
     __syncthreads();
 }
 
-// Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).
-__device__ __forceinline__ void wait_ready_thread(const Args& A, const SegDev* sg, int need) {
+// Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).  Returns the
+// threshold published with that stage.  Only runs holding chunks of the segment wait for it, and the next
+// stage cannot be fitted before they have swept those chunks, so the word read is the one of stage `need`.
+__device__ __forceinline__ float wait_ready_thread(const Args& A, const SegDev* sg, int need) {
     const unsigned target = (unsigned)A.call_id * 16u + (unsigned)need;
     long long spins = 0;
-    while ((int)((unsigned)ld_acquire_s32(&sg->ready) - target) < 0) {     // wrap-safe
+    unsigned long long w;
+    while ((int)((unsigned)(w = ld_acquire_u64(&sg->pub)) - target) < 0) {     // wrap-safe
         if (ld_volatile(&A.ctl->timeout)) break;
         if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
         __nanosleep(spins < 16 ? 20 : 100);
     }
+    return __uint_as_float((unsigned)(w >> 32));
 }
 
 // Warp-level wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).
-__device__ __forceinline__ void wait_ready(const Args& A, const SegDev* sg, int need) {
-    if ((threadIdx.x & 31) == 0) {
-        const unsigned target = (unsigned)A.call_id * 16u + (unsigned)need;
-        long long spins = 0;
-        while ((int)((unsigned)ld_acquire_s32(&sg->ready) - target) < 0) {     // wrap-safe
-            if (ld_volatile(&A.ctl->timeout)) break;
-            if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
-            __nanosleep(spins < 16 ? 20 : 100);
-        }
-    }
-    __syncwarp();
+__device__ __forceinline__ float wait_ready(const Args& A, const SegDev* sg, int need) {
+    float thr = 0.0f;
+    if ((threadIdx.x & 31) == 0) thr = wait_ready_thread(A, sg, need);
+    return __shfl_sync(kFull, thr, 0);
 }
 
 struct Sums { double a, b; int n; };
@@ -238,6 +245,30 @@ __device__ __forceinline__ Sums block_tree(double a, double b, int n, double (*s
         r.a = x; r.b = y; r.n = (int)z;
     }
     return r;
+}
+
+// Block-wide exclusive prefix sum of one int per thread (thread order); `total` is the block's sum.
+// `sm` holds one int per warp and may be reused after the call returns.
+__device__ __forceinline__ int block_exscan(int x, int* sm, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = x;
+    #pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();                       // previous use of sm is over
+    if (lane == 31) sm[warp] = incl;
+    __syncthreads();
+    int w = sm[lane];                      // every warp scans the 32 warp sums itself
+    #pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, w, o);
+        if (lane >= o) w += t;
+    }
+    total = __shfl_sync(kFull, w, 31);
+    const int warp_incl = __shfl_sync(kFull, w, warp);
+    return warp_incl - sm[warp] + incl - x;
 }
 
 // ----------------------------------------------------------------------------
@@ -277,31 +308,61 @@ __device__ inline double stage_ratio(double delta, double delta1, int M, int m) 
     return delta / p;
 }
 
-// Corollary 1.3 / Lemma 2: moment-matched generalised Pareto quantile at tail probability `ratio`.
-// A variance at rounding-noise level (raw-moment form) is treated as zero: the formula's limit is `mean`.
-__device__ inline double gpd_step(double mean, double var, double ratio, int& status) {
+// Logarithms of the stage ratios, computed once per CTA: slot 0 is delta_1 (every stage but the last), slot M
+// the ratio of the last stage of an M-stage schedule (delta for M = 1).
+struct LnTab {
+    const double* ln;       // [kMaxStages + 1] log(ratio)
+    const double* ln_inv;   // [kMaxStages + 1] log(1 / ratio)
+};
+__device__ __forceinline__ int ratio_slot(int M, int m) { return (M == 1 || m == M - 1) ? M : 0; }
+
+// Corollary 1.3 / Lemma 2: moment-matched generalised Pareto quantile at the tail probability whose
+// logarithms are given.  A variance at rounding-noise level (raw-moment form) is treated as zero: the
+// formula's limit is `mean`.
+__device__ inline double gpd_step(double mean, double var, double ln_ratio, double ln_inv_ratio, int& status) {
     if (!(var > 1e-12 * mean * mean)) { status |= kStDegenerate; return mean; }
     const double R = mean * mean / var;
     const double alpha = 0.5 * (1.0 - R);
     const double beta = 0.5 * mean * (R + 1.0);
-    const double t = -alpha * log(ratio);
-    if (fabs(t) < 1e-12) return beta * log(1.0 / ratio);
+    const double t = -alpha * ln_ratio;
+    if (fabs(t) < 1e-12) return beta * ln_inv_ratio;
     return (beta / alpha) * expm1(t);
 }
 
 // Corollary 1.1 / 2.1.
-__device__ inline double exp_step(double mean, double ratio) { return mean * log(1.0 / ratio); }
+__device__ inline double exp_step(double mean, double ln_inv_ratio) { return mean * ln_inv_ratio; }
 
-__device__ inline void publish_eta(SegDev* sg, int m, double eta) {
-    sg->eta[m] = eta;
-    sg->thr_gt = __double2float_rd(eta);
-    sg->thr_ge = __double2float_ru(eta);
+// What the fitting thread hands to its own CTA (the other runs of the segment read SegDev::pub).
+struct Fit {
+    double eta;
+    float thr;          // thr_ge(eta) if the stage is the segment's last, thr_gt(eta) otherwise
+    int stages;         // stages fitted so far
+    bool last;
+};
+
+// Publish a fitted stage: the tagged threshold word goes out first; everything else about the stage is
+// stored by the caller afterwards.  If another stage follows, its sweep shifts by eta, which is therefore
+// stored before the word and released with it.  The word of a last stage carries all that its readers need
+// (they go on to read only their own run's data), so it is a plain strong store with no fence to wait for.
+// The caller's later stores are ordered before any later fit of the segment by the fence and arrival atomic
+// of this CTA's next phase, and before the final placement by the grid barrier.
+__device__ inline Fit publish_stage(const Args& A, SegDev* sg, int stages, bool last, double eta) {
+    Fit f{eta, last ? __double2float_ru(eta) : __double2float_rd(eta), stages, last};
+    const unsigned long long word = ((unsigned long long)__float_as_uint(f.thr) << 32) |
+                                    (unsigned long long)((unsigned)A.call_id * 16u + (unsigned)stages);
+    if (last) {
+        st_relaxed_u64(&sg->pub, word);
+    } else {
+        sg->eta[stages - 1] = eta;
+        st_release_u64(&sg->pub, word);
+    }
+    return f;
 }
 
 // Stage 1 from the segment sums: S1 = sum|x|, and S2 = sum x^2 (GPD) or SL = sum log|x| over the
 // n_nz nonzero magnitudes (gamma).
-__device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n, double S1, double S2_or_SL,
-                                  int n_nz) {
+__device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, double S1, double S2_or_SL,
+                                 int n_nz, int cap, const LnTab& T) {
     int M;
     if (A.max_stages > 0) {
         M = M_state < 1 ? 1 : M_state;
@@ -309,11 +370,10 @@ __device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n,
     } else {
         M = -A.max_stages;
     }
-    const int cap = stage_cap(A.delta, A.delta1);
     const int M_eff = M < cap ? M : cap;
     int status = 0;
     double eta;
-    const double ratio = stage_ratio(A.delta, A.delta1, M_eff, 0);
+    const int slot = ratio_slot(M_eff, 0);
     if (n == 0) {
         eta = __longlong_as_double(0x7ff0000000000000ll);
     } else if (!isfinite(S1) || !isfinite(S2_or_SL)) {
@@ -323,18 +383,19 @@ __device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n,
         status |= kStAllZero;
         eta = __longlong_as_double(0x7ff0000000000000ll);
     } else if (A.sid == kSidExp) {
-        eta = exp_step(S1 / n, ratio);
+        eta = exp_step(S1 / n, T.ln_inv[slot]);
     } else if (A.sid == kSidGpd) {
         const double mu = S1 / n;
-        eta = gpd_step(mu, S2_or_SL / n - mu * mu, ratio, status);
+        eta = gpd_step(mu, S2_or_SL / n - mu * mu, T.ln[slot], T.ln_inv[slot], status);
     } else {
+        const double ratio = stage_ratio(A.delta, A.delta1, M_eff, 0);
         const double mu = S1 / n_nz;
         const double s = log(mu) - S2_or_SL / n_nz;
         double rz = ratio * n / n_nz;
         if (rz > 1.0) rz = 1.0;
         if (s <= 1e-12) {
             status |= kStDegenerate;
-            eta = exp_step(mu, rz);
+            eta = mu * log(1.0 / rz);
             if (!(eta > 0.0)) eta = 0.0;
         } else {
             const double alpha = (3.0 - s + sqrt((s - 3.0) * (s - 3.0) + 24.0 * s)) / (12.0 * s);
@@ -343,37 +404,39 @@ __device__ inline void fit_stage1(const Args& A, SegDev* sg, int M_state, int n,
             if (eta <= 0.0) { status |= kStDegenerate; eta = 0.0; }
         }
     }
+    // an empty segment takes part in no later phase: all its stages count as fitted here
+    const Fit f = publish_stage(A, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
     sg->M_eff = M_eff;
     sg->status = status;
-    for (int m = 0; m < kMaxStages; ++m) { sg->eta[m] = 0.0; sg->k_stage[m] = 0; }
-    // an empty segment takes part in no later phase: all its stage thresholds are set here
-    if (n == 0)
-        for (int m = 1; m < M_eff; ++m) sg->eta[m] = eta;
-    publish_eta(sg, 0, eta);
-    __threadfence();
-    st_release(&sg->ready, (int)((unsigned)A.call_id * 16u + (unsigned)(n == 0 ? M_eff : 1)));
+    sg->eta[0] = eta;
+    for (int m = 1; m < kMaxStages; ++m) sg->eta[m] = (n == 0 && m < M_eff) ? eta : 0.0;
+    for (int m = 0; m < kMaxStages; ++m) sg->k_stage[m] = 0;
+    sg->thr_gt = __double2float_rd(eta);
+    sg->thr_ge = __double2float_ru(eta);
+    return f;
 }
 
-// Stage index m >= 1 (eta_{m+1} in the paper's numbering) from the shifted peaks over eta_m:
-// n_e = #{|x| > eta_m}, Sy = sum(|x| - eta_m), Sy2 = sum(|x| - eta_m)^2.
-__device__ inline void fit_stage_m(const Args& A, SegDev* sg, int m, int n_e, double Sy, double Sy2) {
-    // fields another SM may have written during this call are read through L2
-    const double prev = ld_cg(&sg->eta[m - 1]);
-    sg->k_stage[m - 1] = n_e;
+// Stage index m >= 1 (eta_{m+1} in the paper's numbering) of an M_eff-stage segment from the shifted peaks
+// over prev = eta_m: n_e = #{|x| > eta_m}, Sy = sum(|x| - eta_m), Sy2 = sum(|x| - eta_m)^2.
+__device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, double prev, int n_e, double Sy,
+                                  double Sy2, const LnTab& T) {
     double eta = prev;
+    int status = 0;
     if (n_e > 0) {
-        const double ratio = stage_ratio(A.delta, A.delta1, ld_cg(&sg->M_eff), m);
+        const int slot = ratio_slot(M_eff, m);
         const double ybar = Sy / n_e;
-        int status = ld_cg(&sg->status);
         double inc;
-        if (A.sid == kSidExp) inc = exp_step(ybar, ratio);
-        else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, ratio, status);
-        sg->status = status;
+        if (A.sid == kSidExp) inc = exp_step(ybar, T.ln_inv[slot]);
+        else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, T.ln[slot], T.ln_inv[slot], status);
         eta = prev + inc;
     }
-    publish_eta(sg, m, eta);
-    __threadfence();
-    st_release(&sg->ready, (int)((unsigned)A.call_id * 16u + (unsigned)(m + 1)));
+    const Fit f = publish_stage(A, sg, m + 1, m + 1 == M_eff, eta);
+    sg->k_stage[m - 1] = n_e;
+    if (status) sg->status = ld_cg(&sg->status) | status;     // written by the previous stage's fit (maybe another SM)
+    sg->eta[m] = eta;
+    sg->thr_gt = __double2float_rd(eta);
+    sg->thr_ge = __double2float_ru(eta);
+    return f;
 }
 
 // ----------------------------------------------------------------------------
@@ -489,11 +552,11 @@ __device__ __forceinline__ int ordered_emit(unsigned mask, int base, Emit emit) 
 struct SegView {
     int seg = -1;
     int M_eff = 0;
-    float thr_gt = 0.f, thr_ge = 0.f;
+    float thr_gt = 0.f, thr_ge = 0.f;   // both hold the one threshold of the phase (see RunSegs::thr)
     double eta_prev = 0.0;
 };
 
-// Dynamic chunk queue of a CTA run// Dynamic chunk queue of a CTA run: warps take the next chunk index (ascending or descending).
+// Dynamic chunk queue of a CTA run: warps take the next chunk index (ascending or descending).
 struct ChunkQueue {
     int* sm_next;
     int c0, c1;
@@ -503,6 +566,15 @@ struct ChunkQueue {
         k = __shfl_sync(kFull, k, 0);
         if (k >= c1 - c0) return -1;
         return descending ? c1 - 1 - k : c0 + k;
+    }
+    // As next(), but passes over the chunks whose bit is set in `done` (bit = chunk - c0, first n_done chunks).
+    __device__ __forceinline__ int next_undone(bool descending, const unsigned* done, int n_done) const {
+        for (;;) {
+            const int c = next(descending);
+            if (c < 0) return -1;
+            const int k = c - c0;
+            if (k >= n_done || !((done[k >> 5] >> (k & 31)) & 1u)) return c;
+        }
     }
 };
 
@@ -572,12 +644,12 @@ struct RunSegs {
     int* q1;                    // [kSegCache] one past the last chunk
     int* runs;                  // [kSegCache] CTA runs holding chunks of the segment
     int* m_eff;                 // [kSegCache] stage count of the segment in this call
+    int* n;                     // [kSegCache] elements of the segment
     float* tau;                 // [kSegCache] candidate threshold for the first sweep (< 0: none)
     // thresholds of the phase being swept, published by one thread per segment (see publish_params)
-    float* thr_gt;              // [kSegCache]
-    float* thr_ge;              // [kSegCache]
+    float* thr;                 // [kSegCache] thr_gt of the stage the phase shifts by; thr_ge of the last stage in P5a
     double* eta_prev;           // [kSegCache]
-    volatile int* ok;           // [kSegCache] == phase tag once the three values above are valid
+    volatile int* ok;           // [kSegCache] == phase tag once the two values above are valid
     __device__ __forceinline__ void get(const Args& A, int i, int& a, int& b, int& r) const {
         if (i < kSegCache) { a = q0[i]; b = q1[i]; r = runs[i]; }
         else { a = A.seg_chunk0[seg_lo + i]; b = A.seg_chunk0[seg_lo + i + 1]; r = A.seg_runs[seg_lo + i]; }
@@ -587,15 +659,15 @@ struct RunSegs {
 // One thread per segment of the run waits (bounded) until the segment has the stages this phase needs,
 // then copies its thresholds into the shared-memory cache and marks them valid with the phase tag.
 // need: stages that must be fitted (0: all of the segment's); m_prev: index of the eta the phase shifts by.
+// A segment fitted by this CTA itself already has them (see arrive_and_fit).
 __device__ __forceinline__ void publish_params(const Args& A, const RunSegs& R, int need, int m_prev, int tag) {
     const int i = threadIdx.x;
-    if (i < R.n_seg && i < kSegCache && R.q1[i] > R.q0[i]) {
+    if (i < R.n_seg && i < kSegCache && R.q1[i] > R.q0[i] && R.ok[i] != tag) {
         const SegDev* sg = &A.seg[R.seg_lo + i];
         const int M_eff = R.m_eff[i];
-        wait_ready_thread(A, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
-        R.thr_gt[i] = ld_cg(&sg->thr_gt);
-        R.thr_ge[i] = ld_cg(&sg->thr_ge);
-        R.eta_prev[i] = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
+        R.thr[i] = wait_ready_thread(A, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
+        // only a segment with a further stage is swept in this phase and needs the shift
+        R.eta_prev[i] = (m_prev >= 0 && M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
         __threadfence_block();
         R.ok[i] = tag;
     }
@@ -615,25 +687,25 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
             __nanosleep(20);
         }
         __threadfence_block();
-        v.thr_gt = R.thr_gt[i];
-        v.thr_ge = R.thr_ge[i];
+        v.thr_gt = v.thr_ge = R.thr[i];
         v.eta_prev = R.eta_prev[i];
     } else {
         // beyond the cache (a run spanning more than kSegCache segments): straight from global memory
         const SegDev* sg = &A.seg[seg];
         v.M_eff = seg_stages(A, seg, cap);
-        wait_ready(A, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
-        v.thr_gt = ld_cg(&sg->thr_gt);
-        v.thr_ge = ld_cg(&sg->thr_ge);
-        v.eta_prev = m_prev >= 0 ? ld_cg(&sg->eta[m_prev]) : 0.0;
+        v.thr_gt = v.thr_ge = wait_ready(A, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
+        v.eta_prev = (m_prev >= 0 && v.M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
     }
 }
 
 // `stage` = 0 for the first stage, m >= 1 for the refits.  Every CTA calls this after its warps
 // have written the partials of all chunks of its run.  A segment that lies inside this run alone is
 // fitted at once; one shared with other runs is fitted by the run that arrives last.
-__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, int* sm_small,
-                                               int* sm_large, int* sm_count, double (*sm_red)[3], int stamp_slot) {
+// The fitting thread also puts the result into this CTA's own parameter cache, tagged for the phase that
+// uses it next, so that the CTA does not wait for its own publication to come back through L2.
+__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
+                                               int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3],
+                                               int stamp_slot) {
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {                                   // this CTA's sweep is over
@@ -642,6 +714,25 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
     }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // one thread: fit segment i2 of the run from its sums, publish, and fill the CTA's own cache entry
+    auto fit_and_cache = [&](SegDev* sg, int i2, int M_state, const Sums& r) {
+        const bool cached = i2 < kSegCache;
+        Fit f;
+        if (stage == 0) {
+            f = fit_stage1(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
+        } else {
+            // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
+            const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
+            const double prev = cached ? R.eta_prev[i2] : ld_cg(&sg->eta[stage - 1]);
+            f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T);
+        }
+        if (cached) {
+            R.thr[i2] = f.thr;
+            R.eta_prev[i2] = f.eta;
+            __threadfence_block();
+            R.ok[i2] = f.last ? 100 : f.stages;        // tag of the phase that uses these values next
+        }
+    };
     for (int base = 0; base < R.n_seg; base += kThreads) {
         const int i = base + (int)threadIdx.x;
         if (i < R.n_seg) {
@@ -649,7 +740,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
             R.get(A, i, q0, q1, runs);
             if (q1 > q0) {
                 SegDev* sg = &A.seg[R.seg_lo + i];
-                const bool takes_part = stage == 0 || seg_stages(A, R.seg_lo + i, cap) > stage;
+                const bool takes_part = stage == 0 || (i < kSegCache ? R.m_eff[i] : seg_stages(A, R.seg_lo + i, cap)) > stage;
                 bool complete = takes_part && runs == 1;
                 if (takes_part && runs > 1) {
                     complete = atomicAdd(&sg->arrived, 1) == runs - 1;
@@ -666,33 +757,30 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         }
         __syncthreads();
         const int n_small = sm_count[0], n_large = sm_count[1];
+        // large segments first (other runs wait for them): the whole CTA, threads stride over the chunk
+        // partials, fixed block tree
+        for (int k = 0; k < n_large; ++k) {
+            const int i2 = sm_large[k];
+            int q0, q1, runs;
+            R.get(A, i2, q0, q1, runs);
+            SegDev* sg = &A.seg[R.seg_lo + i2];
+            const int M_state = (stage == 0 && threadIdx.x == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
+            const Sums t = strided_partials(A, q0 + (int)threadIdx.x, q1, kThreads);
+            Sums r = block_tree(t.a, t.b, t.n, sm_red);
+            if (threadIdx.x == 0) fit_and_cache(sg, i2, M_state, r);
+        }
         // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
         for (int k = warp; k < n_small; k += kWarps) {
             const int i2 = sm_small[k];
             int q0, q1, runs;
             R.get(A, i2, q0, q1, runs);
             SegDev* sg = &A.seg[R.seg_lo + i2];
-            const int M_state = (stage == 0 && lane == 0) ? sg->M : 0;     // in flight with the partials
+            // (a cached stage count reproduces itself through fit_stage1's clamps; otherwise the state is
+            // loaded, in flight with the partials)
+            const int M_state = (stage == 0 && lane == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
             const Sums t = strided_partials(A, q0 + lane, q1, 32);
             Sums r = warp_tree(t.a, t.b, t.n);
-            if (lane == 0) {
-                if (stage == 0) fit_stage1(A, sg, M_state, A.seg_n[R.seg_lo + i2], r.a, r.b, r.n);
-                else fit_stage_m(A, sg, stage, r.n, r.a, r.b);
-            }
-        }
-        // large segments: the whole CTA, threads stride over the chunk partials, fixed block tree
-        for (int k = 0; k < n_large; ++k) {
-            const int i2 = sm_large[k];
-            int q0, q1, runs;
-            R.get(A, i2, q0, q1, runs);
-            SegDev* sg = &A.seg[R.seg_lo + i2];
-            const int M_state = (stage == 0 && threadIdx.x == 0) ? sg->M : 0;
-            const Sums t = strided_partials(A, q0 + (int)threadIdx.x, q1, kThreads);
-            Sums r = block_tree(t.a, t.b, t.n, sm_red);
-            if (threadIdx.x == 0) {
-                if (stage == 0) fit_stage1(A, sg, M_state, A.seg_n[R.seg_lo + i2], r.a, r.b, r.n);
-                else fit_stage_m(A, sg, stage, r.n, r.a, r.b);
-            }
+            if (lane == 0) fit_and_cache(sg, i2, M_state, r);
         }
         __syncthreads();
         if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
@@ -714,12 +802,17 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ int sm_next;
     __shared__ int sm_base;
     __shared__ int sm_resweep;
-    __shared__ unsigned sm_gen;
     __shared__ int sm_mloc;
-    __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache], sm_meff[kSegCache];
-    __shared__ float sm_tau[kSegCache], sm_thr_gt[kSegCache], sm_thr_ge[kSegCache];
+    __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache], sm_meff[kSegCache], sm_segn[kSegCache];
+    __shared__ float sm_tau[kSegCache], sm_thr[kSegCache];
+    __shared__ double sm_ln[kMaxStages + 1], sm_ln_inv[kMaxStages + 1];
     __shared__ double sm_eta[kSegCache];
     __shared__ int sm_ok[kSegCache];
+    __shared__ unsigned short sm_items[kCoopItems];
+    __shared__ int sm_cseg[kCoopPass], sm_cbase[kCoopPass], sm_ccnt[kCoopPass];
+    __shared__ unsigned sm_done[kCoopChunks / 32];
+    __shared__ int sm_coop_total;
+    __shared__ int sm_any_tau;
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -731,10 +824,17 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
-    if (threadIdx.x == 0) { sm_gen = ld_acquire(&A.ctl->gen); sm_mloc = 1; }
-    if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; }
+    if (threadIdx.x == 0) sm_mloc = 1;
+    if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
-    RunSegs R{run.z, run.w, sm_q0, sm_q1, sm_runs, sm_meff, sm_tau, sm_thr_gt, sm_thr_ge, sm_eta, sm_ok};
+    RunSegs R{run.z, run.w, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
+    const LnTab T{sm_ln, sm_ln_inv};
+    if (threadIdx.x <= kMaxStages) {
+        const int M = threadIdx.x;                    // slot 0: delta_1; slot M: last stage of M stages
+        const double ratio = M == 0 ? A.delta1 : stage_ratio(A.delta, A.delta1, M, M - 1);
+        sm_ln[M] = log(ratio);
+        sm_ln_inv[M] = log(1.0 / ratio);
+    }
     __syncthreads();
     auto stages_of = [&](int seg) -> int { return seg_stages(A, seg, cap); };
     // cache the run's segment table; find the largest stage count among the run's segments, which
@@ -745,8 +845,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (i < kSegCache) {
             sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[R.seg_lo + i];
             sm_meff[i] = m;
+            sm_segn[i] = A.seg_n[R.seg_lo + i];
             const float tau = A.seg[R.seg_lo + i].spec_thr;
             sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
+            if (sm_tau[i] > 0.0f && q1 > q0) sm_any_tau = 1;
             sm_ok[i] = 0;
         }
         if (q1 > q0) atomicMax(&sm_mloc, m);
@@ -758,7 +860,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
-        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0);
+        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
     __syncthreads();
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
@@ -884,7 +986,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             cur = nxt;
         }
     }
-    arrive_and_fit(A, R, 0, cap, sm_list, sm_scan, sm_count, sm_red, 6);
+    arrive_and_fit(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6);
     if (threadIdx.x == 0) sm_next = 0;
     __syncthreads();
     const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
@@ -962,7 +1064,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 cur = nxt;
             }
         }
-        arrive_and_fit(A, R, 1, cap, sm_list, sm_scan, sm_count, sm_red, 8);
+        arrive_and_fit(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8);
         if (threadIdx.x == 0) sm_next = 0;
         __syncthreads();
         if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
@@ -1008,7 +1110,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     cur = nxt;
                 }
             }
-            arrive_and_fit(A, R, m, cap, sm_list, sm_scan, sm_count, sm_red, 10);
+            arrive_and_fit(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10);
             if (threadIdx.x == 0) sm_next = 0;
             __syncthreads();
             if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns();
@@ -1017,14 +1119,158 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // ------------------------------------------------------------------ P5a: stage survivors per chunk
     int warp_total = 0;
-    publish_params(A, R, 0, -1, 100);
+
+    // Block-wide pass over the full chunks that carry candidate flags (the common case for one- and two-stage
+    // segments).  The flagged slots of up to kCoopPass chunks are listed in shared memory in chunk order
+    // (chunk, slot, lane) and fetched two per thread in one wave, so the whole run costs a few memory round
+    // trips instead of one per chunk and warp.  Listing and fetching need no threshold: they are issued before
+    // the CTA waits for the fits of its segments, and overlap that wait.  Once a segment's threshold is known
+    // its flags either proved valid (eta >= tau: survivors are taken from the fetched slots, a block scan over
+    // the per-slot counts giving each its place in the chunk's staging region, and the chunk is marked in
+    // sm_done) or not (the fetched slots are dropped).  The warp loop below takes every chunk not marked
+    // (ragged chunks, invalid flags, side regions).
+    bool published = false;
+    int coop_n = 0;                       // leading chunks of the run this pass covers
+    if (vec_ok && sm_any_tau) {
+        coop_n = min(c1 - c0, kCoopChunks);
+        for (int i = threadIdx.x; i < kCoopChunks / 32; i += kThreads) sm_done[i] = 0u;
+        __syncthreads();
+        // threshold of cached segment i once its last stage is fitted; true if its flags are valid
+        auto seg_thr = [&](int i, float& thr) -> bool {
+            long long spins = 0;
+            while (R.ok[i] != 100) {                       // published by a thread of this CTA
+                if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+                __nanosleep(20);
+            }
+            __threadfence_block();
+            thr = R.thr[i];
+            return thr >= sm_tau[i];
+        };
+        for (int base = 0; base < coop_n; base += kCoopPass) {
+            // two threads per chunk: this one lists slots jj and jj + 1 of all 32 lanes
+            const int cl = threadIdx.x >> 1;
+            const int k = base + cl;
+            const int c = c0 + k;
+            const int jj = (threadIdx.x & 1) * 2;
+            int seg_i = -1;                       // cache index of the chunk's segment if the chunk carries flags
+            if (k < coop_n) {
+                const int seg = __ldg(A.chunk_seg + c);
+                const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
+                const int i = seg - R.seg_lo;
+                if ((lo & (kChunk - 1)) == 0 && hi == lo + kChunk && i < kSegCache && sm_tau[i] > 0.0f) seg_i = i;
+            }
+            unsigned long long bits = 0ull;       // bit 32 (j - jj) + lane: slot j of that lane is flagged
+            if (seg_i >= 0) {
+                const uint4* fp = reinterpret_cast<const uint4*>(A.cand + (size_t)c * 32);
+                const uint4 fa = __ldcg(fp), fb = __ldcg(fp + 1);
+                // bit j of each of a word's four bytes, gathered into four adjacent bits
+                auto pick = [](unsigned w, int j) -> unsigned { return ((((w >> j) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu; };
+                auto lanes = [&](int j) -> unsigned {
+                    return pick(fa.x, j) | (pick(fa.y, j) << 4) | (pick(fa.z, j) << 8) | (pick(fa.w, j) << 12) |
+                           (pick(fb.x, j) << 16) | (pick(fb.y, j) << 20) | (pick(fb.z, j) << 24) | (pick(fb.w, j) << 28);
+                };
+                bits = (unsigned long long)lanes(jj) | ((unsigned long long)lanes(jj + 1) << 32);
+            }
+            int total = 0;
+            int off = block_exscan(__popcll(bits), sm_warp, total);
+            const bool listed = total <= kCoopItems;       // same for every thread; otherwise the warp loop takes these chunks
+            if (listed) {
+                unsigned long long b = bits;
+                while (b) {
+                    const int q = __ffsll((long long)b) - 1;
+                    b &= b - 1ull;
+                    sm_items[off++] = (unsigned short)((cl << 7) | ((jj + (q >> 5)) << 5) | (q & 31));
+                }
+                if ((threadIdx.x & 1) == 0) { sm_cseg[cl] = seg_i; sm_ccnt[cl] = 0; }
+            }
+            __syncthreads();
+            if (!listed) continue;
+            int carry = 0;                    // survivors of the rounds before this one
+            for (int r0 = 0; r0 < total; r0 += 2 * kThreads) {
+                F8 x[2];
+                int e[2], icl[2];
+                unsigned m8[2];
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int r = r0 + 2 * (int)threadIdx.x + u;
+                    e[u] = -1; icl[u] = 0; m8[u] = 0u;
+                    if (r < total) {
+                        const int it = sm_items[r];
+                        icl[u] = it >> 7;
+                        e[u] = __ldg(A.chunk_start + c0 + base + icl[u]) + ((it >> 5) & 3) * 256 + (it & 31) * kComp;
+                        x[u] = ld8_evict_last(A.residual + e[u]);
+                    }
+                }
+                // the fits are waited for only now, with the slot loads in flight
+                if (!published) { publish_params(A, R, 0, -1, 100); published = true; }
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    float t;
+                    if (e[u] >= 0 && seg_thr(sm_cseg[icl[u]], t)) {
+                        #pragma unroll
+                        for (int cc = 0; cc < kComp; ++cc)
+                            if (fabsf(x[u].v[cc]) >= t) m8[u] |= 1u << cc;
+                    }
+                }
+                const int n0 = __popc(m8[0]), n1 = __popc(m8[1]);
+                int round_total = 0;
+                const int ex = carry + block_exscan(n0 + n1, sm_warp, round_total);
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int r = r0 + 2 * (int)threadIdx.x + u;
+                    // the first listed slot of a chunk records how many survivors precede the chunk
+                    if (e[u] >= 0 && (r == 0 || (sm_items[r - 1] >> 7) != icl[u])) sm_cbase[icl[u]] = ex + (u ? n0 : 0);
+                }
+                __syncthreads();
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if (m8[u]) {
+                        int pos = (e[u] & ~(kChunk - 1)) + ex + (u ? n0 : 0) - sm_cbase[icl[u]];
+                        #pragma unroll
+                        for (int cc = 0; cc < kComp; ++cc) {
+                            if (m8[u] & (1u << cc)) {
+                                A.stage_idx[pos] = e[u] + cc;
+                                A.stage_val[pos] = x[u].v[cc];
+                                A.residual[e[u] + cc] = 0.0f;
+                                ++pos;
+                            }
+                        }
+                        atomicAdd(&sm_ccnt[icl[u]], u ? n1 : n0);
+                    }
+                }
+                carry += round_total;
+            }
+            if (!published) { publish_params(A, R, 0, -1, 100); published = true; }
+            __syncthreads();
+            if (threadIdx.x < kCoopPass) {            // whole warps: one thread per chunk of the pass
+                const int k2 = base + (int)threadIdx.x;
+                int key = -1, cnt = 0;
+                float t;
+                if (k2 < coop_n && sm_cseg[threadIdx.x] >= 0 && seg_thr(sm_cseg[threadIdx.x], t)) {
+                    atomicOr(&sm_done[k2 >> 5], 1u << (k2 & 31));
+                    cnt = sm_ccnt[threadIdx.x];
+                    A.chunk_cnt[c0 + k2] = cnt;
+                    if (cnt) key = __ldg(A.chunk_seg + c0 + k2);
+                }
+                // one counter update per segment and warp
+                const unsigned peers = __match_any_sync(kFull, key);
+                const int sum = __reduce_add_sync(peers, cnt);
+                if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&A.seg[key].k_acc, sum);
+            }
+            if (threadIdx.x == 0) sm_coop_total += carry;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) warp_total += sm_coop_total;
+    }
+    if (!published) publish_params(A, R, 0, -1, 100);
+
     {
         SegView sv;
         bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
-        Desc cur = fetch_desc(A, queue.next(!p1_desc), true, true);
+        Desc cur = fetch_desc(A, queue.next_undone(!p1_desc, sm_done, coop_n), true, true);
         while (cur.c >= 0) {
-            const Desc nxt = fetch_desc(A, queue.next(!p1_desc), true, true);
+            const Desc nxt = fetch_desc(A, queue.next_undone(!p1_desc, sm_done, coop_n), true, true);
             if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
                 seg_count = 0;
@@ -1117,8 +1363,56 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     }
     __syncthreads();
     cta_count = sm_base;
-    grid_barrier(A.ctl, A.G, sm_gen + 1u);
+    grid_barrier(A.ctl, A.barrier_target);
     if (stamper) A.ctl->t_ns[4] = global_ns();
+
+    // Per-segment bookkeeping (counts, adaptation, next candidate threshold) is spread over the grid, one
+    // segment per thread, segment s going to thread (s / G) % kThreads of CTA s % G.  What it reads is
+    // loaded here, ahead of the placement, so that the two chains of memory round trips overlap.
+    struct SegEnd { int k_hat, M_eff, status, calls, M; long long k_sum; float thr, spec_thr; };
+    auto seg_end_load = [&](int s) -> SegEnd {
+        const SegDev* sg = &A.seg[s];
+        return SegEnd{ld_cg(&sg->k_acc), ld_cg(&sg->M_eff), ld_cg(&sg->status), sg->calls, sg->M, sg->k_sum,
+                      ld_cg(&sg->thr_ge), sg->spec_thr};
+    };
+    // per-segment counts, last stage count, adaptation (Algorithm 1, Adapt_Stages)
+    auto seg_end_store = [&](int s, const SegEnd& v, bool timed_out) {
+        SegDev* sg = &A.seg[s];
+        sg->k_acc = 0;
+        A.out_k[s] = v.k_hat;
+        sg->k_stage[v.M_eff - 1] = v.k_hat;
+        int status = v.status | (timed_out ? kStTimeout : 0);
+        if (A.max_stages > 0) {
+            const int calls = v.calls + 1;
+            long long k_sum = v.k_sum + v.k_hat;
+            if (calls % A.Q == 0) {
+                const double k_avg = (double)k_sum / (double)A.Q;
+                const double k_target = A.delta * (double)A.seg_n[s];
+                int M = v.M;
+                if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
+                if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
+                if (M < 1) M = 1;
+                if (M > A.max_stages) M = A.max_stages;
+                sg->M = M;
+                k_sum = 0;
+            }
+            sg->calls = calls;
+            sg->k_sum = k_sum;
+        }
+        // candidate threshold for the next call's first sweep (and whether this call's guess held);
+        // v.M still is the state this call's stage count came from
+        {
+            int m_call = A.max_stages > 0 ? (v.M < 1 ? 1 : (v.M > A.max_stages ? A.max_stages : v.M)) : -A.max_stages;
+            if (m_call > cap) m_call = cap;
+            const float tau_used = (A.spec_enable && m_call <= 2 && v.spec_thr > 0.0f) ? v.spec_thr : -1.0f;
+            if (tau_used > 0.0f) status |= (v.thr >= tau_used ? kStFlagsUsed : kStFlagsMissed);
+        }
+        if (status != v.status) sg->status = status;
+        sg->spec_thr = (v.thr > 0.0f && v.thr < 3.0e38f) ? kSpecRatio * v.thr : -1.0f;
+    };
+    const int s_first = cta + A.G * (int)threadIdx.x;
+    SegEnd first{};
+    if (s_first < A.S) first = seg_end_load(s_first);
 
     // ------------------------------------------------------------------ P5b: final positions
     {
@@ -1174,44 +1468,16 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             __syncthreads();
         }
     }
-    // per-segment counts, last stage count, adaptation (Algorithm 1, Adapt_Stages)
-    for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads) {
-        SegDev* sg = &A.seg[s];
-        const int k_hat = ld_cg(&sg->k_acc);
-        sg->k_acc = 0;
-        A.out_k[s] = k_hat;
-        sg->k_stage[ld_cg(&sg->M_eff) - 1] = k_hat;
-        if (ld_volatile(&A.ctl->timeout)) sg->status = ld_cg(&sg->status) | kStTimeout;
-        if (A.max_stages > 0) {
-            const int calls = sg->calls + 1;
-            long long k_sum = sg->k_sum + k_hat;
-            if (calls % A.Q == 0) {
-                const double k_avg = (double)k_sum / (double)A.Q;
-                const double k_target = A.delta * (double)A.seg_n[s];
-                int M = sg->M;
-                if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
-                if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
-                if (M < 1) M = 1;
-                if (M > A.max_stages) M = A.max_stages;
-                sg->M = M;
-                k_sum = 0;
-            }
-            sg->calls = calls;
-            sg->k_sum = k_sum;
-        }
-        // candidate threshold for the next call's first sweep (and whether this call's guess held)
-        const float thr = ld_cg(&sg->thr_ge);
-        {
-            const float tau_used = (A.spec_enable && seg_stages(A, s, cap) <= 2 && sg->spec_thr > 0.0f) ? sg->spec_thr : -1.0f;
-            if (tau_used > 0.0f) sg->status = ld_cg(&sg->status) | (thr >= tau_used ? kStFlagsUsed : kStFlagsMissed);
-        }
-        sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
+    {
+        const bool timed_out = ld_volatile(&A.ctl->timeout) != 0;
+        if (s_first < A.S) seg_end_store(s_first, first, timed_out);
+        for (int s = s_first + A.G * kThreads; s < A.S; s += A.G * kThreads) seg_end_store(s, seg_end_load(s), timed_out);
     }
 
     if (stamper) A.ctl->t_ns[5] = global_ns();
 }
 
-// Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared.  The ready
+// Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared.  The published
 // words keep their call tags.
 __global__ void sidco_reset_state_kernel(SegDev* seg, int S) {
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
