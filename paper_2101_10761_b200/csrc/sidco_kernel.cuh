@@ -1348,7 +1348,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
     }
     if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
-    __threadfence();
+    // (what this CTA stored for the placement becomes visible to the grid through the barrier below:
+    // CTA barrier, then thread 0's fence and arrival)
     __syncthreads();
     if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns();
     if (stamper) A.ctl->t_ns[12] = global_ns();
