@@ -271,6 +271,28 @@ __device__ __forceinline__ int block_exscan(int x, int* sm, int& total) {
     return warp_incl - sm[warp] + incl - x;
 }
 
+// The same for one half of the CTA (warps 16 h .. 16 h + 15), the two halves working independently: they
+// meet at named barrier 1 + h.  Result valid in the half's first thread.
+__device__ __forceinline__ Sums half_tree(double a, double b, int n, double (*sm)[3], int h) {
+    Sums w = warp_tree(a, b, n);
+    const int lane = threadIdx.x & 31, wh = (threadIdx.x >> 5) & 15;
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + h), "r"(kThreads / 2) : "memory");      // previous use of sm is over
+    if (lane == 0) { sm[wh][0] = w.a; sm[wh][1] = w.b; sm[wh][2] = (double)w.n; }
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + h), "r"(kThreads / 2) : "memory");
+    Sums r{0.0, 0.0, 0};
+    if (wh == 0) {
+        double x = lane < 16 ? sm[lane][0] : 0.0, y = lane < 16 ? sm[lane][1] : 0.0, z = lane < 16 ? sm[lane][2] : 0.0;
+        #pragma unroll
+        for (int o = 8; o > 0; o >>= 1) {
+            x += __shfl_down_sync(kFull, x, o);
+            y += __shfl_down_sync(kFull, y, o);
+            z += __shfl_down_sync(kFull, z, o);
+        }
+        r.a = x; r.b = y; r.n = (int)z;
+    }
+    return r;
+}
+
 // ----------------------------------------------------------------------------
 // closed-form fits (one thread)
 // ----------------------------------------------------------------------------
@@ -757,17 +779,20 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         }
         __syncthreads();
         const int n_small = sm_count[0], n_large = sm_count[1];
-        // large segments first (other runs wait for them): the whole CTA, threads stride over the chunk
-        // partials, fixed block tree
-        for (int k = 0; k < n_large; ++k) {
-            const int i2 = sm_large[k];
-            int q0, q1, runs;
-            R.get(A, i2, q0, q1, runs);
-            SegDev* sg = &A.seg[R.seg_lo + i2];
-            const int M_state = (stage == 0 && threadIdx.x == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
-            const Sums t = strided_partials(A, q0 + (int)threadIdx.x, q1, kThreads);
-            Sums r = block_tree(t.a, t.b, t.n, sm_red);
-            if (threadIdx.x == 0) fit_and_cache(sg, i2, M_state, r);
+        // large segments first (other runs wait for them): half a CTA each, the two halves working on two
+        // segments at a time; threads stride over the chunk partials, fixed tree over the half
+        {
+            const int h = warp >> 4, th = threadIdx.x & (kThreads / 2 - 1);
+            for (int k = h; k < n_large; k += 2) {
+                const int i2 = sm_large[k];
+                int q0, q1, runs;
+                R.get(A, i2, q0, q1, runs);
+                SegDev* sg = &A.seg[R.seg_lo + i2];
+                const int M_state = (stage == 0 && th == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
+                const Sums t = strided_partials(A, q0 + th, q1, kThreads / 2);
+                Sums r = half_tree(t.a, t.b, t.n, sm_red + 16 * h, h);
+                if (th == 0) fit_and_cache(sg, i2, M_state, r);
+            }
         }
         // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
         for (int k = warp; k < n_small; k += kWarps) {
