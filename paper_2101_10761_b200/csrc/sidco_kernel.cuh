@@ -162,6 +162,14 @@ __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned l
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
+// Arrival counter update whose returned value, if it shows that every other run has arrived, also makes
+// their earlier (fenced) stores visible to this thread's later loads.
+__device__ __forceinline__ int atom_add_acquire(int* p, int v) {
+    int old;
+    asm volatile("atom.acquire.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -360,16 +368,56 @@ struct Fit {
     float thr;          // thr_ge(eta) if the stage is the segment's last, thr_gt(eta) otherwise
     int stages;         // stages fitted so far
     bool last;
+    // for the record kept in SegDev (see record_stage)
+    int M_eff, status, n_e;
+    bool empty;         // segment without elements
 };
 
+__device__ __forceinline__ Fit warp_broadcast(const Fit& f) {
+    Fit g;
+    g.eta = __shfl_sync(kFull, f.eta, 0);
+    g.thr = __shfl_sync(kFull, f.thr, 0);
+    g.stages = __shfl_sync(kFull, f.stages, 0);
+    g.last = __shfl_sync(kFull, (int)f.last, 0) != 0;
+    g.M_eff = __shfl_sync(kFull, f.M_eff, 0);
+    g.status = __shfl_sync(kFull, f.status, 0);
+    g.n_e = __shfl_sync(kFull, f.n_e, 0);
+    g.empty = __shfl_sync(kFull, (int)f.empty, 0) != 0;
+    return g;
+}
+
+// The fields of SegDev that describe a fitted stage, other than the published word: written after it, by
+// the threads first, first + step, ... of a group that all hold `f` (a warp, or one thread with step 1).
+// `stage` = 0 writes the whole record of the call's first stage and clears the later stages' entries.
+// These stores are ordered before any later fit of the segment by the fence and arrival atomic of this
+// CTA's next phase, and before the final placement by the grid barrier.
+__device__ __forceinline__ void record_stage(SegDev* sg, int stage, const Fit& f, int first, int step) {
+    if (stage == 0) {
+        for (int q = first; q < 20; q += step) {
+            if (q < 8) sg->eta[q] = (q == 0 || (f.empty && q < f.M_eff)) ? f.eta : 0.0;
+            else if (q < 16) sg->k_stage[q - 8] = 0;
+            else if (q == 16) sg->M_eff = f.M_eff;
+            else if (q == 17) sg->status = f.status;
+            else if (q == 18) sg->thr_gt = __double2float_rd(f.eta);
+            else sg->thr_ge = __double2float_ru(f.eta);
+        }
+    } else {
+        for (int q = first; q < 5; q += step) {
+            if (q == 0) sg->k_stage[stage - 1] = f.n_e;
+            else if (q == 1) sg->eta[stage] = f.eta;
+            else if (q == 2) sg->thr_gt = __double2float_rd(f.eta);
+            else if (q == 3) sg->thr_ge = __double2float_ru(f.eta);
+            else if (f.status) sg->status = ld_cg(&sg->status) | f.status;   // written by the previous stage's fit
+        }
+    }
+}
+
 // Publish a fitted stage: the tagged threshold word goes out first; everything else about the stage is
-// stored by the caller afterwards.  If another stage follows, its sweep shifts by eta, which is therefore
+// stored afterwards (record_stage).  If another stage follows, its sweep shifts by eta, which is therefore
 // stored before the word and released with it.  The word of a last stage carries all that its readers need
 // (they go on to read only their own run's data), so it is a plain strong store with no fence to wait for.
-// The caller's later stores are ordered before any later fit of the segment by the fence and arrival atomic
-// of this CTA's next phase, and before the final placement by the grid barrier.
 __device__ inline Fit publish_stage(const Args& A, SegDev* sg, int stages, bool last, double eta) {
-    Fit f{eta, last ? __double2float_ru(eta) : __double2float_rd(eta), stages, last};
+    Fit f{eta, last ? __double2float_ru(eta) : __double2float_rd(eta), stages, last, 0, 0, 0, false};
     const unsigned long long word = ((unsigned long long)__float_as_uint(f.thr) << 32) |
                                     (unsigned long long)((unsigned)A.call_id * 16u + (unsigned)stages);
     if (last) {
@@ -427,14 +475,10 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
         }
     }
     // an empty segment takes part in no later phase: all its stages count as fitted here
-    const Fit f = publish_stage(A, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
-    sg->M_eff = M_eff;
-    sg->status = status;
-    sg->eta[0] = eta;
-    for (int m = 1; m < kMaxStages; ++m) sg->eta[m] = (n == 0 && m < M_eff) ? eta : 0.0;
-    for (int m = 0; m < kMaxStages; ++m) sg->k_stage[m] = 0;
-    sg->thr_gt = __double2float_rd(eta);
-    sg->thr_ge = __double2float_ru(eta);
+    Fit f = publish_stage(A, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
+    f.M_eff = M_eff;
+    f.status = status;
+    f.empty = n == 0;
     return f;
 }
 
@@ -452,12 +496,10 @@ __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, d
         else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, T.ln[slot], T.ln_inv[slot], status);
         eta = prev + inc;
     }
-    const Fit f = publish_stage(A, sg, m + 1, m + 1 == M_eff, eta);
-    sg->k_stage[m - 1] = n_e;
-    if (status) sg->status = ld_cg(&sg->status) | status;     // written by the previous stage's fit (maybe another SM)
-    sg->eta[m] = eta;
-    sg->thr_gt = __double2float_rd(eta);
-    sg->thr_ge = __double2float_ru(eta);
+    Fit f = publish_stage(A, sg, m + 1, m + 1 == M_eff, eta);
+    f.M_eff = M_eff;
+    f.status = status;
+    f.n_e = n_e;
     return f;
 }
 
@@ -736,24 +778,28 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
     }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // one thread: fit segment i2 of the run from its sums, publish, and fill the CTA's own cache entry
+    // one warp: its first lane fits segment i2 of the run from its sums (M_state and r are that lane's),
+    // publishes, and fills the CTA's own cache entry; all lanes then write the stage's record
     auto fit_and_cache = [&](SegDev* sg, int i2, int M_state, const Sums& r) {
         const bool cached = i2 < kSegCache;
-        Fit f;
-        if (stage == 0) {
-            f = fit_stage1(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
-        } else {
-            // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
-            const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
-            const double prev = cached ? R.eta_prev[i2] : ld_cg(&sg->eta[stage - 1]);
-            f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T);
+        Fit f{};
+        if (lane == 0) {
+            if (stage == 0) {
+                f = fit_stage1(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
+            } else {
+                // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
+                const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
+                const double prev = cached ? R.eta_prev[i2] : ld_cg(&sg->eta[stage - 1]);
+                f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T);
+            }
+            if (cached) {
+                R.thr[i2] = f.thr;
+                R.eta_prev[i2] = f.eta;
+                __threadfence_block();
+                R.ok[i2] = f.last ? 100 : f.stages;        // tag of the phase that uses these values next
+            }
         }
-        if (cached) {
-            R.thr[i2] = f.thr;
-            R.eta_prev[i2] = f.eta;
-            __threadfence_block();
-            R.ok[i2] = f.last ? 100 : f.stages;        // tag of the phase that uses these values next
-        }
+        record_stage(sg, stage, warp_broadcast(f), lane, 32);
     };
     for (int base = 0; base < R.n_seg; base += kThreads) {
         const int i = base + (int)threadIdx.x;
@@ -765,11 +811,8 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                 const bool takes_part = stage == 0 || (i < kSegCache ? R.m_eff[i] : seg_stages(A, R.seg_lo + i, cap)) > stage;
                 bool complete = takes_part && runs == 1;
                 if (takes_part && runs > 1) {
-                    complete = atomicAdd(&sg->arrived, 1) == runs - 1;
-                    if (complete) {
-                        sg->arrived = 0;
-                        __threadfence();     // acquire side: the other runs' partials are read next
-                    }
+                    complete = atom_add_acquire(&sg->arrived, 1) == runs - 1;
+                    if (complete) sg->arrived = 0;     // (the other runs' partials, read next, came with the acquire)
                 }
                 if (complete) {
                     if (q1 - q0 <= kSmallSeg) sm_small[atomicAdd(&sm_count[0], 1)] = i;
@@ -791,7 +834,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                 const int M_state = (stage == 0 && th == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
                 const Sums t = strided_partials(A, q0 + th, q1, kThreads / 2);
                 Sums r = half_tree(t.a, t.b, t.n, sm_red + 16 * h, h);
-                if (th == 0) fit_and_cache(sg, i2, M_state, r);
+                if (th < 32) fit_and_cache(sg, i2, M_state, r);
             }
         }
         // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
@@ -805,7 +848,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
             const int M_state = (stage == 0 && lane == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
             const Sums t = strided_partials(A, q0 + lane, q1, 32);
             Sums r = warp_tree(t.a, t.b, t.n);
-            if (lane == 0) fit_and_cache(sg, i2, M_state, r);
+            fit_and_cache(sg, i2, M_state, r);
         }
         __syncthreads();
         if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
@@ -885,7 +928,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
-        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
+        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s])
+            record_stage(&A.seg[s], 0, fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T), 0, 1);
     __syncthreads();
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
