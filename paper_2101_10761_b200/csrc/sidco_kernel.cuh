@@ -640,6 +640,13 @@ struct ChunkQueue {
             if (k >= n_done || !((done[k >> 5] >> (k & 31)) & 1u)) return c;
         }
     }
+    // The next entry of a list of n chunk numbers (relative to c0) instead.
+    __device__ __forceinline__ int next_listed(const int* list, int n) const {
+        int k = 0;
+        if ((threadIdx.x & 31) == 0) k = atomicAdd(sm_next, 1);
+        k = __shfl_sync(kFull, k, 0);
+        return k < n ? c0 + list[k] : -1;
+    }
 };
 
 // Chunk descriptor, fetched one chunk ahead so that its loads overlap the current chunk's work.
@@ -1332,14 +1339,32 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (threadIdx.x == 0) warp_total += sm_coop_total;
     }
     if (!published) publish_params(A, R, 0, -1, 100);
+    // The chunks left for the warp loop, if the pass above covered the whole run: listed, so that the warps
+    // do not take turns at the queue for every chunk already done (few are left).
+    int n_rest = -1;                      // < 0: no list, the loop goes through the queue and skips the chunks done
+    if (coop_n == c1 - c0 && coop_n > 0) {
+        for (int k = threadIdx.x; k < coop_n; k += kThreads)
+            if (!((sm_done[k >> 5] >> (k & 31)) & 1u)) {
+                const int p = atomicAdd(&sm_count[0], 1);
+                if (p < kThreads) sm_list[p] = k;
+            }
+        __syncthreads();
+        n_rest = sm_count[0];
+        __syncthreads();
+        if (threadIdx.x == 0) sm_count[0] = 0;
+        if (n_rest > kThreads) n_rest = -1;          // more than the list holds
+    }
+    auto next_chunk = [&]() -> int {
+        return n_rest >= 0 ? queue.next_listed(sm_list, n_rest) : queue.next_undone(!p1_desc, sm_done, coop_n);
+    };
 
     {
         SegView sv;
         bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
-        Desc cur = fetch_desc(A, queue.next_undone(!p1_desc, sm_done, coop_n), true, true);
+        Desc cur = fetch_desc(A, next_chunk(), true, true);
         while (cur.c >= 0) {
-            const Desc nxt = fetch_desc(A, queue.next_undone(!p1_desc, sm_done, coop_n), true, true);
+            const Desc nxt = fetch_desc(A, next_chunk(), true, true);
             if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
                 seg_count = 0;
