@@ -1211,8 +1211,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         coop_n = min(c1 - c0, kCoopChunks);
         for (int i = threadIdx.x; i < kCoopChunks / 32; i += kThreads) sm_done[i] = 0u;
         __syncthreads();
-        // threshold of cached segment i once its last stage is fitted; true if its flags are valid
-        auto seg_thr = [&](int i, float& thr) -> bool {
+        // Threshold of a chunk's segment once its last stage is fitted; true if the chunk's listed slots
+        // hold all its survivors.  `tag` is the segment's cache index, plus kAllSlots if all of the chunk's
+        // slots were listed (then no flags are involved).
+        constexpr int kAllSlots = 1 << 16;
+        auto seg_thr = [&](int tag, float& thr) -> bool {
+            const int i = tag & (kAllSlots - 1);
             long long spins = 0;
             while (R.ok[i] != 100) {                       // published by a thread of this CTA
                 if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
@@ -1220,7 +1224,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             }
             __threadfence_block();
             thr = R.thr[i];
-            return thr >= sm_tau[i];
+            return (tag & kAllSlots) || thr >= sm_tau[i];
         };
         for (int base = 0; base < coop_n; base += kCoopPass) {
             // two threads per chunk: this one lists slots jj and jj + 1 of all 32 lanes
@@ -1228,17 +1232,41 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             const int k = base + cl;
             const int c = c0 + k;
             const int jj = (threadIdx.x & 1) * 2;
-            int seg_i = -1;                       // cache index of the chunk's segment if the chunk carries flags
+            // Chunks taken here: full chunks that carry flags, and ragged chunks made of whole slots, all of
+            // which are listed (a run has few of them).  Both need acc as the source of the final selection,
+            // i.e. a segment with at most two stages.
+            int seg_i = -1;                       // see seg_thr
+            unsigned long long bits = 0ull;       // bit 32 (j - jj) + lane: slot j of that lane is listed
+            uint4 fa = make_uint4(0u, 0u, 0u, 0u), fb = fa;      // the chunk's 32 flag bytes
             if (k < coop_n) {
+                // (loaded whether or not the chunk turns out to carry flags, so that this costs one round
+                // trip, not two)
+                const uint4* fp = reinterpret_cast<const uint4*>(A.cand + (size_t)c * 32);
+                fa = __ldcg(fp);
+                fb = __ldcg(fp + 1);
                 const int seg = __ldg(A.chunk_seg + c);
                 const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
                 const int i = seg - R.seg_lo;
-                if ((lo & (kChunk - 1)) == 0 && hi == lo + kChunk && i < kSegCache && sm_tau[i] > 0.0f) seg_i = i;
+                if (i < kSegCache && sm_meff[i] <= 2) {
+                    const int wb = lo & ~(kChunk - 1);
+                    if (lo == wb && hi == wb + kChunk) {
+                        if (sm_tau[i] > 0.0f) seg_i = i;
+                    } else if (((lo | hi) & (kComp - 1)) == 0) {
+                        seg_i = i | kAllSlots;
+                        #pragma unroll
+                        for (int dj = 0; dj < 2; ++dj) {
+                            const int row = wb + (jj + dj) * 256;                     // slot row: 32 lanes x 8 elements
+                            const int a = max(lo, row), b = min(hi, row + 256);
+                            if (b > a) {
+                                const int l0 = (a - row) / kComp, nl = (b - a) / kComp;  // lanes l0 .. l0 + nl - 1
+                                const unsigned m = (nl >= 32 ? kFull : ((1u << nl) - 1u)) << l0;
+                                bits |= (unsigned long long)m << (32 * dj);
+                            }
+                        }
+                    }
+                }
             }
-            unsigned long long bits = 0ull;       // bit 32 (j - jj) + lane: slot j of that lane is flagged
-            if (seg_i >= 0) {
-                const uint4* fp = reinterpret_cast<const uint4*>(A.cand + (size_t)c * 32);
-                const uint4 fa = __ldcg(fp), fb = __ldcg(fp + 1);
+            if (seg_i >= 0 && !(seg_i & kAllSlots)) {
                 // bit j of each of a word's four bytes, gathered into four adjacent bits
                 auto pick = [](unsigned w, int j) -> unsigned { return ((((w >> j) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu; };
                 auto lanes = [&](int j) -> unsigned {
@@ -1251,11 +1279,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             int off = block_exscan(__popcll(bits), sm_warp, total);
             const bool listed = total <= kCoopItems;       // same for every thread; otherwise the warp loop takes these chunks
             if (listed) {
-                unsigned long long b = bits;
-                while (b) {
-                    const int q = __ffsll((long long)b) - 1;
-                    b &= b - 1ull;
-                    sm_items[off++] = (unsigned short)((cl << 7) | ((jj + (q >> 5)) << 5) | (q & 31));
+                #pragma unroll
+                for (int dj = 0; dj < 2; ++dj) {
+                    unsigned m = (unsigned)(bits >> (32 * dj));
+                    const int head = (cl << 7) | ((jj + dj) << 5);
+                    if (seg_i >= 0 && (seg_i & kAllSlots)) {        // a ragged chunk's row: one run of lanes
+                        const int l0 = __ffs(m) - 1, nl = __popc(m);
+                        for (int q = 0; q < nl; ++q) sm_items[off + q] = (unsigned short)(head | (l0 + q));
+                        off += nl;
+                    } else {
+                        while (m) {
+                            const int q = __ffs(m) - 1;
+                            m &= m - 1u;
+                            sm_items[off++] = (unsigned short)(head | q);
+                        }
+                    }
                 }
                 if ((threadIdx.x & 1) == 0) { sm_cseg[cl] = seg_i; sm_ccnt[cl] = 0; }
             }
@@ -1264,16 +1302,17 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             int carry = 0;                    // survivors of the rounds before this one
             for (int r0 = 0; r0 < total; r0 += 2 * kThreads) {
                 F8 x[2];
-                int e[2], icl[2];
+                int e[2], icl[2], clo[2];
                 unsigned m8[2];
                 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int r = r0 + 2 * (int)threadIdx.x + u;
-                    e[u] = -1; icl[u] = 0; m8[u] = 0u;
+                    e[u] = -1; icl[u] = 0; clo[u] = 0; m8[u] = 0u;
                     if (r < total) {
                         const int it = sm_items[r];
                         icl[u] = it >> 7;
-                        e[u] = __ldg(A.chunk_start + c0 + base + icl[u]) + ((it >> 5) & 3) * 256 + (it & 31) * kComp;
+                        clo[u] = __ldg(A.chunk_start + c0 + base + icl[u]);       // staging region of the chunk starts here
+                        e[u] = (clo[u] & ~(kChunk - 1)) + ((it >> 5) & 3) * 256 + (it & 31) * kComp;
                         x[u] = ld8_evict_last(A.residual + e[u]);
                     }
                 }
@@ -1301,7 +1340,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     if (m8[u]) {
-                        int pos = (e[u] & ~(kChunk - 1)) + ex + (u ? n0 : 0) - sm_cbase[icl[u]];
+                        int pos = clo[u] + ex + (u ? n0 : 0) - sm_cbase[icl[u]];
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc) {
                             if (m8[u] & (1u << cc)) {
@@ -1326,7 +1365,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     atomicOr(&sm_done[k2 >> 5], 1u << (k2 & 31));
                     cnt = sm_ccnt[threadIdx.x];
                     A.chunk_cnt[c0 + k2] = cnt;
-                    if (cnt) key = __ldg(A.chunk_seg + c0 + k2);
+                    if (cnt) key = R.seg_lo + (sm_cseg[threadIdx.x] & (kAllSlots - 1));
                 }
                 // one counter update per segment and warp
                 const unsigned peers = __match_any_sync(kFull, key);
