@@ -49,7 +49,8 @@ constexpr int kChunk = 1024;                      // window: elements per full c
 constexpr int kComp = 8;                          // elements per slot: one 32-byte access per lane
 constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4)
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
-constexpr int kSegCache = 512;                    // segments of a CTA run whose table entries sit in shared memory
+constexpr int kSegCache = 256;                    // segments of a CTA run whose table entries sit in shared memory
+constexpr int kOutCache = 1024;                   // survivors of a run kept in shared memory for the final placement
 constexpr int kCoopChunks = 4096;                 // chunks of a run the block-wide flagged-slot pass can cover
 constexpr int kCoopPass = kThreads / 2;           // chunks per pass of it (two threads per chunk)
 constexpr int kCoopItems = 4096;                  // flagged slots one pass can list
@@ -883,6 +884,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ double sm_ln[kMaxStages + 1], sm_ln_inv[kMaxStages + 1];
     __shared__ double sm_eta[kSegCache];
     __shared__ int sm_ok[kSegCache];
+    __shared__ int sm_oidx[kOutCache];
+    __shared__ float sm_oval[kOutCache];
     __shared__ unsigned short sm_items[kCoopItems];
     __shared__ int sm_cseg[kCoopPass], sm_cbase[kCoopPass], sm_ccnt[kCoopPass];
     __shared__ unsigned sm_done[kCoopChunks / 32];
@@ -1205,8 +1208,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     // the per-slot counts giving each its place in the chunk's staging region, and the chunk is marked in
     // sm_done) or not (the fetched slots are dropped).  The warp loop below takes every chunk not marked
     // (ragged chunks, invalid flags, side regions).
+    // Survivors found by this pass are also kept in shared memory at their rank within the run (the passes
+    // and their scans go through the run in order).  If the pass ends up covering every chunk of the run and
+    // the survivors fit, the final placement copies them from there instead of reading the staging regions.
     bool published = false;
     int coop_n = 0;                       // leading chunks of the run this pass covers
+    int before_pass = 0;                  // survivors found by the passes before the current one
     if (vec_ok && sm_any_tau) {
         coop_n = min(c1 - c0, kCoopChunks);
         for (int i = threadIdx.x; i < kCoopChunks / 32; i += kThreads) sm_done[i] = 0u;
@@ -1341,13 +1348,16 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 for (int u = 0; u < 2; ++u) {
                     if (m8[u]) {
                         int pos = clo[u] + ex + (u ? n0 : 0) - sm_cbase[icl[u]];
+                        int rank = before_pass + ex + (u ? n0 : 0);
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc) {
                             if (m8[u] & (1u << cc)) {
                                 A.stage_idx[pos] = e[u] + cc;
                                 A.stage_val[pos] = x[u].v[cc];
                                 A.residual[e[u] + cc] = 0.0f;
+                                if (rank < kOutCache) { sm_oidx[rank] = e[u] + cc; sm_oval[rank] = x[u].v[cc]; }
                                 ++pos;
+                                ++rank;
                             }
                         }
                         atomicAdd(&sm_ccnt[icl[u]], u ? n1 : n0);
@@ -1373,6 +1383,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                 if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&A.seg[key].k_acc, sum);
             }
             if (threadIdx.x == 0) sm_coop_total += carry;
+            before_pass += carry;
             __syncthreads();
         }
         if (threadIdx.x == 0) warp_total += sm_coop_total;
@@ -1393,6 +1404,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (threadIdx.x == 0) sm_count[0] = 0;
         if (n_rest > kThreads) n_rest = -1;          // more than the list holds
     }
+    const bool place_from_smem = n_rest == 0 && before_pass <= kOutCache;
     auto next_chunk = [&]() -> int {
         return n_rest >= 0 ? queue.next_listed(sm_list, n_rest) : queue.next_undone(!p1_desc, sm_done, coop_n);
     };
@@ -1557,8 +1569,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         __syncthreads();
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
-        // chunk bases by a block-wide exclusive scan, kThreads chunks at a time
-        for (int pass = c0; pass < c1 && cta_count > 0; pass += kThreads) {
+        if (place_from_smem) {
+            // every survivor of the run sits in shared memory at its rank
+            for (int r = threadIdx.x; r < cta_count; r += kThreads) {
+                A.out_idx[run_base + r] = sm_oidx[r];
+                A.out_val[run_base + r] = sm_oval[r];
+            }
+        }
+        // otherwise: chunk bases by a block-wide exclusive scan, kThreads chunks at a time
+        for (int pass = c0; pass < c1 && cta_count > 0 && !place_from_smem; pass += kThreads) {
             const int c = pass + (int)threadIdx.x;
             const int cnt = c < c1 ? ld_cg(A.chunk_cnt + c) : 0;
             int incl = cnt;
