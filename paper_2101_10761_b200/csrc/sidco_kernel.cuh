@@ -1562,10 +1562,14 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
 
     // ------------------------------------------------------------------ P5b: final positions
     {
-        int below = 0;
-        for (int c = threadIdx.x; c < cta; c += kThreads) below += ld_cg(A.cta_total + c);
-        Sums r = block_tree(0.0, 0.0, below, sm_red);
-        if (threadIdx.x == 0) sm_base = r.n;
+        // survivors of the runs below this one: summed by one warp (a grid has a few hundred CTAs at most)
+        if (warp == 0) {
+            int below = 0;
+            for (int c = lane; c < cta; c += 32) below += ld_cg(A.cta_total + c);
+            #pragma unroll
+            for (int o = 16; o > 0; o >>= 1) below += __shfl_down_sync(kFull, below, o);
+            if (lane == 0) sm_base = below;
+        }
         __syncthreads();
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
