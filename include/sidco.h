@@ -52,6 +52,7 @@ extern "C" {
 #define SIDCO_E_WORKSPACE   (-8)   /* caller-provided workspace too small or misaligned */
 #define SIDCO_E_ALIAS       (-9)   /* grad and residual overlap */
 #define SIDCO_E_SIZE        (-10)  /* size beyond the limit of this entry point */
+#define SIDCO_E_CAPTURE     (-11)  /* the call would have to allocate or upload tables while `stream` is capturing */
 
 /* per-segment status bits */
 #define SIDCO_ST_NONFINITE  1   /* a magnitude was NaN/Inf: nothing is selected in the segment */
@@ -100,6 +101,11 @@ typedef struct sidco_seg_debug {
  *             segment s occupies positions [sum_{t<s} out_k[t], +out_k[s]) of out_idx/out_val.
  * stream      all device work is enqueued here; the call does not synchronise, except that the first
  *             call for a residual pointer (or for a new segment table) allocates and uploads tables.
+ *             Every later call enqueues one kernel whose arguments depend only on the arguments given
+ *             here (the call counter and the "residual is empty" mark live in the workspace and are
+ *             advanced by the kernel), so such calls may be recorded by stream capture and replayed as a
+ *             CUDA graph.  A call that would have to allocate or upload while `stream` is capturing
+ *             returns SIDCO_E_CAPTURE and enqueues nothing.
  *
  * 32-byte aligned grad and residual take the vectorised path; other alignments are handled with scalar
  * accesses.
@@ -137,8 +143,10 @@ int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_o
  *     larger inputs are rejected with SIDCO_E_SIZE before anything is enqueued;
  *   - there is one workspace per device, shared by every call: two calls that overlap on the GPU (for
  *     example on different streams) race on it and corrupt each other; serialise them;
- *   - the workspace keeps the contents the previous call left.  The counters that must start at zero are
- *     cleared on `stream` before each launch.  The stage-adaptation state lives in the workspace too and
+ *   - the workspace keeps the contents the previous call left.  The counters and records that must start
+ *     at zero are cleared on `stream` together with the table upload, i.e. on the first call for a
+ *     (residual pointer, segment table) pair; after that they carry on from call to call.  The
+ *     stage-adaptation state lives in the workspace too and
  *     belongs to the last (residual pointer, segment table) pair: calling with a different pair rebuilds
  *     the tables, resets M to 1 and synchronises `stream` once;
  *   - the first call on a device looks up the device address of the array (cudaGetSymbolAddress) and

@@ -83,9 +83,6 @@ struct Context {
     size_t ws_bytes = 0;
     bool ws_owned = false;
     bool tables_valid = false;
-    unsigned call_id = 0;                  // tags the per-segment published words
-    unsigned barrier_count = 0;            // grid-barrier arrivals recorded in the workspace's Control so far
-    bool residual_is_zero = false;         // set by a state reset: the next call does not read the residual
     Layout L{};
     // staging for sidco_compress_host
     float* h_grad = nullptr; float* h_res = nullptr;
@@ -235,7 +232,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
         if ((e = cudaMemcpy(seg_host.data(), (char*)c->ws + c->L.seg, sizeof(SegDev) * S, cudaMemcpyDeviceToHost)) !=
             cudaSuccess)
             return e;
-        for (auto& sg : seg_host) { sg.arrived = 0; sg.k_acc = 0; }
+        for (auto& sg : seg_host) { sg.arrived = 0; sg.k_acc = 0; sg.pub = 0; }    // (the call numbering restarts below)
     } else {
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
         for (auto& sg : seg_host) {
@@ -255,7 +252,6 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
-    c->barrier_count = 0;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
@@ -282,6 +278,10 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     const bool same = c->tables_valid && c->S == S &&
                       std::memcmp(c->offsets.data(), off, sizeof(int64_t) * (S + 1)) == 0;
     if (!same) {
+        // allocation, uploads and a stream synchronisation: not something a capturing stream can record
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return (int)e;
+        if (cap != cudaStreamCaptureStatusNone) return SIDCO_E_CAPTURE;
         if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
     }
     char* base = (char*)c->ws;
@@ -322,11 +322,6 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.C = c->T;
     a.S = c->S;
     a.G = c->G;
-    c->call_id = (c->call_id + 1u) & 0x0fffffffu;
-    a.call_id = (int)c->call_id;
-    a.barrier_target = c->barrier_count + (unsigned)c->G;
-    a.residual_is_zero = c->residual_is_zero ? 1 : 0;
-    c->residual_is_zero = false;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
     // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
     static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
@@ -338,7 +333,6 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
     e = launch_persistent(fn, c->G, kargs, stream);
     if (e != cudaSuccess) return (int)e;
-    c->barrier_count += (unsigned)c->G;
     g_launches.fetch_add(1);
     return 0;
 }
@@ -403,7 +397,6 @@ struct StaticContext {
     int32_t seg_chunk0[kStaticMaxSegs + 1], seg_n[kStaticMaxSegs + 1], seg_runs[kStaticMaxSegs + 1];
     int32_t cta_chunk0[kMaxGrid + 1];
     int4 cta_desc[kMaxGrid + 1];
-    unsigned call_id = 0;
     SegDev seg_init[kStaticMaxSegs + 1];
 };
 
@@ -511,16 +504,17 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = up(L.cta_desc, c.cta_desc, sizeof(int4) * (c.G + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
         // the uploads read the fixed host arrays: let them finish before those can change again
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
         c.key = residual;
         c.tables_valid = true;
     }
     const Layout& L = c.L;
-    // The array keeps whatever the last call left.  The barrier and completion counters must start at
-    // zero, so they are cleared on the stream before every launch; everything else is either rewritten
-    // before it is read or is state that is meant to persist.
-    if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
+    // The array keeps whatever the last call left.  What must start at zero (the control block: barrier
+    // arrivals, call number, time-out flag; and the segment records) was cleared with the upload above, when
+    // this residual and segment table were first seen; from then on it is state that is meant to persist,
+    // and everything else is rewritten before it is read.
     unsigned char* base = c.base;
     Args a{};
     a.grad = grad;
@@ -558,9 +552,6 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.C = c.T;
     a.S = c.S;
     a.G = c.G;
-    c.call_id = (c.call_id + 1u) & 0x0fffffffu;
-    a.call_id = (int)c.call_id;
-    a.barrier_target = (unsigned)c.G;      // the Control block, arrival count included, was cleared above
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
     a.spec_enable = 1;
     void* kargs[] = {(void*)&a};
@@ -669,9 +660,11 @@ int sidco_reset_state(const float* residual) {
     char* base = (char*)c->ws;
     if ((e = cudaMemcpy(base + c->L.seg, seg.data(), sizeof(SegDev) * (c->S + 1), cudaMemcpyHostToDevice)) != cudaSuccess)
         return (int)e;
-    if ((e = cudaMemset(base + c->L.ctl, 0, sizeof(Control))) != cudaSuccess) return (int)e;
-    c->barrier_count = 0;
-    c->residual_is_zero = true;
+    // call numbering and barrier count restart with the segment records; the residual counts as empty
+    Control ctl;
+    std::memset(&ctl, 0, sizeof(Control));
+    ctl.residual_is_zero = 1;
+    if ((e = cudaMemcpy(base + c->L.ctl, &ctl, sizeof(Control), cudaMemcpyHostToDevice)) != cudaSuccess) return (int)e;
     return 0;
 }
 
@@ -681,11 +674,10 @@ int sidco_reset_state_async(const float* residual, void* stream) {
     if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
     Context* c = it->second;
     sidco::sidco_reset_state_kernel<<<(c->S + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
-        (SegDev*)((char*)c->ws + c->L.seg), c->S);
+        (SegDev*)((char*)c->ws + c->L.seg), c->S, (Control*)((char*)c->ws + c->L.ctl));
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
-    c->residual_is_zero = true;
     return 0;
 }
 
@@ -834,6 +826,8 @@ const char* sidco_error_string(int code) {
         case SIDCO_E_WORKSPACE: return "workspace too small, misaligned, or set too late";
         case SIDCO_E_ALIAS: return "grad and residual overlap";
         case SIDCO_E_SIZE: return "size beyond the limit of this entry point";
+        case SIDCO_E_CAPTURE:
+            return "first call for this residual and segment table must be made before stream capture begins";
         default: break;
     }
     if (code > 0) return cudaGetErrorString((cudaError_t)code);

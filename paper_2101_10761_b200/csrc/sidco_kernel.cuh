@@ -86,9 +86,12 @@ struct SegDev {
 
 struct Control {
     unsigned count;      // grid barrier arrivals since the workspace was set up (never reset by the kernel)
-    unsigned unused;
+    unsigned seq;        // calls completed since then: call number seq + 1 tags SegDev::pub and gives the barrier
+                         // its target, (seq + 1) * G arrivals.  Advanced by the kernel itself, so that a launch's
+                         // arguments do not change from call to call (a recorded launch can be replayed)
     int timeout;         // set when a bounded wait ran out
-    int pad;
+    int residual_is_zero;  // the next call takes the residual's contents as zeros and does not read them
+                         // (set by a state reset, cleared by the call)
     unsigned long long t_ns[16];  // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
 };
 
@@ -124,9 +127,6 @@ struct Args {
     double delta, delta1, eps_H, eps_L;
     int Q, sid, max_stages;
     int C, S, G;
-    int call_id;                 // per-workspace call number, tags SegDev::pub
-    unsigned barrier_target;     // value of Control::count once every CTA of this call has arrived
-    int residual_is_zero;        // the residual's contents are to be taken as zeros and not read
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
 };
@@ -138,6 +138,7 @@ struct Args {
 __device__ __forceinline__ int ld_cg(const int* p) { return __ldcg(p); }
 __device__ __forceinline__ float ld_cg(const float* p) { return __ldcg(p); }
 __device__ __forceinline__ double ld_cg(const double* p) { return __ldcg(p); }
+__device__ __forceinline__ unsigned ld_cg(const unsigned* p) { return __ldcg(p); }
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -203,8 +204,8 @@ __device__ __forceinline__ void grid_barrier(Control* ctl, unsigned target) {
 // Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).  Returns the
 // threshold published with that stage.  Only runs holding chunks of the segment wait for it, and the next
 // stage cannot be fitted before they have swept those chunks, so the word read is the one of stage `need`.
-__device__ __forceinline__ float wait_ready_thread(const Args& A, const SegDev* sg, int need) {
-    const unsigned target = (unsigned)A.call_id * 16u + (unsigned)need;
+__device__ __forceinline__ float wait_ready_thread(const Args& A, unsigned call_id, const SegDev* sg, int need) {
+    const unsigned target = call_id * 16u + (unsigned)need;
     long long spins = 0;
     unsigned long long w;
     while ((int)((unsigned)(w = ld_acquire_u64(&sg->pub)) - target) < 0) {     // wrap-safe
@@ -216,9 +217,9 @@ __device__ __forceinline__ float wait_ready_thread(const Args& A, const SegDev* 
 }
 
 // Warp-level wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).
-__device__ __forceinline__ float wait_ready(const Args& A, const SegDev* sg, int need) {
+__device__ __forceinline__ float wait_ready(const Args& A, unsigned call_id, const SegDev* sg, int need) {
     float thr = 0.0f;
-    if ((threadIdx.x & 31) == 0) thr = wait_ready_thread(A, sg, need);
+    if ((threadIdx.x & 31) == 0) thr = wait_ready_thread(A, call_id, sg, need);
     return __shfl_sync(kFull, thr, 0);
 }
 
@@ -344,6 +345,7 @@ __device__ inline double stage_ratio(double delta, double delta1, int M, int m) 
 struct LnTab {
     const double* ln;       // [kMaxStages + 1] log(ratio)
     const double* ln_inv;   // [kMaxStages + 1] log(1 / ratio)
+    unsigned call_id;       // number of this call (tags the published words)
 };
 __device__ __forceinline__ int ratio_slot(int M, int m) { return (M == 1 || m == M - 1) ? M : 0; }
 
@@ -417,10 +419,10 @@ __device__ __forceinline__ void record_stage(SegDev* sg, int stage, const Fit& f
 // stored afterwards (record_stage).  If another stage follows, its sweep shifts by eta, which is therefore
 // stored before the word and released with it.  The word of a last stage carries all that its readers need
 // (they go on to read only their own run's data), so it is a plain strong store with no fence to wait for.
-__device__ inline Fit publish_stage(const Args& A, SegDev* sg, int stages, bool last, double eta) {
+__device__ inline Fit publish_stage(unsigned call_id, SegDev* sg, int stages, bool last, double eta) {
     Fit f{eta, last ? __double2float_ru(eta) : __double2float_rd(eta), stages, last, 0, 0, 0, false};
     const unsigned long long word = ((unsigned long long)__float_as_uint(f.thr) << 32) |
-                                    (unsigned long long)((unsigned)A.call_id * 16u + (unsigned)stages);
+                                    (unsigned long long)(call_id * 16u + (unsigned)stages);
     if (last) {
         st_relaxed_u64(&sg->pub, word);
     } else {
@@ -476,7 +478,7 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
         }
     }
     // an empty segment takes part in no later phase: all its stages count as fitted here
-    Fit f = publish_stage(A, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
+    Fit f = publish_stage(T.call_id, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
     f.M_eff = M_eff;
     f.status = status;
     f.empty = n == 0;
@@ -497,7 +499,7 @@ __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, d
         else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, T.ln[slot], T.ln_inv[slot], status);
         eta = prev + inc;
     }
-    Fit f = publish_stage(A, sg, m + 1, m + 1 == M_eff, eta);
+    Fit f = publish_stage(T.call_id, sg, m + 1, m + 1 == M_eff, eta);
     f.M_eff = M_eff;
     f.status = status;
     f.n_e = n_e;
@@ -711,6 +713,7 @@ __device__ __forceinline__ Sums strided_partials(const Args& A, int first, int q
 
 // Table entries of the segments of a CTA run, cached in shared memory at kernel start.
 struct RunSegs {
+    unsigned call_id;           // number of this call
     int seg_lo, n_seg;          // segments seg_lo .. seg_lo + n_seg - 1 have chunks in (or between) this run
     int* q0;                    // [kSegCache] first chunk
     int* q1;                    // [kSegCache] one past the last chunk
@@ -737,7 +740,7 @@ __device__ __forceinline__ void publish_params(const Args& A, const RunSegs& R, 
     if (i < R.n_seg && i < kSegCache && R.q1[i] > R.q0[i] && R.ok[i] != tag) {
         const SegDev* sg = &A.seg[R.seg_lo + i];
         const int M_eff = R.m_eff[i];
-        R.thr[i] = wait_ready_thread(A, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
+        R.thr[i] = wait_ready_thread(A, R.call_id, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
         // only a segment with a further stage is swept in this phase and needs the shift
         R.eta_prev[i] = (m_prev >= 0 && M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
         __threadfence_block();
@@ -765,7 +768,7 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
         // beyond the cache (a run spanning more than kSegCache segments): straight from global memory
         const SegDev* sg = &A.seg[seg];
         v.M_eff = seg_stages(A, seg, cap);
-        v.thr_gt = v.thr_ge = wait_ready(A, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
+        v.thr_gt = v.thr_ge = wait_ready(A, R.call_id, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
         v.eta_prev = (m_prev >= 0 && v.M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
     }
 }
@@ -891,13 +894,14 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ unsigned sm_done[kCoopChunks / 32];
     __shared__ int sm_coop_total;
     __shared__ int sm_any_tau;
+    __shared__ unsigned sm_call;
+    __shared__ int sm_reszero;
 
     const int cta = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int4 run = __ldg(A.cta_desc + cta);          // {first chunk, end chunk, first segment, segments}
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
-    const bool res_zero = A.residual_is_zero != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
@@ -905,8 +909,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     if (threadIdx.x == 0) sm_mloc = 1;
     if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
-    RunSegs R{run.z, run.w, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
-    const LnTab T{sm_ln, sm_ln_inv};
+    // What changes from call to call lives in the workspace (and is advanced after the grid barrier below,
+    // which no CTA passes before every CTA has read it here).  The loads are issued now and their values
+    // handed to the CTA after the table loop, whose own loads they overlap.
+    unsigned seq_loaded = 0u;
+    int reszero_loaded = 0;
+    if (threadIdx.x == 0) {
+        seq_loaded = ld_cg(&A.ctl->seq);
+        reszero_loaded = ld_cg(&A.ctl->residual_is_zero);
+    }
     if (threadIdx.x <= kMaxStages) {
         const int M = threadIdx.x;                    // slot 0: delta_1; slot M: last stage of M stages
         const double ratio = M == 0 ? A.delta1 : stage_ratio(A.delta, A.delta1, M, M - 1);
@@ -917,14 +928,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     auto stages_of = [&](int seg) -> int { return seg_stages(A, seg, cap); };
     // cache the run's segment table; find the largest stage count among the run's segments, which
     // is the number of statistics phases this CTA takes part in
-    for (int i = threadIdx.x; i < R.n_seg; i += kThreads) {
-        const int q0 = A.seg_chunk0[R.seg_lo + i], q1 = A.seg_chunk0[R.seg_lo + i + 1];
-        const int m = stages_of(R.seg_lo + i);
+    const int run_seg_lo = run.z, run_n_seg = run.w;
+    for (int i = threadIdx.x; i < run_n_seg; i += kThreads) {
+        const int q0 = A.seg_chunk0[run_seg_lo + i], q1 = A.seg_chunk0[run_seg_lo + i + 1];
+        const int m = stages_of(run_seg_lo + i);
         if (i < kSegCache) {
-            sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[R.seg_lo + i];
+            sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[run_seg_lo + i];
             sm_meff[i] = m;
-            sm_segn[i] = A.seg_n[R.seg_lo + i];
-            const float tau = A.seg[R.seg_lo + i].spec_thr;
+            sm_segn[i] = A.seg_n[run_seg_lo + i];
+            const float tau = A.seg[run_seg_lo + i].spec_thr;
             sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
             if (sm_tau[i] > 0.0f && q1 > q0) sm_any_tau = 1;
             sm_ok[i] = 0;
@@ -936,11 +948,17 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const bool p1_desc = A.cta_dir[cta] != 0;
     int resweep = 0;             // chunks of acc this warp read a second time in full
 
+    if (threadIdx.x == 0) { sm_call = seq_loaded + 1u; sm_reszero = reszero_loaded; }
+    __syncthreads();
+    const unsigned call_id = sm_call;
+    const bool res_zero = sm_reszero != 0;
+    RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
+    const LnTab T{sm_ln, sm_ln_inv, call_id};
+
     // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
         if (A.seg_chunk0[s + 1] == A.seg_chunk0[s])
             record_stage(&A.seg[s], 0, fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T), 0, 1);
-    __syncthreads();
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
     // that precedes their last fit records which slots may hold survivors).  It depends on state the
@@ -1509,8 +1527,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     }
     __syncthreads();
     cta_count = sm_base;
-    grid_barrier(A.ctl, A.barrier_target);
+    grid_barrier(A.ctl, call_id * (unsigned)A.G);
     if (stamper) A.ctl->t_ns[4] = global_ns();
+    if (cta == 0 && threadIdx.x == 0) {                 // this call is over as far as the next one's tags go
+        A.ctl->seq = call_id;
+        A.ctl->residual_is_zero = 0;
+    }
 
     // Per-segment bookkeeping (counts, adaptation, next candidate threshold) is spread over the grid, one
     // segment per thread, segment s going to thread (s / G) % kThreads of CTA s % G.  What it reads is
@@ -1634,10 +1656,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     if (stamper) A.ctl->t_ns[5] = global_ns();
 }
 
-// Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared.  The published
-// words keep their call tags.
-__global__ void sidco_reset_state_kernel(SegDev* seg, int S) {
+// Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared, the residual
+// declared empty.  The published words keep their call tags.
+__global__ void sidco_reset_state_kernel(SegDev* seg, int S, Control* ctl) {
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s == 0) ctl->residual_is_zero = 1;
     if (s < S) {
         seg[s].M = 1;
         seg[s].calls = 0;
