@@ -27,7 +27,7 @@ class GpuRun:
         self.d = int(self.off[-1])
         dev = "cuda:0"
         cap = self.d + 8 + base_shift
-        # base_shift > 0 gives pointers that are not 16-byte aligned (scalar path)
+        # base_shift > 0 gives pointers that are not 32-byte aligned (scalar path)
         self._res_store = torch.zeros(cap, dtype=torch.float32, device=dev)
         self._grad_store = torch.zeros(cap, dtype=torch.float32, device=dev)
         self.res = self._res_store[base_shift:base_shift + self.d]

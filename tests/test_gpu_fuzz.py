@@ -55,7 +55,7 @@ def test_random_segment_tables(seed):
 @pytest.mark.parametrize("sid,max_stages", [(0, -1), (1, 3), (2, -2)])
 def test_more_segments_per_run_than_the_cache_holds(sid, max_stages):
     """~150,000 segments of 1-4 elements: every CTA run spans about a thousand segments, more than the
-    512 whose parameters are cached in shared memory and more than one 1024-thread pass of the arrival loop."""
+    256 whose parameters are cached in shared memory and more than one 1024-thread pass of the arrival loop."""
     r = rng(77)
     sizes = [int(x) for x in r.integers(1, 5, 150000)]
     scales = np.exp(r.uniform(np.log(1e-4), np.log(1e-2), len(sizes)))
