@@ -59,7 +59,7 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.side_val = take(sizeof(float) * (size_t)(d + 4));
     L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
     L.stage_val = take(sizeof(float) * (size_t)(d + 4));
-    L.cta_total = take(sizeof(int32_t) * (size_t)(G + 1));
+    L.cta_total = take(sizeof(unsigned long long) * (size_t)(G + 1));
     L.cand = take(32 * (size_t)(T + 1));
     L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
     L.cta_ns = take(sizeof(unsigned long long) * 4 * (size_t)(G + 1));
@@ -232,7 +232,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
         if ((e = cudaMemcpy(seg_host.data(), (char*)c->ws + c->L.seg, sizeof(SegDev) * S, cudaMemcpyDeviceToHost)) !=
             cudaSuccess)
             return e;
-        for (auto& sg : seg_host) { sg.arrived = 0; sg.k_acc = 0; sg.pub = 0; }    // (the call numbering restarts below)
+        for (auto& sg : seg_host) { sg.arrived = 0; sg.k_acc = 0; sg.k_arr = 0; sg.pub = 0; }    // (the call numbering restarts below)
     } else {
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
         for (auto& sg : seg_host) {
@@ -252,6 +252,8 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
+    // (the call numbering restarts: no run's published count may carry a number of the old numbering)
+    if ((e = cudaMemset(base + L.cta_total, 0, sizeof(unsigned long long) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
@@ -306,7 +308,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.side_val = (float*)(base + L.side_val);
     a.stage_idx = (int32_t*)(base + L.stage_idx);
     a.stage_val = (float*)(base + L.stage_val);
-    a.cta_total = (int32_t*)(base + L.cta_total);
+    a.cta_pub = (unsigned long long*)(base + L.cta_total);
     a.cand = (unsigned char*)(base + L.cand);
     a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.cta_ns = (unsigned long long*)(base + L.cta_ns);
@@ -505,6 +507,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.cta_total, 0, sizeof(unsigned long long) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
         // the uploads read the fixed host arrays: let them finish before those can change again
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
         c.key = residual;
@@ -536,7 +539,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.side_val = (float*)(base + L.side_val);
     a.stage_idx = (int32_t*)(base + L.stage_idx);
     a.stage_val = (float*)(base + L.stage_val);
-    a.cta_total = (int32_t*)(base + L.cta_total);
+    a.cta_pub = (unsigned long long*)(base + L.cta_total);
     a.cand = base + L.cand;
     a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.cta_ns = (unsigned long long*)(base + L.cta_ns);
@@ -664,6 +667,7 @@ int sidco_reset_state(const float* residual) {
     Control ctl;
     std::memset(&ctl, 0, sizeof(Control));
     ctl.residual_is_zero = 1;
+    if ((e = cudaMemset(base + c->L.cta_total, 0, sizeof(unsigned long long) * (c->G + 1))) != cudaSuccess) return (int)e;
     if ((e = cudaMemcpy(base + c->L.ctl, &ctl, sizeof(Control), cudaMemcpyHostToDevice)) != cudaSuccess) return (int)e;
     return 0;
 }

@@ -71,7 +71,8 @@ struct SegDev {
     int32_t M_eff;       // stages used by this call
     int32_t status;
     int32_t arrived;     // CTA runs of this segment finished in the current phase (self-resetting)
-    int32_t k_acc;       // survivors counted so far in this call (integer atomics; self-resetting)
+    int32_t k_acc;       // survivors counted so far in this call by runs that keep no shared-memory count for the
+                         // segment (integer atomics; self-resetting)
     int32_t M;           // adaptation state: stage count for the next adaptive call
     int32_t calls;
     long long k_sum;
@@ -80,15 +81,20 @@ struct SegDev {
     // word: the fp32 compare threshold of the newest stage, thr_ge if that stage is the segment's last,
     // thr_gt otherwise, so that a waiting thread has it with the same load that tells it the stage is fitted.
     unsigned long long pub;
+    // Survivor count of the call and the runs that have reported theirs: each run adds (count << 32) + 1 with one
+    // atomic, and the run whose addition completes the arrivals has the segment's total in the value returned,
+    // writes out_k and does the adaptation step (self-resetting).
+    unsigned long long k_arr;
     float spec_thr;      // candidate threshold for the next call's first sweep (<= 0: none), see P1
     int32_t pad;
 };
 
 struct Control {
-    unsigned count;      // grid barrier arrivals since the workspace was set up (never reset by the kernel)
-    unsigned seq;        // calls completed since then: call number seq + 1 tags SegDev::pub and gives the barrier
-                         // its target, (seq + 1) * G arrivals.  Advanced by the kernel itself, so that a launch's
-                         // arguments do not change from call to call (a recorded launch can be replayed)
+    unsigned count;      // CTAs that have finished, over all calls since the workspace was set up (never reset by
+                         // the kernel): the one that brings it to (seq + 1) * G closes the call
+    unsigned seq;        // calls completed since then: call number seq + 1 tags SegDev::pub and Args::cta_pub.
+                         // Advanced by the kernel itself, so that a launch's arguments do not change from call to
+                         // call (a recorded launch can be replayed)
     int timeout;         // set when a bounded wait ran out
     int residual_is_zero;  // the next call takes the residual's contents as zeros and does not read them
                          // (set by a state reset, cleared by the call)
@@ -117,7 +123,7 @@ struct Args {
     float* side_val;             // [d]
     int32_t* stage_idx;          // [d]
     float* stage_val;            // [d]
-    int32_t* cta_total;          // [G]
+    unsigned long long* cta_pub; // [G] {call number, survivors of the run}: published once the run's selection is done
     unsigned char* cand;         // [C][32] per-lane slot flags of full chunks: slot may hold a survivor
     int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
     unsigned long long* cta_ns;  // [G][4] globaltimer when the CTA finished its P1, P3, last P4, P5a sweep
@@ -172,33 +178,16 @@ __device__ __forceinline__ int atom_add_acquire(int* p, int v) {
     return old;
 }
 
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
-}
-
-// Grid-wide barrier, used once per call: every CTA adds one arrival to a counter that is never reset and
-// waits until it reaches the value the host computed for this call (arrivals before the call + grid size),
-// so the last arrival releases the others with the same atomic that records it.  All CTAs of the
-// cooperative launch are resident, so the wait normally ends within microseconds; it is nevertheless
-// bounded, and a CTA whose wait runs out raises the timeout flag, which ends every other wait of the call.
-__device__ __forceinline__ void grid_barrier(Control* ctl, unsigned target) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const unsigned old = atomicAdd(&ctl->count, 1u);
-        if ((int)(old + 1u - target) < 0) {
-            long long spins = 0;
-            while ((int)(ld_acquire(&ctl->count) - target) < 0) {       // wrap-safe
-                if (ld_volatile(&ctl->timeout)) break;
-                if (++spins > kSpinLimit) { atomicExch(&ctl->timeout, 1); break; }
-                __nanosleep(spins < 64 ? 20 : 200);
-            }
-        }
-        __threadfence();
-    }
-    __syncthreads();
 }
 
 // Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).  Returns the
@@ -208,9 +197,13 @@ __device__ __forceinline__ float wait_ready_thread(const Args& A, unsigned call_
     const unsigned target = call_id * 16u + (unsigned)need;
     long long spins = 0;
     unsigned long long w;
-    while ((int)((unsigned)(w = ld_acquire_u64(&sg->pub)) - target) < 0) {     // wrap-safe
-        if (ld_volatile(&A.ctl->timeout)) break;
-        if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+    // (polled with plain strong loads: the word carries the threshold itself; a reader that goes on to load
+    // eta, stored before a non-last stage's word and released with it, orders that load with a fence)
+    while ((int)((unsigned)(w = ld_relaxed_u64(&sg->pub)) - target) < 0) {     // wrap-safe
+        // (the time-out flag is looked at now and then only: a second dependent load in every round would
+        // double the time it takes to notice the word)
+        if ((++spins & 15) == 0 && ld_volatile(&A.ctl->timeout)) break;
+        if (spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
         __nanosleep(spins < 16 ? 20 : 100);
     }
     return __uint_as_float((unsigned)(w >> 32));
@@ -398,7 +391,7 @@ __device__ __forceinline__ void record_stage(SegDev* sg, int stage, const Fit& f
     if (stage == 0) {
         for (int q = first; q < 20; q += step) {
             if (q < 8) sg->eta[q] = (q == 0 || (f.empty && q < f.M_eff)) ? f.eta : 0.0;
-            else if (q < 16) sg->k_stage[q - 8] = 0;
+            else if (q < 16) { if (q - 8 >= f.M_eff) sg->k_stage[q - 8] = 0; }   // the others are written by later fits / the count
             else if (q == 16) sg->M_eff = f.M_eff;
             else if (q == 17) sg->status = f.status;
             else if (q == 18) sg->thr_gt = __double2float_rd(f.eta);
@@ -742,7 +735,12 @@ __device__ __forceinline__ void publish_params(const Args& A, const RunSegs& R, 
         const int M_eff = R.m_eff[i];
         R.thr[i] = wait_ready_thread(A, R.call_id, sg, need == 0 ? M_eff : (need < M_eff ? need : M_eff));
         // only a segment with a further stage is swept in this phase and needs the shift
-        R.eta_prev[i] = (m_prev >= 0 && M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
+        double eta_prev = 0.0;
+        if (m_prev >= 0 && M_eff > need) {
+            __threadfence();                       // acquire side of the stage's release
+            eta_prev = ld_cg(&sg->eta[m_prev]);
+        }
+        R.eta_prev[i] = eta_prev;
         __threadfence_block();
         R.ok[i] = tag;
     }
@@ -769,7 +767,11 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
         const SegDev* sg = &A.seg[seg];
         v.M_eff = seg_stages(A, seg, cap);
         v.thr_gt = v.thr_ge = wait_ready(A, R.call_id, sg, need == 0 ? v.M_eff : (need < v.M_eff ? need : v.M_eff));
-        v.eta_prev = (m_prev >= 0 && v.M_eff > need) ? ld_cg(&sg->eta[m_prev]) : 0.0;
+        v.eta_prev = 0.0;
+        if (m_prev >= 0 && v.M_eff > need) {
+            __threadfence();                       // acquire side of the stage's release
+            v.eta_prev = ld_cg(&sg->eta[m_prev]);
+        }
     }
 }
 
@@ -887,6 +889,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ double sm_ln[kMaxStages + 1], sm_ln_inv[kMaxStages + 1];
     __shared__ double sm_eta[kSegCache];
     __shared__ int sm_ok[kSegCache];
+    __shared__ int sm_segk[kSegCache];      // survivors of the run per cached segment
     __shared__ int sm_oidx[kOutCache];
     __shared__ float sm_oval[kOutCache];
     __shared__ unsigned short sm_items[kCoopItems];
@@ -940,6 +943,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
             if (sm_tau[i] > 0.0f && q1 > q0) sm_any_tau = 1;
             sm_ok[i] = 0;
+            sm_segk[i] = 0;
         }
         if (q1 > q0) atomicMax(&sm_mloc, m);
     }
@@ -954,11 +958,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const bool res_zero = sm_reszero != 0;
     RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
     const LnTab T{sm_ln, sm_ln_inv, call_id};
-
-    // Segments without chunks (n = 0) never see an arrival: give them their defaults here.
-    for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
-        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s])
-            record_stage(&A.seg[s], 0, fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T), 0, 1);
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
     // that precedes their last fit records which slots may hold survivors).  It depends on state the
@@ -1393,12 +1392,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
                     atomicOr(&sm_done[k2 >> 5], 1u << (k2 & 31));
                     cnt = sm_ccnt[threadIdx.x];
                     A.chunk_cnt[c0 + k2] = cnt;
-                    if (cnt) key = R.seg_lo + (sm_cseg[threadIdx.x] & (kAllSlots - 1));
+                    if (cnt) key = sm_cseg[threadIdx.x] & (kAllSlots - 1);
                 }
-                // one counter update per segment and warp
+                // one counter update per segment and warp (the pass takes cached segments only)
                 const unsigned peers = __match_any_sync(kFull, key);
                 const int sum = __reduce_add_sync(peers, cnt);
-                if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&A.seg[key].k_acc, sum);
+                if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sm_segk[key], sum);
             }
             if (threadIdx.x == 0) sm_coop_total += carry;
             before_pass += carry;
@@ -1423,6 +1422,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         if (n_rest > kThreads) n_rest = -1;          // more than the list holds
     }
     const bool place_from_smem = n_rest == 0 && before_pass <= kOutCache;
+    // survivors of a segment found by the warp loop: into the run's shared-memory count if the segment has one
+    auto add_seg_count = [&](int seg, int n) {
+        const int i = seg - R.seg_lo;
+        if (i < kSegCache) atomicAdd(&sm_segk[i], n);
+        else atomicAdd(&A.seg[seg].k_acc, n);
+    };
     auto next_chunk = [&]() -> int {
         return n_rest >= 0 ? queue.next_listed(sm_list, n_rest) : queue.next_undone(!p1_desc, sm_done, coop_n);
     };
@@ -1435,7 +1440,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         while (cur.c >= 0) {
             const Desc nxt = fetch_desc(A, next_chunk(), true, true);
             if (cur.seg != sv.seg) {
-                if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
+                if (seg_count && lane == 0) add_seg_count(sv.seg, seg_count);
                 seg_count = 0;
                 view_load(A, R, sv, cur.seg, 0, -1, 100, cap);
                 // multi-stage segments keep their exceedances in the side region; single-stage ones
@@ -1508,55 +1513,48 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             warp_total += cnt;
             cur = nxt;
         }
-        if (seg_count && lane == 0) atomicAdd(&A.seg[sv.seg].k_acc, seg_count);
+        if (seg_count && lane == 0) add_seg_count(sv.seg, seg_count);
     }
     if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
-    // (what this CTA stored for the placement becomes visible to the grid through the barrier below:
-    // CTA barrier, then thread 0's fence and arrival)
     __syncthreads();
     if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns();
     if (stamper) A.ctl->t_ns[12] = global_ns();
     // next call: start the first sweep where this call's last full sweep over acc ended
     if (threadIdx.x == 0) A.cta_dir[cta] = (2 * sm_resweep >= c1 - c0) ? (p1_desc ? 1 : 0) : (p1_desc ? 0 : 1);
+
+    // No grid-wide barrier follows.  The run's survivor count is published as one tagged word, which the runs
+    // above it poll for their output base; a segment's total count comes out of the atomic by which the last of
+    // its runs reports (SegDev::k_arr).  Neither needs a fence: the words carry everything their readers use,
+    // and what this CTA stored for its own placement it reads back itself.
     int cta_count = 0;
     if (warp == 0) {
         int x = sm_warp[lane];
         #pragma unroll
         for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(kFull, x, o);
-        if (lane == 0) { A.cta_total[cta] = x; sm_base = x; }
+        if (lane == 0) {
+            st_relaxed_u64(&A.cta_pub[cta], ((unsigned long long)call_id << 32) | (unsigned)x);
+            sm_base = x;
+        }
     }
     __syncthreads();
     cta_count = sm_base;
-    grid_barrier(A.ctl, call_id * (unsigned)A.G);
-    if (stamper) A.ctl->t_ns[4] = global_ns();
-    if (cta == 0 && threadIdx.x == 0) {                 // this call is over as far as the next one's tags go
-        A.ctl->seq = call_id;
-        A.ctl->residual_is_zero = 0;
-    }
 
-    // Per-segment bookkeeping (counts, adaptation, next candidate threshold) is spread over the grid, one
-    // segment per thread, segment s going to thread (s / G) % kThreads of CTA s % G.  What it reads is
-    // loaded here, ahead of the placement, so that the two chains of memory round trips overlap.
-    struct SegEnd { int k_hat, M_eff, status, calls, M; long long k_sum; float thr, spec_thr; };
-    auto seg_end_load = [&](int s) -> SegEnd {
-        const SegDev* sg = &A.seg[s];
-        return SegEnd{ld_cg(&sg->k_acc), ld_cg(&sg->M_eff), ld_cg(&sg->status), sg->calls, sg->M, sg->k_sum,
-                      ld_cg(&sg->thr_ge), sg->spec_thr};
-    };
-    // per-segment counts, last stage count, adaptation (Algorithm 1, Adapt_Stages)
-    auto seg_end_store = [&](int s, const SegEnd& v, bool timed_out) {
+    // Per-segment end of call: counts, last stage count, adaptation (Algorithm 1, Adapt_Stages), next call's
+    // candidate threshold.  Done by the thread whose report completes the segment; reads nothing that another
+    // CTA wrote during this call except through that report.
+    const bool timed_out = ld_volatile(&A.ctl->timeout) != 0;
+    auto seg_finish = [&](int s, int M_eff, int k_hat, float thr) {
         SegDev* sg = &A.seg[s];
-        sg->k_acc = 0;
-        A.out_k[s] = v.k_hat;
-        sg->k_stage[v.M_eff - 1] = v.k_hat;
-        int status = v.status | (timed_out ? kStTimeout : 0);
+        A.out_k[s] = k_hat;
+        sg->k_stage[M_eff - 1] = k_hat;
+        if (timed_out) atomicOr(&sg->status, (int)kStTimeout);
         if (A.max_stages > 0) {
-            const int calls = v.calls + 1;
-            long long k_sum = v.k_sum + v.k_hat;
+            const int calls = sg->calls + 1;
+            long long k_sum = sg->k_sum + k_hat;
             if (calls % A.Q == 0) {
                 const double k_avg = (double)k_sum / (double)A.Q;
                 const double k_target = A.delta * (double)A.seg_n[s];
-                int M = v.M;
+                int M = sg->M;
                 if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
                 if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
                 if (M < 1) M = 1;
@@ -1567,32 +1565,71 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             sg->calls = calls;
             sg->k_sum = k_sum;
         }
-        // candidate threshold for the next call's first sweep (and whether this call's guess held);
-        // v.M still is the state this call's stage count came from
-        {
-            int m_call = A.max_stages > 0 ? (v.M < 1 ? 1 : (v.M > A.max_stages ? A.max_stages : v.M)) : -A.max_stages;
-            if (m_call > cap) m_call = cap;
-            const float tau_used = (A.spec_enable && m_call <= 2 && v.spec_thr > 0.0f) ? v.spec_thr : -1.0f;
-            if (tau_used > 0.0f) status |= (v.thr >= tau_used ? kStFlagsUsed : kStFlagsMissed);
-        }
-        if (status != v.status) sg->status = status;
-        sg->spec_thr = (v.thr > 0.0f && v.thr < 3.0e38f) ? kSpecRatio * v.thr : -1.0f;
+        sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
     };
-    const int s_first = cta + A.G * (int)threadIdx.x;
-    SegEnd first{};
-    if (s_first < A.S) first = seg_end_load(s_first);
+    for (int ib = 0; ib < R.n_seg; ib += kThreads) {
+        const int i = ib + (int)threadIdx.x;
+        if (i < R.n_seg) {
+            int q0, q1, runs;
+            R.get(A, i, q0, q1, runs);
+            if (q1 > q0) {
+                const int s = R.seg_lo + i;
+                SegDev* sg = &A.seg[s];
+                if (i < kSegCache) {
+                    const int cnt = sm_segk[i];
+                    unsigned long long old = 0ull;
+                    if (runs > 1) old = atomicAdd(&sg->k_arr, ((unsigned long long)(unsigned)cnt << 32) | 1ull);
+                    if (runs == 1 || (int)(old & 0xFFFFFFFFull) == runs - 1) {
+                        if (runs > 1) sg->k_arr = 0ull;
+                        seg_finish(s, R.m_eff[i], (int)(old >> 32) + cnt, R.thr[i]);
+                    }
+                } else {
+                    // no shared-memory count: the warps added to k_acc; report after those additions
+                    __threadfence();
+                    const bool last = runs == 1 || atom_add_acquire(&sg->arrived, 1) == runs - 1;
+                    if (last) {
+                        const int k_hat = ld_cg(&sg->k_acc);
+                        sg->k_acc = 0;
+                        sg->arrived = 0;
+                        const float thr = __uint_as_float((unsigned)(ld_acquire_u64(&sg->pub) >> 32));
+                        seg_finish(s, seg_stages(A, s, cap), k_hat, thr);
+                    }
+                }
+            }
+        }
+    }
+
+    // Segments without chunks (n = 0) never see an arrival or a report: their defaults and their end of call
+    // are done here, spread over the grid.
+    for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
+        if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) {
+            const Fit f = fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
+            record_stage(&A.seg[s], 0, f, 0, 1);
+            seg_finish(s, f.M_eff, 0, f.thr);
+        }
 
     // ------------------------------------------------------------------ P5b: final positions
     {
-        // survivors of the runs below this one: summed by one warp (a grid has a few hundred CTAs at most)
+        // survivors of the runs below this one: each run's word is polled (bounded) until it carries this
+        // call's number; summed by one warp (a grid has a few hundred CTAs at most)
         if (warp == 0) {
             int below = 0;
-            for (int c = lane; c < cta; c += 32) below += ld_cg(A.cta_total + c);
+            for (int c = lane; c < cta; c += 32) {
+                unsigned long long w;
+                long long spins = 0;
+                while ((unsigned)((w = ld_relaxed_u64(&A.cta_pub[c])) >> 32) != call_id) {
+                    if ((++spins & 15) == 0 && ld_volatile(&A.ctl->timeout)) break;
+                    if (spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+                    __nanosleep(spins < 64 ? 20 : 100);
+                }
+                below += (int)(unsigned)w;
+            }
             #pragma unroll
             for (int o = 16; o > 0; o >>= 1) below += __shfl_down_sync(kFull, below, o);
             if (lane == 0) sm_base = below;
         }
         __syncthreads();
+        if (stamper) A.ctl->t_ns[4] = global_ns();
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
         if (place_from_smem) {
@@ -1647,10 +1684,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             __syncthreads();
         }
     }
-    {
-        const bool timed_out = ld_volatile(&A.ctl->timeout) != 0;
-        if (s_first < A.S) seg_end_store(s_first, first, timed_out);
-        for (int s = s_first + A.G * kThreads; s < A.S; s += A.G * kThreads) seg_end_store(s, seg_end_load(s), timed_out);
+    // The CTA that finishes last closes the call: from then on the next call's number is in force.  (Every CTA
+    // read the current one at its start, long before it could get here.)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned done = atomicAdd(&A.ctl->count, 1u) + 1u;
+        if (done == call_id * (unsigned)A.G) {
+            A.ctl->seq = call_id;
+            A.ctl->residual_is_zero = 0;
+        }
     }
 
     if (stamper) A.ctl->t_ns[5] = global_ns();
