@@ -274,17 +274,20 @@ __device__ __forceinline__ int block_exscan(int x, int* sm, int& total) {
     return warp_incl - sm[warp] + incl - x;
 }
 
-// The same for one half of the CTA (warps 16 h .. 16 h + 15), the two halves working independently: they
-// meet at named barrier 1 + h.  Result valid in the half's first thread.
-__device__ __forceinline__ Sums half_tree(double a, double b, int n, double (*sm)[3], int h) {
+// The same for one group of kFitGroupWarps warps (warps g * kFitGroupWarps ...), the groups working
+// independently: a group meets at named barrier 1 + g.  Result valid in the group's first thread.
+constexpr int kFitGroupWarps = 12;
+constexpr int kFitGroups = 2;            // the remaining warps fit small segments meanwhile
+__device__ __forceinline__ Sums group_tree(double a, double b, int n, double (*sm)[3], int g) {
     Sums w = warp_tree(a, b, n);
-    const int lane = threadIdx.x & 31, wh = (threadIdx.x >> 5) & 15;
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + h), "r"(kThreads / 2) : "memory");      // previous use of sm is over
-    if (lane == 0) { sm[wh][0] = w.a; sm[wh][1] = w.b; sm[wh][2] = (double)w.n; }
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + h), "r"(kThreads / 2) : "memory");
+    const int lane = threadIdx.x & 31, wg = (threadIdx.x >> 5) - g * kFitGroupWarps;
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(32 * kFitGroupWarps) : "memory");   // previous use of sm is over
+    if (lane == 0) { sm[wg][0] = w.a; sm[wg][1] = w.b; sm[wg][2] = (double)w.n; }
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(32 * kFitGroupWarps) : "memory");
     Sums r{0.0, 0.0, 0};
-    if (wh == 0) {
-        double x = lane < 16 ? sm[lane][0] : 0.0, y = lane < 16 ? sm[lane][1] : 0.0, z = lane < 16 ? sm[lane][2] : 0.0;
+    if (wg == 0) {
+        const bool in = lane < kFitGroupWarps;
+        double x = in ? sm[lane][0] : 0.0, y = in ? sm[lane][1] : 0.0, z = in ? sm[lane][2] : 0.0;
         #pragma unroll
         for (int o = 8; o > 0; o >>= 1) {
             x += __shfl_down_sync(kFull, x, o);
@@ -835,23 +838,26 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         }
         __syncthreads();
         const int n_small = sm_count[0], n_large = sm_count[1];
-        // large segments first (other runs wait for them): half a CTA each, the two halves working on two
-        // segments at a time; threads stride over the chunk partials, fixed tree over the half
-        {
-            const int h = warp >> 4, th = threadIdx.x & (kThreads / 2 - 1);
-            for (int k = h; k < n_large; k += 2) {
+        // Large segments (other runs wait for them) are fitted by two groups of twelve warps, two segments at
+        // a time: threads stride over the chunk partials, fixed tree over the group.  The other eight warps
+        // take the small segments meanwhile (all warps do if there is no large one).
+        const int g = warp / kFitGroupWarps;
+        if (g < kFitGroups) {
+            const int tg = threadIdx.x - g * 32 * kFitGroupWarps;
+            for (int k = g; k < n_large; k += kFitGroups) {
                 const int i2 = sm_large[k];
                 int q0, q1, runs;
                 R.get(A, i2, q0, q1, runs);
                 SegDev* sg = &A.seg[R.seg_lo + i2];
-                const int M_state = (stage == 0 && th == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
-                const Sums t = strided_partials(A, q0 + th, q1, kThreads / 2);
-                Sums r = half_tree(t.a, t.b, t.n, sm_red + 16 * h, h);
-                if (th < 32) fit_and_cache(sg, i2, M_state, r);
+                const int M_state = (stage == 0 && tg == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
+                const Sums t = strided_partials(A, q0 + tg, q1, 32 * kFitGroupWarps);
+                Sums r = group_tree(t.a, t.b, t.n, sm_red + kFitGroupWarps * g, g);
+                if (tg < 32) fit_and_cache(sg, i2, M_state, r);
             }
         }
         // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
-        for (int k = warp; k < n_small; k += kWarps) {
+        const int small_first = n_large ? kFitGroups * kFitGroupWarps : 0;       // warps that take them
+        for (int k = warp - small_first; k >= 0 && k < n_small; k += kWarps - small_first) {
             const int i2 = sm_small[k];
             int q0, q1, runs;
             R.get(A, i2, q0, q1, runs);
