@@ -918,6 +918,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     if (threadIdx.x == 0) sm_mloc = 1;
     if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
+    if (threadIdx.x < kCoopChunks / 32) sm_done[threadIdx.x] = 0u;
     // What changes from call to call lives in the workspace (and is advanced after the grid barrier below,
     // which no CTA passes before every CTA has read it here).  The loads are issued now and their values
     // handed to the CTA after the table loop, whose own loads they overlap.
@@ -1236,11 +1237,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     // the survivors fit, the final placement copies them from there instead of reading the staging regions.
     bool published = false;
     int coop_n = 0;                       // leading chunks of the run this pass covers
+    int coop_done = 0;                    // chunks it took
     int before_pass = 0;                  // survivors found by the passes before the current one
     if (vec_ok && sm_any_tau) {
         coop_n = min(c1 - c0, kCoopChunks);
-        for (int i = threadIdx.x; i < kCoopChunks / 32; i += kThreads) sm_done[i] = 0u;
-        __syncthreads();
         // Threshold of a chunk's segment once its last stage is fitted; true if the chunk's listed slots
         // hold all its survivors.  `tag` is the segment's cache index, plus kAllSlots if all of the chunk's
         // slots were listed (then no flags are involved).
@@ -1390,11 +1390,13 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             }
             if (!published) { publish_params(A, R, 0, -1, 100); published = true; }
             __syncthreads();
+            bool took = false;
             if (threadIdx.x < kCoopPass) {            // whole warps: one thread per chunk of the pass
                 const int k2 = base + (int)threadIdx.x;
                 int key = -1, cnt = 0;
                 float t;
                 if (k2 < coop_n && sm_cseg[threadIdx.x] >= 0 && seg_thr(sm_cseg[threadIdx.x], t)) {
+                    took = true;
                     atomicOr(&sm_done[k2 >> 5], 1u << (k2 & 31));
                     cnt = sm_ccnt[threadIdx.x];
                     A.chunk_cnt[c0 + k2] = cnt;
@@ -1407,7 +1409,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
             }
             if (threadIdx.x == 0) sm_coop_total += carry;
             before_pass += carry;
-            __syncthreads();
+            coop_done += __syncthreads_count(took);
         }
         if (threadIdx.x == 0) warp_total += sm_coop_total;
     }
@@ -1415,7 +1417,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     // The chunks left for the warp loop, if the pass above covered the whole run: listed, so that the warps
     // do not take turns at the queue for every chunk already done (few are left).
     int n_rest = -1;                      // < 0: no list, the loop goes through the queue and skips the chunks done
-    if (coop_n == c1 - c0 && coop_n > 0) {
+    if (coop_n == c1 - c0 && coop_done == coop_n) {
+        n_rest = 0;                       // nothing left (the usual case)
+    } else if (coop_n == c1 - c0 && coop_n > 0) {
         for (int k = threadIdx.x; k < coop_n; k += kThreads)
             if (!((sm_done[k >> 5] >> (k & 31)) & 1u)) {
                 const int p = atomicAdd(&sm_count[0], 1);
@@ -1442,7 +1446,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         SegView sv;
         bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
-        Desc cur = fetch_desc(A, next_chunk(), true, true);
+        Desc cur = fetch_desc(A, n_rest == 0 ? -1 : next_chunk(), true, true);
         while (cur.c >= 0) {
             const Desc nxt = fetch_desc(A, next_chunk(), true, true);
             if (cur.seg != sv.seg) {
