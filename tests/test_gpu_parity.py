@@ -207,6 +207,59 @@ print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [o
     assert outs[0] == outs[1] == outs[2]
 
 
+@pytest.mark.parametrize("delta", [0.01, 0.03])
+def test_many_survivors_per_run(delta):
+    """About a thousand (delta = 0.01) or three thousand (0.03) survivors per CTA: around and above what a run keeps
+    in shared memory for the placement, and more flagged slots than one round (0.01) or one pass (0.03) of the
+    block-wide selection takes."""
+    wl = W.config(3)
+    off = wl.seg_offsets
+    run = GpuRun(off)
+    res_o = np.zeros(wl.d, np.float32)
+    try:
+        for call in range(3):
+            g = wl.draw(call)
+            ora = O.sidco_compress(g, res_o, off, f32(delta), O.SID_EXP, -1)
+            gpu = run.step(g, f32(delta), O.SID_EXP, -1)
+            check_parity(gpu, ora, off)
+            res_o = ora.residual
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("sid,max_stages", [(0, -1), (2, -2)])
+def test_long_runs_of_chunks_per_cta(sid, max_stages):
+    """With three CTAs a run holds about 4800 chunks: the block-wide selection pass then needs several passes
+    and does not cover the whole run, so the per-warp loop has to skip what the pass took.  Three calls, so
+    that candidate flags exist from the second call on."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import sys, numpy as np
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+from oracle import sidco_oracle as O
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, check_parity, f32
+sid, ms = %d, %d
+wl = W.config(3)
+off, delta = wl.seg_offsets, f32(0.001)
+run = GpuRun(off)
+res_o = np.zeros(wl.d, np.float32)
+for call in range(3):
+    g = wl.draw(call)
+    ora = O.sidco_compress(g, res_o, off, delta, sid, ms)
+    gpu = run.step(g, delta, sid, ms)
+    check_parity(gpu, ora, off)
+    res_o = ora.residual
+run.close()
+print("parity ok")
+''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)), sid, max_stages)
+    env = dict(os.environ, SIDCO_GRID="3")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and "parity ok" in r.stdout, (r.stdout[-1000:], r.stderr[-3000:])
+
+
 @pytest.mark.parametrize("use_async", [False, True])
 def test_reset_declares_the_residual_empty(use_async):
     """After a reset the next call must behave as if the residual were all zeros, whatever it holds,
