@@ -59,8 +59,8 @@ extern "C" {
 #define SIDCO_ST_DEGENERATE 2   /* a fit took one of its degenerate-case rules */
 #define SIDCO_ST_ALL_ZERO   4   /* every magnitude is zero: nothing is selected */
 #define SIDCO_ST_TIMEOUT    8   /* a bounded wait inside the kernel ran out; results are invalid */
-#define SIDCO_ST_FLAGS_USED   16  /* informational: the final selection read only pre-flagged slots of acc */
-#define SIDCO_ST_FLAGS_MISSED 32  /* informational: the threshold fell below the pre-flagging bound; acc was re-read */
+#define SIDCO_ST_FLAGS_USED   16  /* reserved: informational bit of earlier versions, not set any more */
+#define SIDCO_ST_FLAGS_MISSED 32  /* reserved: informational bit of earlier versions, not set any more */
 
 typedef struct sidco_seg_debug {
     int32_t M_used;                       /* stages used by the last call (after the cap for delta) */

@@ -20,7 +20,7 @@ SID_EXP, SID_GAMMA, SID_GPD = 0, 1, 2
 MAX_STAGES = 8
 
 ST_NONFINITE, ST_DEGENERATE, ST_ALL_ZERO, ST_TIMEOUT = 1, 2, 4, 8
-ST_FLAGS_USED, ST_FLAGS_MISSED = 16, 32      # informational
+ST_FLAGS_USED, ST_FLAGS_MISSED = 16, 32      # reserved, not set any more
 
 
 class SegDebug(C.Structure):

@@ -61,7 +61,7 @@ constexpr long long kSpinLimit = 1ll << 22;       // bounded waits: ~1 s with th
 static_assert(kWarps == 32, "block_tree and the scans assume 32 warps per CTA");
 
 enum { kSidExp = 0, kSidGamma = 1, kSidGpd = 2 };
-enum { kStNonFinite = 1, kStDegenerate = 2, kStAllZero = 4, kStTimeout = 8, kStFlagsUsed = 16, kStFlagsMissed = 32 };
+enum { kStNonFinite = 1, kStDegenerate = 2, kStAllZero = 4, kStTimeout = 8 };
 
 struct SegDev {
     double eta[kMaxStages];
