@@ -3,6 +3,7 @@
 #include "sidco_kernel.cuh"
 
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -268,6 +269,15 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     return cudaSuccess;
 }
 
+// Logarithms of the stage ratios (see Args::ln_ratio).
+void fill_ln_tables(Args& a, double delta, double delta1) {
+    for (int M = 0; M <= sidco::kMaxStages; ++M) {
+        const double ratio = M == 0 ? delta1 : sidco::stage_ratio(delta, delta1, M, M - 1);
+        a.ln_ratio[M] = std::log(ratio);
+        a.ln_inv_ratio[M] = std::log(1.0 / ratio);
+    }
+}
+
 // Cooperative launch: all CTAs of the persistent kernel are co-resident.
 cudaError_t launch_persistent(const void* fn, int grid, void** kargs, cudaStream_t stream) {
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), kargs, 0, stream);
@@ -316,6 +326,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;
     a.delta1 = prm.delta1;
+    fill_ln_tables(a, (double)delta, prm.delta1);
     a.eps_H = prm.eps_H;
     a.eps_L = prm.eps_L;
     a.Q = prm.Q;
@@ -547,6 +558,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;
     a.delta1 = g_params.delta1;
+    fill_ln_tables(a, (double)delta, g_params.delta1);
     a.eps_H = g_params.eps_H;
     a.eps_L = g_params.eps_L;
     a.Q = g_params.Q;

@@ -131,6 +131,9 @@ struct Args {
     Control* ctl;
     // scalars
     double delta, delta1, eps_H, eps_L;
+    // log(ratio) and log(1 / ratio) of the stage ratios, from the host: slot 0 is delta_1 (every stage but the
+    // last), slot M the ratio of the last stage of an M-stage schedule (delta for M = 1)
+    double ln_ratio[kMaxStages + 1], ln_inv_ratio[kMaxStages + 1];
     int Q, sid, max_stages;
     int C, S, G;
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
@@ -328,7 +331,7 @@ __device__ __forceinline__ int seg_stages(const Args& A, int seg, int cap) {
 }
 
 // Tail ratio of stage m (0-based) out of M: delta_1 for every non-final stage, the rest for the last.
-__device__ inline double stage_ratio(double delta, double delta1, int M, int m) {
+__host__ __device__ inline double stage_ratio(double delta, double delta1, int M, int m) {
     if (M == 1) return delta;
     if (m < M - 1) return delta1;
     double p = 1.0;
@@ -336,8 +339,8 @@ __device__ inline double stage_ratio(double delta, double delta1, int M, int m) 
     return delta / p;
 }
 
-// Logarithms of the stage ratios, computed once per CTA: slot 0 is delta_1 (every stage but the last), slot M
-// the ratio of the last stage of an M-stage schedule (delta for M = 1).
+// Logarithms of the stage ratios (Args::ln_ratio, Args::ln_inv_ratio): slot 0 is delta_1 (every stage but the
+// last), slot M the ratio of the last stage of an M-stage schedule (delta for M = 1).
 struct LnTab {
     const double* ln;       // [kMaxStages + 1] log(ratio)
     const double* ln_inv;   // [kMaxStages + 1] log(1 / ratio)
@@ -880,7 +883,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
 // ----------------------------------------------------------------------------
 
 template <int SID>
-__global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Args A) {
+__global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __grid_constant__ Args A) {
     __shared__ double sm_red[kWarps][3];
     __shared__ int sm_list[kThreads];
     __shared__ int sm_scan[kThreads];
@@ -892,7 +895,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     __shared__ int sm_mloc;
     __shared__ int sm_q0[kSegCache], sm_q1[kSegCache], sm_runs[kSegCache], sm_meff[kSegCache], sm_segn[kSegCache];
     __shared__ float sm_tau[kSegCache], sm_thr[kSegCache];
-    __shared__ double sm_ln[kMaxStages + 1], sm_ln_inv[kMaxStages + 1];
     __shared__ double sm_eta[kSegCache];
     __shared__ int sm_ok[kSegCache];
     __shared__ int sm_segk[kSegCache];      // survivors of the run per cached segment
@@ -912,11 +914,18 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
+    // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
+    // of the last call) ended, so that it begins on the lines most recently left in L2.
+    const bool p1_desc = A.cta_dir[cta] != 0;
+    // The first chunk of every warp is fixed (chunk number `warp` of the sweep; the queue starts behind
+    // these), so that its descriptor can be fetched now, under the set-up that follows.
+    const int first_chunk = warp < c1 - c0 ? (p1_desc ? c1 - 1 - warp : c0 + warp) : -1;
+    const Desc first_desc = fetch_desc(A, first_chunk, false);
     const int cap = stage_cap(A.delta, A.delta1);
     const bool stamper = (cta == 0 && threadIdx.x == 0);
     if (stamper) A.ctl->t_ns[0] = global_ns();
     if (threadIdx.x == 0) sm_mloc = 1;
-    if (threadIdx.x == 0) { sm_next = 0; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
+    if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
     if (threadIdx.x < kCoopChunks / 32) sm_done[threadIdx.x] = 0u;
     // What changes from call to call lives in the workspace (and is advanced after the grid barrier below,
@@ -927,12 +936,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     if (threadIdx.x == 0) {
         seq_loaded = ld_cg(&A.ctl->seq);
         reszero_loaded = ld_cg(&A.ctl->residual_is_zero);
-    }
-    if (threadIdx.x <= kMaxStages) {
-        const int M = threadIdx.x;                    // slot 0: delta_1; slot M: last stage of M stages
-        const double ratio = M == 0 ? A.delta1 : stage_ratio(A.delta, A.delta1, M, M - 1);
-        sm_ln[M] = log(ratio);
-        sm_ln_inv[M] = log(1.0 / ratio);
     }
     __syncthreads();
     auto stages_of = [&](int seg) -> int { return seg_stages(A, seg, cap); };
@@ -954,9 +957,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         }
         if (q1 > q0) atomicMax(&sm_mloc, m);
     }
-    // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
-    // of the last call) ended, so that it begins on the lines most recently left in L2.
-    const bool p1_desc = A.cta_dir[cta] != 0;
     int resweep = 0;             // chunks of acc this warp read a second time in full
 
     if (threadIdx.x == 0) { sm_call = seq_loaded + 1u; sm_reszero = reszero_loaded; }
@@ -964,7 +964,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
     const unsigned call_id = sm_call;
     const bool res_zero = sm_reszero != 0;
     RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
-    const LnTab T{sm_ln, sm_ln_inv, call_id};
+    const LnTab T{A.ln_ratio, A.ln_inv_ratio, call_id};
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
     // that precedes their last fit records which slots may hold survivors).  It depends on state the
@@ -981,7 +981,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const Arg
         int tau_seg = -1;
         float tau = -1.0f;
         bool keep = true;          // ask for L2 residency of this segment's acc lines
-        Desc cur = fetch_desc(A, queue.next(p1_desc), false);
+        Desc cur = first_desc;
         while (cur.c >= 0) {
             const Desc nxt = fetch_desc(A, queue.next(p1_desc), false);
             const int c = cur.c, lo = cur.lo, hi = cur.hi;
