@@ -185,8 +185,8 @@ int sidco_reset_state_async(const float* residual, void* stream);
  * (`out` has room for n_segs entries).  Synchronises the device; meant for tests and logging. */
 int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);
 
-/* Phase breakdown of the last call in microseconds, from device timestamps taken by one CTA at the
- * grid-wide barriers: us_out[0] error compensation + stage-1 statistics and fit, [1] stage-2 side-buffer
+/* Phase breakdown of the last call in microseconds, from device timestamps taken by the first CTA as it
+ * moves from phase to phase (the other CTAs move on their own): us_out[0] error compensation + stage-1 statistics and fit, [1] stage-2 side-buffer
  * compaction and fit, [2] stages 3..M, [3] survivor staging + residual zeroing, [4] final placement and
  * adaptation, [5] whole kernel; then finer marks of that CTA alone: [6] its first sweep, [7] its arrivals
  * and fits after it, [8] its stage-2 sweep, [9] arrivals and fits after it, [10] arrivals and fits of the

@@ -7,10 +7,12 @@
 // Inside a run the warps pull chunks from a shared-memory queue and work on them
 // without any block-level synchronisation: a chunk is loaded, reduced with warp
 // shuffles, and compacted with ballots by one warp.  A CTA moves from one phase to
-// the next on its own: a warp that needs a segment's threshold waits (bounded) on
-// that segment's "stages ready" word, which the run completing the segment's
-// statistics publishes with release semantics.  One grid-wide barrier remains,
-// before the final placement, which needs every CTA's survivor count:
+// the next on its own: a run that needs a segment's threshold waits (bounded) on
+// that segment's published word {call number, stages fitted, threshold}, which
+// the run completing the segment's statistics stores.  There is no grid-wide
+// barrier: for the final placement every run publishes its survivor count as a
+// tagged word that the runs above it poll, and a segment's total count comes out
+// of the atomic by which the last of its runs reports.
 //
 //   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
 //       of every chunk; the CTA whose run completes a segment sums the per-chunk
@@ -26,12 +28,17 @@
 //       segments with more stages compact their exceedances, in order, into the
 //       chunk's side region
 //   P4  (m = 3..M) statistics of side-region entries above eta_{m-1}; fit eta_m
-//   P5a survivors |x| >= eta_M staged per chunk in ascending order (from the
-//       flagged slots of acc or all of acc for M <= 2, from the side region
-//       otherwise), selected residual entries zeroed
-//   P5b CTA bases from the per-CTA totals, chunk bases by a block scan, staged
-//       survivors copied to their final ascending positions, per-segment counts
-//       and stage adaptation (Algorithm 1, Adapt_Stages)
+//   P5a survivors |x| >= eta_M staged per chunk in ascending order, selected
+//       residual entries zeroed.  A block-wide pass lists the flagged slots of
+//       the run's full chunks (and all slots of its ragged chunks) in shared
+//       memory and fetches them in one wave; a per-warp loop takes what that
+//       pass cannot (invalid flags: all of acc; three or more stages: the side
+//       region)
+//   P5b base of the run = published counts of the runs below; survivors copied
+//       to their final ascending positions (from shared memory, or from the
+//       staging regions through a block scan of the chunk counts); per-segment
+//       counts and stage adaptation (Algorithm 1, Adapt_Stages) by the thread
+//       whose report completes the segment
 //
 // Reductions are deterministic and independent of the grid: per-lane sequential
 // accumulation in a fixed order, a fixed shuffle tree per chunk, and a fixed-order
@@ -392,7 +399,9 @@ __device__ __forceinline__ Fit warp_broadcast(const Fit& f) {
 // the threads first, first + step, ... of a group that all hold `f` (a warp, or one thread with step 1).
 // `stage` = 0 writes the whole record of the call's first stage and clears the later stages' entries.
 // These stores are ordered before any later fit of the segment by the fence and arrival atomic of this
-// CTA's next phase, and before the final placement by the grid barrier.
+// CTA's next phase.  Nothing else reads them during the call: the end of the call takes a segment's stage
+// count and threshold from the run's own cache or from the published word, and writes only entries that
+// this record leaves alone (k_stage[M_eff - 1], the adaptation state).
 __device__ __forceinline__ void record_stage(SegDev* sg, int stage, const Fit& f, int first, int step) {
     if (stage == 0) {
         for (int q = first; q < 20; q += step) {
@@ -928,9 +937,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
     if (threadIdx.x < kCoopChunks / 32) sm_done[threadIdx.x] = 0u;
-    // What changes from call to call lives in the workspace (and is advanced after the grid barrier below,
-    // which no CTA passes before every CTA has read it here).  The loads are issued now and their values
-    // handed to the CTA after the table loop, whose own loads they overlap.
+    // What changes from call to call lives in the workspace (and is advanced by the CTA that finishes the call
+    // last, long after every CTA has read it here).  The loads are issued now and their values handed to the
+    // CTA after the table loop, whose own loads they overlap.
     unsigned seq_loaded = 0u;
     int reszero_loaded = 0;
     if (threadIdx.x == 0) {
