@@ -1159,17 +1159,30 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             A.part_n[c] = r.n;
                         }
                     } else {
+                        // The side region also takes the entries equal to eta_1: they are no exceedances (the
+                        // statistics above leave them out), but if no later stage raises the threshold
+                        // (eta_M = eta_1, e.g. a segment of equal magnitudes) the final rule |x| >= eta_M selects them.
+                        // (An fp32 magnitude can equal eta_1 only if eta_1 is an fp32 value, which then is thr_gt.)
+                        unsigned keep_mask = mask;
+                        if ((double)sv.thr_gt == sv.eta_prev) {
+                            #pragma unroll
+                            for (int j = 0; j < kSlots; ++j)
+                                #pragma unroll
+                                for (int cc = 0; cc < kComp; ++cc)
+                                    if (fabsf(v[j][cc]) == sv.thr_gt) keep_mask |= 1u << (8 * j + cc);
+                            keep_mask &= valid;
+                        }
                         const int e0 = wb + lane * kComp;
-                        const int cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                        const int cnt = ordered_emit(keep_mask, lo, [&](int p, int j, int cc) {
                             A.side_idx[p] = e0 + j * 256 + cc;
                             A.side_val[p] = v[j][cc];
                         });
-                        Sums r = warp_tree(sy, sy2, 0);
+                        Sums r = warp_tree(sy, sy2, __popc(mask));
                         if (lane == 0) {
                             A.part[3 * (size_t)c + 0] = r.a;
                             A.part[3 * (size_t)c + 1] = r.b;
-                            A.part_n[c] = cnt;
-                            A.side_cnt[c] = cnt;
+                            A.part_n[c] = r.n;          // exceedances (the next fit's count)
+                            A.side_cnt[c] = cnt;        // entries stored
                         }
                     }
                 }

@@ -207,6 +207,33 @@ print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [o
     assert outs[0] == outs[1] == outs[2]
 
 
+@pytest.mark.parametrize("sid", SIDS)
+@pytest.mark.parametrize("M", [2, 3])
+def test_ties_with_the_first_threshold(sid, M):
+    """Segments whose magnitudes are all equal (or that hold one element) make the moment-matched fit return
+    eta_1 = the magnitude itself, no later stage raises it, and the rule |x| >= eta_M selects everything.  The
+    elements equal to eta_1 are no exceedances, yet must reach the final selection.  Indices are compared
+    exactly here (the usual tolerance band would hide a miss), over several calls."""
+    sizes = [1, 4000, 7, 1, 2500, 3000]
+    off = W.offsets_from_sizes(sizes)
+    d = int(off[-1])
+    run = GpuRun(off)
+    res_o = np.zeros(d, np.float32)
+    try:
+        for call in range(3):
+            g = W.ragged_case(40 + call, sizes, 1e-2)
+            g[off[1]:off[2]] = np.float32(0.25) * np.where(np.arange(4000) % 3 == 0, -1, 1)     # equal magnitudes
+            g[off[4]:off[5]] = np.float32(0.125 * (call + 1))
+            ora = O.sidco_compress(g, res_o, off, f32(0.05), sid, -M)
+            gpu = run.step(g, f32(0.05), sid, -M)
+            check_parity(gpu, ora, off)
+            assert np.array_equal(gpu["idx"], ora.idx), f"call {call}: index sets differ"
+            assert np.array_equal(gpu["residual"].view(np.uint32), ora.residual.view(np.uint32))
+            res_o = ora.residual
+    finally:
+        run.close()
+
+
 @pytest.mark.parametrize("delta", [0.01, 0.03])
 def test_many_survivors_per_run(delta):
     """About a thousand (delta = 0.01) or three thousand (0.03) survivors per CTA: around and above what a run keeps
