@@ -52,6 +52,37 @@ def test_random_segment_tables(seed):
              zero_frac=float(r.choice([0.0, 0.0, 0.5])))
 
 
+@pytest.mark.parametrize("seed", [6277, 6286, 6295, 6298, 6309, 6331] + list(range(7000, 7018)))
+def test_random_tables_long_sequences(seed):
+    """A second generator: up to 80 segments that also come as whole slots (multiples of 8) and whole windows
+    (multiples of 1024), up to eight calls per case so that errors of one call show in the next, exact zeros in
+    some.  The first six seeds are cases that an earlier version failed (one-element segments with a
+    moment-matched multi-stage fit: entries equal to the first threshold)."""
+    r = rng(seed)
+    n_segs = int(r.integers(1, 80))
+    kinds = r.integers(0, 6, n_segs)
+    sizes = []
+    for kd in kinds:
+        if kd == 0:
+            sizes.append(int(r.integers(0, 8)))
+        elif kd == 1:
+            sizes.append(int(r.integers(1, 300)))
+        elif kd == 2:
+            sizes.append(int(r.integers(900, 5000)))
+        elif kd == 3:
+            sizes.append(int(r.integers(20000, 90000)))
+        elif kd == 4:
+            sizes.append(8 * int(r.integers(1, 40000)))
+        else:
+            sizes.append(1024 * int(r.integers(1, 400)))
+    scales = np.exp(r.uniform(np.log(1e-6), np.log(1e-1), n_segs))
+    delta = float(r.choice([0.3, 0.1, 0.03, 0.01, 0.003, 0.001, 0.0003]))
+    sid = int(r.integers(0, 3))
+    max_stages = int(r.choice([-1, -2, -3, -5, 2, 4, 6]))
+    calls = int(r.integers(2, 9))
+    run_case(sizes, scales, delta, sid, max_stages, calls, seed, zero_frac=float(r.choice([0.0, 0.0, 0.0, 0.3])))
+
+
 @pytest.mark.parametrize("sid,max_stages", [(0, -1), (1, 3), (2, -2)])
 def test_more_segments_per_run_than_the_cache_holds(sid, max_stages):
     """~150,000 segments of 1-4 elements: every CTA run spans about a thousand segments, more than the
