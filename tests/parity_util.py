@@ -94,6 +94,10 @@ def check_parity(gpu, ora: O.Result, offsets, state=None, check_status=True):
             eta = ora.report[s].eta[-1]
             assert abs(abs(float(acc[j])) - eta) <= BAND_RTOL * eta, \
                 f"index {j} (seg {s}) differs outside the band: |x|={abs(float(acc[j]))!r} eta={eta!r}"
+            # the band is there for thresholds that differ in their last bits; with the same threshold on both
+            # sides the comparison |x| >= eta has one answer
+            assert gpu["debug"][s].eta[ora.report[s].M_used - 1] != eta, \
+                f"index {j} (seg {s}): same threshold {eta!r} on both sides but different selections"
         band_total = diff.size
     # per-segment counts agree with the GPU's own index list
     counts = np.bincount(np.searchsorted(off[1:], g_idx, side="right"), minlength=S)[:S] if g_idx.size else np.zeros(S, int)
