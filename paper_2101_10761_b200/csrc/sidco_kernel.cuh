@@ -1616,13 +1616,17 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         seg_finish(s, R.m_eff[i], (int)(old >> 32) + cnt, R.thr[i]);
                     }
                 } else {
-                    // no shared-memory count: the warps added to k_acc; report after those additions
+                    // no shared-memory count: the warps added to k_acc; report (arrival only) after those additions
                     __threadfence();
-                    const bool last = runs == 1 || atom_add_acquire(&sg->arrived, 1) == runs - 1;
+                    bool last = runs == 1;
+                    if (!last) {
+                        last = (int)(atomicAdd(&sg->k_arr, 1ull) & 0xFFFFFFFFull) == runs - 1;
+                        __threadfence();                   // acquire side: the other runs' additions to k_acc
+                    }
                     if (last) {
                         const int k_hat = ld_cg(&sg->k_acc);
                         sg->k_acc = 0;
-                        sg->arrived = 0;
+                        if (runs > 1) sg->k_arr = 0ull;
                         const float thr = __uint_as_float((unsigned)(ld_acquire_u64(&sg->pub) >> 32));
                         seg_finish(s, seg_stages(A, s, cap), k_hat, thr);
                     }
