@@ -1261,7 +1261,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     int coop_n = 0;                       // leading chunks of the run this pass covers
     int coop_done = 0;                    // chunks it took
     int before_pass = 0;                  // survivors found by the passes before the current one
-    if (vec_ok && sm_any_tau) {
+    // (A run of at most one chunk per warp goes straight to the warp loop: its two round trips beat the pass.)
+    if (vec_ok && sm_any_tau && c1 - c0 > kWarps) {
         coop_n = min(c1 - c0, kCoopChunks);
         // Threshold of a chunk's segment once its last stage is fitted; true if the chunk's listed slots
         // hold all its survivors.  `tag` is the segment's cache index, plus kAllSlots if all of the chunk's
