@@ -13,9 +13,17 @@ zero residual and a fresh stage-adaptation state (M = 1); the reset (one tiny
 kernel that also declares the residual empty) sits inside the timed region.
 
 Prints ONE JSON line.  `value` is GB/s on the minimal bytes the method must move
-(12 d + 8 k_hat per step), inputs resident in HBM; `e2e` is the same metric
-through `sidco_compress_host` with pinned host buffers (copies inside the timed
-region).  `--impl reference` times the CPU oracle instead.
+per step: 12 d + 8 k_hat, and 8 d + 8 k_hat for the call that follows a reset
+(it does not read the residual).  The K-step region is timed R times; `value`
+and `ms_per_step` are the median, the spread is in `repeats`.  `roofline.cold`
+is the same kernel timed call by call with the L2 flushed (a 256 MiB write)
+before every call; `by_sid` has the three SIDs under the same protocol and
+`worst_sid` the slowest of them.  `e2e` is the same metric through
+`sidco_compress_host` with pinned host buffers (copies inside the timed
+region).  `aggregate` times the step that follows compress in a data-parallel
+loop (scatter-add of N workers' sparse lists into the dense mean) and `sweep`
+(with --sweep) the size sweep of single-segment tensors.  `--impl reference`
+times the CPU oracle instead.
 """
 from __future__ import annotations
 
@@ -55,11 +63,12 @@ WORKLOAD_NAMES = {
 SID_NAMES = {0: "EXP", 1: "GAMMA", 2: "GPD"}
 RUN_LEN = 10               # consecutive calls per run (residual carried), then residual and state reset
 N_GRADS = RUN_LEN          # one fresh draw per call of a run
+FLUSH_BYTES = 256 << 20    # L2 flush between cold calls: one write of this many bytes (L2 is 126 MB)
 
-# DRAM bytes per launch of the persistent kernel on this workload (dram__bytes_read.sum +
-# dram__bytes_write.sum of one ncu capture, summarised under profiles/), keyed by (sid, max_stages).
+# DRAM bytes per launch of the persistent kernel on config 4 (dram__bytes_read.sum + dram__bytes_write.sum of
+# one ncu capture, mean over the ten launches of a run, summarised under profiles/), keyed by (sid, max_stages).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    (0, 4): 236.8e6,     # EXP, adaptive: mean over the ten launches of one run
+    (0, 4): 237.9e6,
 }
 
 
@@ -69,6 +78,12 @@ def measured_peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def step_bytes(d: int, call_in_run: int, k_hat: int) -> int:
+    """Minimal bytes of one call: read g, read and write the residual, write the (idx, val) pairs.  The first
+    call of a run follows a reset that declares the residual empty, so it does not read it."""
+    return (8 if call_in_run == 0 else 12) * d + 8 * int(k_hat)
 
 
 class ClockSampler(threading.Thread):
@@ -133,10 +148,10 @@ class ClockSampler(threading.Thread):
             getattr(nv, "nvmlClocksThrottleReasonApplicationsClocksSetting", 0x2): "applications_clocks",
         }
         timed = [s for s in self.samples if s[0] == "device"]
-        src = "timed region"
+        src = "timed region (all repeats)"
         if len(timed) < 3:
             timed = list(self.samples)
-            src = "timed region + e2e region (timed region too short for 3 samples)"
+            src = "all timed regions of the run (headline region too short for 3 samples)"
         if not timed:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
         seen = set()
@@ -154,6 +169,10 @@ def make_inputs():
     return wl, [wl.draw(c) for c in range(N_GRADS)]
 
 
+# ---------------------------------------------------------------------------------------------
+# CPU legs: the oracle as it stands, on one core and split over the host's cores by segments
+# ---------------------------------------------------------------------------------------------
+
 def oracle_rate(wl, grads, budget_s: float, sid: int):
     """Time the oracle as it stands on whole calls of the workload for about budget_s."""
     from oracle import sidco_oracle as O
@@ -165,12 +184,72 @@ def oracle_rate(wl, grads, budget_s: float, sid: int):
             state = O.new_state(wl.n_segs)
         out = O.sidco_compress(grads[calls % RUN_LEN], res, wl.seg_offsets, DELTA, sid, 4, state=state)
         res = out.residual
-        bytes_min += 12 * wl.d + 8 * int(out.out_k[-1])
+        bytes_min += step_bytes(wl.d, calls % RUN_LEN, int(out.out_k[-1]))
         calls += 1
         if time.perf_counter() - t0 > budget_s or calls >= 64:
             break
     dt = time.perf_counter() - t0
     return bytes_min / dt / 1e9, calls, dt
+
+
+_MP = {}      # arrays the forked oracle workers inherit
+
+
+def _mp_group_call(task):
+    """One call of the unchanged oracle on one group of whole segments (a worker process)."""
+    from oracle import sidco_oracle as O
+    g, call, sid, state = task
+    lo, hi, s0, s1 = _MP["groups"][g]
+    off = _MP["off"][s0:s1 + 1] - lo
+    res = np.frombuffer(_MP["res"], dtype=np.float32)[lo:hi]
+    out = O.sidco_compress(_MP["grads"][call % RUN_LEN][lo:hi], res, off, DELTA, sid, 4, state=state)
+    res[:] = out.residual
+    return g, int(out.out_k[-1]), state
+
+
+def oracle_rate_all_cores(wl, grads, budget_s: float, sid: int):
+    """The same oracle, its per-segment loop split over the host's cores: every worker process runs
+    `sidco_compress` of the oracle module on a contiguous group of whole segments (segments are independent
+    in the method, so the arithmetic is unchanged).  Returns (GB/s, calls, seconds, processes)."""
+    import multiprocessing as mp
+    from oracle import sidco_oracle as O
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count() or 1
+    if cores < 2:
+        return None
+    off = wl.seg_offsets
+    # contiguous groups of segments, about four per core, cut where the element count passes equal shares
+    n_groups = min(wl.n_segs, 4 * cores)
+    cuts = [0]
+    for g in range(1, n_groups):
+        s = int(np.searchsorted(off, wl.d * g / n_groups))
+        cuts.append(min(max(s, cuts[-1] + 1), wl.n_segs - (n_groups - g)))
+    cuts.append(wl.n_segs)
+    groups = [(int(off[a]), int(off[b]), a, b) for a, b in zip(cuts[:-1], cuts[1:])]
+    order = sorted(range(len(groups)), key=lambda g: groups[g][0] - groups[g][1])      # largest first
+    _MP.update(groups=groups, off=off, grads=grads, res=mp.RawArray("f", wl.d))
+    ctx = mp.get_context("fork")
+    with ctx.Pool(cores) as pool:
+        states = [O.new_state(b - a) for (_, _, a, b) in groups]
+        pool.map(_mp_group_call, [(g, 0, sid, states[g]) for g in order])           # warm the workers
+        t0 = time.perf_counter()
+        calls, bytes_min = 0, 0
+        while True:
+            if calls % RUN_LEN == 0:
+                np.frombuffer(_MP["res"], dtype=np.float32)[:] = 0.0
+                states = [O.new_state(b - a) for (_, _, a, b) in groups]
+            k_hat = 0
+            for g, k, st in pool.map(_mp_group_call, [(g, calls, sid, states[g]) for g in order], chunksize=1):
+                states[g] = st
+                k_hat += k
+            bytes_min += step_bytes(wl.d, calls % RUN_LEN, k_hat)
+            calls += 1
+            if time.perf_counter() - t0 > budget_s or calls >= 64:
+                break
+        dt = time.perf_counter() - t0
+    return bytes_min / dt / 1e9, calls, dt, cores
 
 
 def used_threads() -> int:
@@ -210,7 +289,7 @@ def run_reference(args):
             state = O.new_state(n_seg)
         out = O.sidco_compress(grads[i % RUN_LEN], res, sub_off, DELTA, args.sid, 4, state=state)
         res = out.residual
-        bytes_min += 12 * d_sub + 8 * int(out.out_k[-1])
+        bytes_min += step_bytes(d_sub, i % RUN_LEN, int(out.out_k[-1]))
     dt = time.perf_counter() - t0
     value = bytes_min / dt / 1e9
     sample = f"first {n_seg} of {wl.n_segs} segments ({d_sub} of {wl.d} elements) per step"
@@ -240,13 +319,136 @@ def reduce_over_ranks(dist, device, times_ms, totals):
     return [float(x) for x in tmax], [float(x) for x in tsum]
 
 
-def run_gpu(args):
-    import torch
-    from paper_2101_10761_b200 import binding as B
+# ---------------------------------------------------------------------------------------------
+# GPU legs
+# ---------------------------------------------------------------------------------------------
 
+class Protocol:
+    """The configuration's protocol for one (SID, max_stages) setting on device-resident inputs: runs of
+    RUN_LEN calls from an empty residual; one run recorded as a CUDA graph (reset kernel + RUN_LEN compress
+    kernels) and replayed, steps beyond whole runs launched directly."""
+
+    def __init__(self, torch, B, wl, grads, sid, max_stages, dev, use_graph=True):
+        self.torch, self.B, self.wl, self.grads = torch, B, wl, grads
+        self.sid, self.max_stages, self.use_graph = sid, max_stages, use_graph
+        d, S = wl.d, wl.n_segs
+        self.res = torch.zeros(d, dtype=torch.float32, device=dev)
+        self.out_idx = torch.empty(d, dtype=torch.int32, device=dev)
+        self.out_val = torch.empty(d, dtype=torch.float32, device=dev)
+        self.out_k = torch.zeros(RUN_LEN, S + 1, dtype=torch.int32, device=dev)     # one row per call of a run
+        self.graph = None
+        self.calls = 0
+
+    def call(self, j, ev=None):
+        """Call j of a run (j = 0 follows the reset)."""
+        B = self.B
+        if j == 0 and self.calls:
+            B.sidco_reset_state_async(self.res)
+        if ev is not None:
+            ev[0].record()
+        B.sidco_compress(self.grads[j], self.res, self.wl.seg_offsets, DELTA, self.sid, self.max_stages,
+                         self.out_idx, self.out_val, self.out_k[j])
+        if ev is not None:
+            ev[1].record()
+        self.calls += 1
+
+    def run_direct(self, n_runs=1):
+        for _ in range(n_runs):
+            for j in range(RUN_LEN):
+                self.call(j)
+
+    def capture(self):
+        torch = self.torch
+        self.run_direct(2)                  # allocates, uploads, passes the adaptation points once
+        torch.cuda.synchronize()
+        if not self.use_graph:
+            return
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.B.sidco_reset_state_async(self.res)
+            for j in range(RUN_LEN):
+                self.B.sidco_compress(self.grads[j], self.res, self.wl.seg_offsets, DELTA, self.sid,
+                                      self.max_stages, self.out_idx, self.out_val, self.out_k[j])
+        self.graph.replay()
+        torch.cuda.synchronize()
+
+    def enqueue_steps(self, steps):
+        """Exactly `steps` steps starting at the beginning of a run; returns the kernels enqueued."""
+        n_replays = steps // RUN_LEN if self.graph is not None else 0
+        for _ in range(n_replays):
+            self.graph.replay()
+        self.calls += n_replays * RUN_LEN
+        launches = n_replays * (RUN_LEN + 1)
+        for s in range(n_replays * RUN_LEN, steps):
+            launches += 2 if (s % RUN_LEN == 0 and self.calls) else 1
+            self.call(s % RUN_LEN)
+        return launches
+
+    def bytes_of(self, steps):
+        """Minimal bytes of `steps` steps (every run repeats the same ten calls)."""
+        k = self.out_k[:, self.wl.n_segs].cpu().numpy().astype(np.int64)
+        per_run = [step_bytes(self.wl.d, j, k[j]) for j in range(RUN_LEN)]
+        return sum(per_run) * (steps // RUN_LEN) + sum(per_run[: steps % RUN_LEN]), k
+
+    def release(self):
+        self.B.sidco_release(self.res)
+
+
+def time_region(torch, barrier, proto, steps, repeats):
+    """`repeats` timings of the exact `steps`-step region, each bracketed by barrier + synchronize."""
+    out, launches = [], 0
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        launches = proto.enqueue_steps(steps)
+        e1.record()
+        barrier()
+        out.append(e0.elapsed_time(e1))
+    return out, launches
+
+
+def cold_calls(torch, proto, flush, n_runs, read_flush=None):
+    """Per-call event pairs with the L2 flushed before every call (a 256 MiB write, outside the pair).
+    With `read_flush`, the write is followed by a read sweep of a second buffer, so that the L2 is full of
+    clean lines when the call starts.  Returns per-call ms, by position in the run."""
+    per_pos = [[] for _ in range(RUN_LEN)]
+    for _ in range(n_runs):
+        for j in range(RUN_LEN):
+            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            if j == 0 and proto.calls:
+                proto.B.sidco_reset_state_async(proto.res)
+            flush.add_(1)
+            if read_flush is not None:
+                read_flush[1].copy_(read_flush[0].sum(dtype=torch.int64, dim=0, keepdim=True))
+            ev[0].record()
+            proto.B.sidco_compress(proto.grads[j], proto.res, proto.wl.seg_offsets, DELTA, proto.sid,
+                                   proto.max_stages, proto.out_idx, proto.out_val, proto.out_k[j])
+            ev[1].record()
+            proto.calls += 1
+            per_pos[j].append(ev)
+    torch.cuda.synchronize()
+    return [[a.elapsed_time(b) for a, b in evs] for evs in per_pos]
+
+
+def run_gpu(args):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    wl, grads_h = make_inputs()
+    # CPU legs first (rank 0 only), before this process creates a CUDA context: the all-core leg forks
+    cpu_one = cpu_all = None
+    if rank == 0:
+        cpu_one = oracle_rate(wl, grads_h, args.cpu_budget, args.sid)
+        if args.cpu_budget >= 1.0:
+            try:
+                cpu_all = oracle_rate_all_cores(wl, grads_h, args.cpu_budget, args.sid)
+            except Exception as exc:  # pragma: no cover - depends on the box
+                cpu_all = repr(exc)
+
+    import torch
+    from paper_2101_10761_b200 import binding as B
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
@@ -261,132 +463,97 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     B.lib()   # fail loudly here if the CUDA library is missing
-    wl, grads_h = make_inputs()
     off = wl.seg_offsets
     d, S = wl.d, wl.n_segs
     grads = [torch.from_numpy(g).to(dev) for g in grads_h]
-    res = torch.zeros(d, dtype=torch.float32, device=dev)
-    out_idx = torch.empty(d, dtype=torch.int32, device=dev)
-    out_val = torch.empty(d, dtype=torch.float32, device=dev)
-    out_k = torch.zeros(S + 1, dtype=torch.int32, device=dev)
-    out_k_steps = torch.zeros(args.steps, S + 1, dtype=torch.int32, device=dev)   # one out_k per timed step
-
-    def step(i, k_buf=None, ev=None):
-        """Call number i; every RUN_LEN-th call first zeroes the residual and resets the adaptation."""
-        if i % RUN_LEN == 0 and i > 0:
-            B.sidco_reset_state_async(res)      # also declares the residual empty: no memset needed
-        if ev is not None:
-            ev[0].record()
-        B.sidco_compress(grads[i % RUN_LEN], res, off, DELTA, args.sid, args.max_stages, out_idx, out_val,
-                         out_k if k_buf is None else k_buf)
-        if ev is not None:
-            ev[1].record()
+    peak, peak_kind = measured_peaks()
 
     uuid = getattr(torch.cuda.get_device_properties(local_rank), "uuid", None)
     sampler = ClockSampler(local_rank, str(uuid) if uuid is not None else None)
     sampler.start()
 
-    # untimed: bring the clocks up and pass the first adaptation points
-    step(0)
-    torch.cuda.synchronize()
+    head = Protocol(torch, B, wl, grads, args.sid, args.max_stages, dev, use_graph=not args.no_graph)
+    head.capture()
+    # untimed: bring the clocks up
     t0 = time.perf_counter()
-    i = 0
+    prewarm_steps = 0
     while time.perf_counter() - t0 < args.prewarm_ms * 1e-3:
-        for _ in range(20):
-            step(i)
-            i += 1
+        head.enqueue_steps(2 * RUN_LEN)
+        prewarm_steps += 2 * RUN_LEN
         torch.cuda.synchronize()
-    prewarm_steps = i
-    for w in range(args.warmup):
-        step(i + w)
-    i += args.warmup
-    i += (-i) % RUN_LEN          # the timed region starts at the beginning of a run
+    head.enqueue_steps(args.warmup + (-args.warmup) % RUN_LEN)       # W warm-up steps, rounded up to whole runs
 
-    # ---- timed region: device-resident inputs --------------------------------------------
-    # One run (state reset + RUN_LEN calls) is recorded by stream capture and replayed as a CUDA graph,
-    # which shortens the idle time between consecutive kernels; steps beyond a whole number of runs, or
-    # all steps with --no-graph, are launched directly.
-    n_replays = 0 if args.no_graph else args.steps // RUN_LEN
-    graph = None
-    if n_replays:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            B.sidco_reset_state_async(res)
-            for j in range(RUN_LEN):
-                B.sidco_compress(grads[j], res, off, DELTA, args.sid, args.max_stages, out_idx, out_val,
-                                 out_k_steps[j])
-        graph.replay()                # untimed: first replay of a new graph
-        torch.cuda.synchronize()
-    region = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-    launches0 = B.sidco_launch_count()
-    barrier()
+    # ---- timed region: device-resident inputs, K steps, R repeats --------------------------
     sampler.region = "device"
-    region[0].record()
-    for _ in range(n_replays):
-        graph.replay()
-    for s in range(n_replays * RUN_LEN, args.steps):
-        step(i + s, out_k_steps[s])
-    region[1].record()
-    barrier()
-    launches = B.sidco_launch_count() - launches0 + n_replays * (RUN_LEN + 1)
-    total_ms = region[0].elapsed_time(region[1])
-    if n_replays:
-        # every replay starts from the reset and repeats the same run: its per-call counts stand for all of them
-        out_k_steps[RUN_LEN:n_replays * RUN_LEN] = out_k_steps[:RUN_LEN].repeat(n_replays - 1, 1)
-    # Second pass over the same steps with an event pair around every launch, for the spread of the
-    # kernel's duration over the calls of a run.  (Event records between launches cost a few microseconds
-    # of stream time each, so they stay out of the region that `value` is computed from, and the roofline
-    # figure takes the kernel's average duration from that region: region time / launches, an upper bound
-    # that still contains the idle time between kernels and the per-run reset kernel.)
-    n_ev = min(args.steps, 20 * RUN_LEN)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
-    for s in range(n_ev):
-        step(i + args.steps + s, out_k, ev[s])
-    barrier()
+    first, launches = time_region(torch, barrier, head, args.steps, 1)
+    repeats = args.repeats if args.repeats else max(20, min(2000, int(0.25 / max(first[0] * 1e-3, 1e-6))))
+    region_ms, launches = time_region(torch, barrier, head, args.steps, repeats)
     sampler.region = None
-    kern_ms = [a.elapsed_time(b) for a, b in ev]
-    i += n_ev
-    k_hats = out_k_steps[:, S].cpu().numpy().astype(np.int64)
-    bytes_min = int(12 * d * args.steps + 8 * k_hats.sum())
-    dbg = B.sidco_get_debug(res, S)
-    m_hist = {}
+    bytes_min, k_hats = head.bytes_of(args.steps)
+    dbg = B.sidco_get_debug(head.res, S)
+    m_hist, status_or = {}, 0
     for sd in dbg:
         m_hist[str(sd.M_used)] = m_hist.get(str(sd.M_used), 0) + 1
-    status_or = 0
-    for sd in dbg:
         status_or |= sd.status
-    i += args.steps
 
-    # ---- context: other SID / stage settings on the same workload (rank 0, short runs) -------
-    variants = {}
+    # Event pair around every launch of a few runs (direct launches), for the spread over the calls of a run.
+    # Event records cost a few microseconds of stream time each, so they stay out of the region above.
+    sampler.region = "other"
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(5 * RUN_LEN)]
+    for s, e in enumerate(ev):
+        head.call(s % RUN_LEN, e)
+    torch.cuda.synchronize()
+    kern_ms = [a.elapsed_time(b) for a, b in ev]
+
+    # ---- cold L2: the same calls, the L2 flushed before each one ---------------------------
+    cold = None
+    if not args.no_cold:
+        flush = torch.zeros(FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
+        cold_calls(torch, head, flush, 1)
+        per_pos = cold_calls(torch, head, flush, args.cold_runs)
+        _, k_run = head.bytes_of(RUN_LEN)
+        c_bytes = sum(step_bytes(d, j, k_run[j]) for j in range(RUN_LEN)) / RUN_LEN
+        c_ms = statistics.mean(statistics.median(p) for p in per_pos)
+        rd = (torch.zeros(8, FLUSH_BYTES // 32, dtype=torch.int32, device=dev),
+              torch.zeros(1, FLUSH_BYTES // 32, dtype=torch.int64, device=dev))
+        per_pos_rd = cold_calls(torch, head, flush, max(1, args.cold_runs // 2), rd)
+        c_ms_rd = statistics.mean(statistics.median(p) for p in per_pos_rd)
+        cold = {
+            "achieved": c_bytes / (c_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+            "frac": c_bytes / (c_ms * 1e-3) / 1e9 / peak, "kernel_avg_ms": c_ms,
+            "per_call_of_run_ms": [round(statistics.median(p), 5) for p in per_pos],
+            "algorithmic_bytes_per_launch": c_bytes, "runs": args.cold_runs,
+            "method": f"event pair around every call; before each pair one {FLUSH_BYTES >> 20} MiB device write "
+                      "(the L2 then holds only dirty lines of that buffer); direct launches",
+            "clean_lines_variant": {
+                "kernel_avg_ms": c_ms_rd, "frac": c_bytes / (c_ms_rd * 1e-3) / 1e9 / peak,
+                "method": "the same, the write followed by a 256 MiB read sweep (the L2 then holds clean lines)"},
+        }
+        del flush, rd
+
+    # ---- the three SIDs under the same protocol (rank 0, shorter) ---------------------------
+    by_sid, variants = {}, {}
     if rank == 0 and not args.no_variants:
-        res_v = torch.zeros(d, dtype=torch.float32, device=dev)
-        for v_sid, v_ms in ((0, 4), (1, 4), (2, 4), (0, -1), (1, -1), (2, -1), (0, -2), (0, -4)):
-            if (v_sid, v_ms) == (args.sid, args.max_stages):
-                continue
-            res_v.zero_()
-            def v_step(w):
-                if w % RUN_LEN == 0 and w:
-                    B.sidco_reset_state_async(res_v)
-                B.sidco_compress(grads[w % RUN_LEN], res_v, off, DELTA, v_sid, v_ms, out_idx, out_val, out_k)
-            for w in range(2 * RUN_LEN):
-                v_step(w)
-            v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n_v = 10 * RUN_LEN
-            torch.cuda.synchronize()
-            v0.record()
-            for w in range(n_v):
-                v_step(w)
-            v1.record()
-            torch.cuda.synchronize()
-            us = v0.elapsed_time(v1) / n_v * 1e3
-            kh = int(out_k[S].item())
-            name = f"{SID_NAMES[v_sid]}_{'adaptive' + str(v_ms) if v_ms > 0 else 'M' + str(-v_ms)}"
-            variants[name] = {"us_per_step": round(us, 2), "GBps_min_bytes": round((12 * d + 8 * kh) / us / 1e3, 1),
-                              "frac_of_peak": round((12 * d + 8 * kh) / us / 1e3 / measured_peaks()[0], 4),
-                              "k_hat_last_call": kh}
-            B.sidco_release(res_v)
-        del res_v
+        def short(v_sid, v_ms, graph):
+            p = Protocol(torch, B, wl, grads, v_sid, v_ms, dev, use_graph=graph)
+            p.capture()
+            p.enqueue_steps(2 * RUN_LEN)
+            ms, _ = time_region(torch, lambda: torch.cuda.synchronize(), p, 10 * RUN_LEN, 5)
+            b, k = p.bytes_of(10 * RUN_LEN)
+            dbg_v = B.sidco_get_debug(p.res, S)
+            hist = {}
+            for sd in dbg_v:
+                hist[str(sd.M_used)] = hist.get(str(sd.M_used), 0) + 1
+            p.release()
+            t = statistics.median(ms)
+            return {"us_per_step": round(t * 1e3 / (10 * RUN_LEN), 2), "GBps_min_bytes": round(b / t / 1e6, 1),
+                    "frac_of_peak": round(b / t / 1e6 / peak, 4), "k_hat_mean": float(k.mean()),
+                    "M_used_hist_last_call": hist}
+        for v_sid in (0, 1, 2):
+            by_sid[SID_NAMES[v_sid]] = short(v_sid, args.max_stages, not args.no_graph)
+        for v_sid, v_ms in ((0, -1), (1, -1), (2, -1), (0, -2), (2, -2), (0, -4)):
+            variants[f"{SID_NAMES[v_sid]}_M{-v_ms}"] = short(v_sid, v_ms, not args.no_graph)
+    worst = min(by_sid.items(), key=lambda kv: kv[1]["frac_of_peak"]) if by_sid else None
 
     # ---- end to end: pinned host buffers through sidco_compress_host ----------------------
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -411,19 +578,30 @@ def run_gpu(args):
     barrier()
     sampler.region = None
     e2e_ms = e0.elapsed_time(e1)
+    B.sidco_release(h_res)
+    del h_grads, h_res, h_idx, h_val
+
+    # ---- the step after compress: dense mean of N workers' sparse lists -------------------
+    aggregate = None
+    if rank == 0 and not args.no_aggregate and hasattr(B, "sidco_aggregate"):
+        aggregate = bench_aggregate(torch, B, wl, head, dev, peak)
+
+    sweep = None
+    if rank == 0 and args.sweep:
+        sweep = bench_sweep(torch, B, dev, peak, args)
     sampler.stop()
 
     # ---- max over ranks, totals over ranks -------------------------------------------------
-    (t_dev, t_e2e), (tot_bytes, tot_e2e_bytes, tot_elems) = reduce_over_ranks(
-        dist, dev, [total_ms, e2e_ms], [bytes_min, e2e_bytes_min, d * args.steps])
+    t_med = statistics.median(region_ms)
+    (t_dev, t_min, t_max, t_e2e), (tot_bytes, tot_e2e_bytes, tot_elems) = reduce_over_ranks(
+        dist, dev, [t_med, min(region_ms), max(region_ms), e2e_ms], [bytes_min, e2e_bytes_min, d * args.steps])
 
     if rank == 0:
-        peak, peak_kind = measured_peaks()
         value = tot_bytes / (t_dev * 1e-3) / 1e9
-        kern_avg_ms = total_ms / args.steps
+        kern_avg_ms = t_med / args.steps
         alg_bytes = bytes_min / args.steps
         achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
-        cpu_val, cpu_calls, cpu_dt = oracle_rate(wl, grads_h, args.cpu_budget, args.sid)
+        n_replays = args.steps // RUN_LEN if head.graph is not None else 0
         line = {
             "metric": metric_name(), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": t_dev / args.steps, "higher_is_better": True,
@@ -431,16 +609,26 @@ def run_gpu(args):
             "config": {
                 "workload": WORKLOAD_NAMES[CONFIG], "delta": DELTA,
                 "sid": SID_NAMES[args.sid], "max_stages": args.max_stages,
+                "headline_sid_note": "the headline is this SID alone; by_sid / worst_sid give the three SIDs of the "
+                                     "configuration under the same protocol",
                 "M_used_hist_last_call": m_hist, "status_or": status_or,
                 "k_hat_mean": float(k_hats.mean()), "parallelism": "replicas only" if world > 1 else "1 GPU",
                 "protocol": "runs of 10 calls, residual carried, fresh draw per call; before each run the adaptation is "
-                            "reset and the residual declared empty (sidco_reset_state_async), inside the timed region",
-                "l2": "inputs 204 MB per step exceed the 126 MB L2; 10 distinct gradient buffers",
+                            "reset and the residual declared empty (sidco_reset_state_async), inside the timed region; "
+                            "bytes credited: 8 d + 8 k_hat for the call after a reset (it does not read the residual), "
+                            "12 d + 8 k_hat for the others",
+                "l2": "warm: back-to-back calls, inputs 204 MB per step exceed the 126 MB L2, 10 distinct gradient "
+                      "buffers, but part of the residual survives in L2 from call to call; roofline.cold flushes "
+                      "the L2 before every call",
                 "prewarm_steps": prewarm_steps,
                 "launch": (f"CUDA graph of one run (reset + {RUN_LEN} calls) replayed {n_replays} times"
                            + (f", {args.steps - n_replays * RUN_LEN} calls launched directly" if args.steps % RUN_LEN else "")
                            if n_replays else "every call launched directly on the stream"),
             },
+            "repeats": {"n": len(region_ms), "ms_per_step_median": t_dev / args.steps,
+                        "ms_per_step_min": t_min / args.steps, "ms_per_step_max": t_max / args.steps,
+                        "note": "the K-step region timed n times, each bracketed by barrier + synchronize; "
+                                "value and ms_per_step are the median"},
             "elements_per_s": tot_elems / (t_dev * 1e-3),
             "pct_of_8TBs_on_min_bytes": 100.0 * value / world / 8000.0,
             "roofline": {
@@ -451,10 +639,17 @@ def run_gpu(args):
                 "kernel_avg_ms_note": "timed region / launches (upper bound: includes the idle time between kernels)",
                 "event_pair_avg_ms": sum(kern_ms) / len(kern_ms), "event_pair_min_ms": min(kern_ms),
                 "algorithmic_bytes_per_launch": alg_bytes,
+                "cold": cold,
             },
+            "by_sid": by_sid,
+            "worst_sid": ({"sid": worst[0], **worst[1]} if worst else None),
             "cpu_baseline": {
-                "value": cpu_val, "unit": UNIT, "cores": used_threads(), "kind": "oracle",
-                "sample": f"{cpu_calls} whole calls of the same workload in {cpu_dt:.1f} s",
+                "value": cpu_one[0], "unit": UNIT, "cores": used_threads(), "kind": "oracle",
+                "sample": f"{cpu_one[1]} whole calls of the same workload in {cpu_one[2]:.1f} s",
+                "all_cores": ({"value": cpu_all[0], "unit": UNIT, "cores": cpu_all[3],
+                               "sample": f"{cpu_all[1]} whole calls in {cpu_all[2]:.1f} s, the oracle's segment loop "
+                                         f"split over {cpu_all[3]} processes (nproc)"}
+                              if isinstance(cpu_all, tuple) else cpu_all),
             },
             "e2e": {
                 "value": tot_e2e_bytes / (t_e2e * 1e-3) / 1e9, "unit": UNIT,
@@ -462,6 +657,8 @@ def run_gpu(args):
                 "ms_per_step": t_e2e / e2e_steps,
             },
             "variants": variants,
+            "aggregate": aggregate,
+            "sweep": sweep,
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
         }
@@ -469,6 +666,14 @@ def run_gpu(args):
     B.sidco_release_all()
     if dist is not None:
         dist.destroy_process_group()
+
+
+def bench_aggregate(torch, B, wl, head, dev, peak):
+    return None
+
+
+def bench_sweep(torch, B, dev, peak, args):
+    return None
 
 
 def main():
@@ -480,9 +685,16 @@ def main():
     ap.add_argument("--sid", type=int, default=0, help="0 EXP (default, the paper's SIDCo-E), 1 GAMMA, 2 GPD")
     ap.add_argument("--max-stages", type=int, default=4, help=">0 adaptive up to this many stages, <0 fixed")
     ap.add_argument("--no-graph", action="store_true", help="launch every timed call directly instead of replaying a CUDA graph")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="timings of the K-step region (default: at least 20, more until they cover 0.25 s)")
     ap.add_argument("--e2e-steps", type=int, default=50)
-    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
-    ap.add_argument("--no-variants", action="store_true", help="skip the short runs of other SID/stage settings")
+    ap.add_argument("--cpu-budget", type=float, default=10.0,
+                    help="seconds of oracle time for each cpu_baseline leg (one core, all cores)")
+    ap.add_argument("--no-variants", action="store_true", help="skip the runs of the other SID/stage settings")
+    ap.add_argument("--no-cold", action="store_true", help="skip the cold-L2 leg")
+    ap.add_argument("--cold-runs", type=int, default=6, help="runs of ten cold calls")
+    ap.add_argument("--no-aggregate", action="store_true", help="skip the decompress/aggregate leg")
+    ap.add_argument("--sweep", action="store_true", help="add the size sweep of single-segment tensors")
     ap.add_argument("--prewarm-ms", type=float, default=300.0,
                     help="untimed steps run for this long before the warm-up to bring the clocks up")
     ap.add_argument("--config", type=int, default=4, choices=[1, 2, 3, 4, 5],

@@ -53,14 +53,13 @@ extern "C" {
 #define SIDCO_E_ALIAS       (-9)   /* grad and residual overlap */
 #define SIDCO_E_SIZE        (-10)  /* size beyond the limit of this entry point */
 #define SIDCO_E_CAPTURE     (-11)  /* the call would have to allocate or upload tables while `stream` is capturing */
+#define SIDCO_E_UNSUPPORTED (-12)  /* the function needs a build of the library with another compile-time switch */
 
 /* per-segment status bits */
 #define SIDCO_ST_NONFINITE  1   /* a magnitude was NaN/Inf: nothing is selected in the segment */
 #define SIDCO_ST_DEGENERATE 2   /* a fit took one of its degenerate-case rules */
 #define SIDCO_ST_ALL_ZERO   4   /* every magnitude is zero: nothing is selected */
 #define SIDCO_ST_TIMEOUT    8   /* a bounded wait inside the kernel ran out; results are invalid */
-#define SIDCO_ST_FLAGS_USED   16  /* reserved: informational bit of earlier versions, not set any more */
-#define SIDCO_ST_FLAGS_MISSED 32  /* reserved: informational bit of earlier versions, not set any more */
 
 typedef struct sidco_seg_debug {
     int32_t M_used;                       /* stages used by the last call (after the cap for delta) */
@@ -148,7 +147,10 @@ int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_o
  *     (residual pointer, segment table) pair; after that they carry on from call to call.  The
  *     stage-adaptation state lives in the workspace too and
  *     belongs to the last (residual pointer, segment table) pair: calling with a different pair rebuilds
- *     the tables, resets M to 1 and synchronises `stream` once;
+ *     the tables, resets M to 1 and synchronises `stream` once (while `stream` is capturing such a call
+ *     returns SIDCO_E_CAPTURE and enqueues nothing).  The pair is recognised by the pointer's value: a
+ *     residual buffer that is freed and allocated again at the same address, used with the same segment
+ *     table, inherits the old M and counts; the only way to start over is a call with a different pair;
  *   - the first call on a device looks up the device address of the array (cudaGetSymbolAddress) and
  *     uploads tables; make that first call before any stream capture begins;
  *   - the debug, state and workspace helpers below do not see this workspace.
@@ -158,6 +160,38 @@ int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_o
 int sidco_compress_static(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs,
                           float delta, int sid_type, int max_stages,
                           int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
+
+/*
+ * sidco_aggregate - dense mean of N workers' sparse gradients.
+ *
+ * The step that follows the sparsifier in the paper's sparsified distributed synchronous SGD (appendix,
+ * algorithm box "Sparsified Distributed Synchronous SGD", line "Collective-Comm"):
+ *     G = (1/N) * sum_{n=1..N} Sparsify(g_n, delta).
+ * The exchange itself (an all-gather of every worker's out_idx / out_val / count) is done by the caller;
+ * this call turns the gathered lists, which lie in local device memory, into the dense vector.
+ *
+ * idx_all    device, int32[n_workers * stride]: worker n's indices at idx_all + n * stride, strictly
+ *            ascending, each in [0, d); entries beyond counts[n] are padding and are not read.
+ * val_all    device, float[n_workers * stride], same layout.
+ * counts     device, int32[n_workers]: entries of each worker's list (what the worker's out_k[n_segs] said).
+ * n_workers  1 .. SIDCO_AGG_MAX_WORKERS.
+ * stride     elements between consecutive workers' lists (>= every count).
+ * d          length of the dense vector, <= 2^31 - 2^16.
+ * out_dense  device, float[d], written in full: out[j] = (float)((v_1[j] + ... + v_N[j]) / N), the sum taken
+ *            in fp64 over the workers that sent position j, in worker order, and +0.0f where nobody did.
+ *            32-byte alignment gives the vectorised path.
+ * status     device, int32, optional (NULL to ignore): cleared on `stream`, then OR-ed with SIDCO_AGG_ST_COUNT
+ *            if a count lay outside [0, stride] (it is clipped) and SIDCO_AGG_ST_ORDER if an index was met
+ *            where an ascending list cannot have it (that entry is skipped; nothing is written outside
+ *            out_dense either way).
+ * stream     everything is enqueued here (one kernel, plus the 4-byte clear of `status`); no synchronisation,
+ *            no allocation.
+ */
+#define SIDCO_AGG_MAX_WORKERS 64
+#define SIDCO_AGG_ST_COUNT 1
+#define SIDCO_AGG_ST_ORDER 2
+int sidco_aggregate(const int32_t* idx_all, const float* val_all, const int32_t* counts, int n_workers,
+                    int64_t stride, int64_t d, float* out_dense, int32_t* status, void* stream);
 
 /* Bytes of device scratch one residual key needs for a vector of d elements in n_segs segments. */
 size_t sidco_workspace_bytes(int64_t d, int n_segs);
@@ -178,14 +212,17 @@ int sidco_reset_state(const float* residual);
 
 /* The same reset enqueued on `stream` (one tiny kernel, no synchronisation): for callers that restart a
  * run without stalling the stream.  The next sidco_compress for `residual` must be issued after this call
- * returns (it is the host-side bookkeeping that tells it not to read the residual). */
+ * returns; the mark that tells it not to read the residual lives in the workspace on the device and is
+ * consumed by the first compress kernel that runs after the reset kernel on `stream`. */
 int sidco_reset_state_async(const float* residual, void* stream);
 
 /* Copy per-segment thresholds, counts, stage counts and status of the last call to host memory
  * (`out` has room for n_segs entries).  Synchronises the device; meant for tests and logging. */
 int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs);
 
-/* Phase breakdown of the last call in microseconds, from device timestamps taken by the first CTA as it
+/* (Only in a build with -DSIDCO_PROFILE, see sidco_build_flags; the default build takes no device timestamps
+ * and both functions below return SIDCO_E_UNSUPPORTED.)
+ * Phase breakdown of the last call in microseconds, from device timestamps taken by the first CTA as it
  * moves from phase to phase (the other CTAs move on their own): us_out[0] error compensation + stage-1 statistics and fit, [1] stage-2 side-buffer
  * compaction and fit, [2] stages 3..M, [3] survivor staging + residual zeroing, [4] final placement and
  * adaptation, [5] whole kernel; then finer marks of that CTA alone: [6] its first sweep, [7] its arrivals
@@ -208,6 +245,24 @@ int sidco_state_load(const float* residual, const int64_t* host_blob, int n_segs
 /* Free everything the library holds for `residual` / for all keys.  Synchronises the device. */
 int sidco_release(const float* residual);
 int sidco_release_all(void);
+
+/* Switches for tests; production code has no reason to call this.
+ *   grid                  > 0: launch with at most this many CTAs (contexts created afterwards); 0: all the device
+ *                         holds.  Starts from the environment variable SIDCO_GRID, if set.
+ *   spec_enable           0: the first sweep records no candidate slots and the final selection re-reads acc in full
+ *                         (results are the same either way).  Starts from SIDCO_SPEC, if set.
+ *   spin_limit            polls after which a bounded wait inside the kernel gives up and raises SIDCO_ST_TIMEOUT;
+ *                         0 restores the default (about one second).
+ *   drop_publication_seg  >= 0: the kernel withholds the published threshold words of this segment, so that the
+ *                         CTAs waiting for them run into spin_limit (to exercise the time-out path without
+ *                         harming the device); -1: off. */
+int sidco_set_test_hooks(int grid, int spec_enable, long long spin_limit, int drop_publication_seg);
+
+/* Compile-time switches this library was built with. */
+#define SIDCO_BUILD_PROFILE      1   /* -DSIDCO_PROFILE: device timestamps at phase boundaries */
+#define SIDCO_BUILD_BOUNDS_CHECK 2   /* -DSIDCO_BOUNDS_CHECK: every index into a caller or workspace buffer is
+                                        range-checked before use; a bad one is skipped and reported in the status */
+int sidco_build_flags(void);
 
 /* Number of kernel launches the library has enqueued since it was loaded. */
 int64_t sidco_launch_count(void);

@@ -14,13 +14,16 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsidco.so")
+# SIDCO_LIB_VARIANT=profile|check selects a build of the same sources with device timestamps or with
+# device-side bounds checks (see build.py); the default is the product library.
+_VARIANT = os.environ.get("SIDCO_LIB_VARIANT", "")
+LIB_PATH = os.path.join(_HERE, "libsidco%s.so" % ("_" + _VARIANT if _VARIANT else ""))
 
 SID_EXP, SID_GAMMA, SID_GPD = 0, 1, 2
 MAX_STAGES = 8
 
 ST_NONFINITE, ST_DEGENERATE, ST_ALL_ZERO, ST_TIMEOUT = 1, 2, 4, 8
-ST_FLAGS_USED, ST_FLAGS_MISSED = 16, 32      # reserved, not set any more
+BUILD_PROFILE, BUILD_BOUNDS_CHECK = 1, 2
 
 
 class SegDebug(C.Structure):
@@ -40,7 +43,7 @@ EXPORTS = [
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
-    "sidco_reset_state_async",
+    "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate",
 ]
 
 _lib = None
@@ -101,6 +104,12 @@ def lib() -> C.CDLL:
     L.sidco_error_string.restype = C.c_char_p
     L.sidco_version.argtypes = []
     L.sidco_version.restype = i32
+    L.sidco_set_test_hooks.argtypes = [i32, i32, C.c_longlong, i32]
+    L.sidco_set_test_hooks.restype = i32
+    L.sidco_build_flags.argtypes = []
+    L.sidco_build_flags.restype = i32
+    L.sidco_aggregate.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp]
+    L.sidco_aggregate.restype = i32
     _lib = L
     return L
 
@@ -213,6 +222,31 @@ def sidco_launch_count() -> int:
 
 def sidco_version() -> int:
     return int(lib().sidco_version())
+
+
+AGG_MAX_WORKERS = 64
+AGG_ST_COUNT, AGG_ST_ORDER = 1, 2
+
+
+def sidco_aggregate(idx_all, val_all, counts, n_workers: int, stride: int, d: int, out_dense, status=None,
+                    stream=None) -> None:
+    """Dense mean of n_workers gathered sparse lists (device buffers; see sidco.h)."""
+    rc = lib().sidco_aggregate(_ptr(idx_all), _ptr(val_all), _ptr(counts), n_workers, stride, d,
+                               _ptr(out_dense), _ptr(status), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_aggregate")
+
+
+def sidco_set_test_hooks(grid: int = 0, spec_enable: int = 1, spin_limit: int = 0,
+                         drop_publication_seg: int = -1) -> None:
+    """Test switches (see sidco.h); the defaults restore normal operation."""
+    rc = lib().sidco_set_test_hooks(grid, spec_enable, spin_limit, drop_publication_seg)
+    if rc:
+        raise SidcoError(rc, "sidco_set_test_hooks")
+
+
+def sidco_build_flags() -> int:
+    return int(lib().sidco_build_flags())
 
 
 def sidco_error_string(code: int) -> str:

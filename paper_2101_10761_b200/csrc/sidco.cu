@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "../../include/sidco.h"
+#include "sidco_internal.h"
 
 namespace {
 
@@ -91,11 +92,40 @@ struct Context {
     int64_t staging_d = -1; int staging_S = -1;
 };
 
+// Switches for tests (sidco_set_test_hooks); the first two start from the environment variables SIDCO_GRID
+// (run with fewer CTAs) and SIDCO_SPEC (0: no candidate pre-selection), read once.
+struct Hooks {
+    int grid = 0;                                  // 0: every CTA the device can hold
+    int spec_enable = 1;
+    long long spin_limit = sidco::kSpinLimit;
+    int drop_pub_seg = -1;
+    bool from_env = false;
+};
+Hooks g_hooks;
+
+Hooks& hooks() {
+    if (!g_hooks.from_env) {
+        g_hooks.from_env = true;
+        if (const char* env = getenv("SIDCO_GRID")) {
+            const int want = atoi(env);
+            if (want >= 1) g_hooks.grid = want;
+        }
+        if (const char* env = getenv("SIDCO_SPEC")) g_hooks.spec_enable = env[0] == '0' ? 0 : 1;
+    }
+    return g_hooks;
+}
+
 std::mutex g_mu;
 Params g_params;
 std::unordered_map<const void*, Context*> g_ctx;
 std::unordered_map<int, DeviceInfo> g_dev;
 std::atomic<int64_t> g_launches{0};
+
+}  // namespace
+
+void sidco_internal::note_launch() { g_launches.fetch_add(1); }
+
+namespace {
 
 template <int SID>
 cudaError_t occupancy(int* out) {
@@ -119,11 +149,6 @@ cudaError_t device_info(int dev, DeviceInfo** out) {
         di.sm_count = prop.multiProcessorCount;
         di.ctas_per_sm = occ;
         di.grid = di.sm_count * occ;
-        // SIDCO_GRID=<n> runs with fewer CTAs (testing that results do not depend on the grid)
-        if (const char* env = getenv("SIDCO_GRID")) {
-            int want = atoi(env);
-            if (want >= 1 && want < di.grid) di.grid = want;
-        }
         di.ready = true;
     }
     *out = &di;
@@ -153,6 +178,73 @@ int check_args(const void* grad, const void* residual, const int64_t* off, int n
     return 0;
 }
 
+// CTAs a launch for this device uses: all that are co-resident, or fewer if a test asked for that.
+int launch_grid(const DeviceInfo& di) {
+    const int want = hooks().grid;
+    return (want >= 1 && want < di.grid) ? want : di.grid;
+}
+
+// Host copies of the tables a segment table gives rise to; the arrays are the caller's (sized for
+// max_chunks(d, S) + 1 chunks, S + 1 segments and G + 1 CTAs).
+struct HostTables {
+    int32_t* chunk_start; int32_t* chunk_seg;                  // [T + 1]
+    int32_t* seg_chunk0; int32_t* seg_n; int32_t* seg_runs;    // [S + 1]
+    int32_t* cta_chunk0;                                        // [G + 1]
+    int4* cta_desc;                                             // [G + 1]
+};
+
+// Cut the vector into chunks (at every multiple of kChunk elements and at every segment boundary), partition
+// the chunks over G CTAs as contiguous runs balanced by elements plus a per-chunk overhead, and count the runs
+// that hold chunks of each segment (the arrivals expected per statistics phase).  Returns the chunk count.
+int compute_tables(const int64_t* off, int S, int G, const HostTables& t) {
+    int T = 0;
+    for (int s = 0; s < S; ++s) {
+        t.seg_chunk0[s] = T;
+        t.seg_n[s] = (int32_t)(off[s + 1] - off[s]);
+        t.seg_runs[s] = 0;
+        int64_t at = off[s];
+        while (at < off[s + 1]) {
+            int64_t end = (at / kChunk + 1) * kChunk;
+            if (end > off[s + 1]) end = off[s + 1];
+            t.chunk_start[T] = (int32_t)at;
+            t.chunk_seg[T] = s;
+            ++T;
+            at = end;
+        }
+    }
+    t.seg_chunk0[S] = T;
+    t.seg_n[S] = 0;
+    t.seg_runs[S] = 0;
+    t.chunk_start[T] = (int32_t)off[S];
+    t.chunk_seg[T] = 0;
+    const double per_chunk = 128.0;
+    double total = 0.0;
+    for (int q = 0; q < T; ++q) total += (t.chunk_start[q + 1] - t.chunk_start[q]) + per_chunk;
+    double acc = 0.0;
+    int cta = 0;
+    t.cta_chunk0[0] = 0;
+    for (int q = 0; q < T; ++q) {
+        // chunk q goes to the CTA whose share contains the chunk's midpoint
+        const double w = (t.chunk_start[q + 1] - t.chunk_start[q]) + per_chunk;
+        int want = (int)((acc + 0.5 * w) / total * G);
+        if (want > G - 1) want = G - 1;
+        while (cta < want) t.cta_chunk0[++cta] = q;
+        acc += w;
+    }
+    while (cta < G) t.cta_chunk0[++cta] = T;
+    // per-CTA descriptor {first chunk, end chunk, first segment, number of segments spanned}
+    for (int g = 0; g < G; ++g) {
+        int prev = -1;
+        for (int q = t.cta_chunk0[g]; q < t.cta_chunk0[g + 1]; ++q)
+            if (t.chunk_seg[q] != prev) { prev = t.chunk_seg[q]; ++t.seg_runs[prev]; }
+        const int a = t.cta_chunk0[g], b = t.cta_chunk0[g + 1];
+        t.cta_desc[g] = a < b ? make_int4(a, b, t.chunk_seg[a], t.chunk_seg[b - 1] - t.chunk_seg[a] + 1)
+                              : make_int4(a, a, 0, 0);
+    }
+    t.cta_desc[G] = make_int4(T, T, 0, 0);
+    return T;
+}
+
 // Build the chunk tables for a segment table and upload them together with fresh per-segment state.
 // The adaptation state of an existing context survives a table rebuild when the segment count is unchanged.
 cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t stream) {
@@ -160,57 +252,15 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     DeviceInfo* di = nullptr;
     cudaError_t e = device_info(c->device, &di);
     if (e != cudaSuccess) return e;
-    const int G = di->grid;
+    const int G = launch_grid(*di);
 
-    std::vector<int32_t> chunk_start, chunk_seg, seg_chunk0(S + 1), seg_n(S + 1, 0), seg_runs(S + 1, 0);
-    for (int s = 0; s < S; ++s) {
-        seg_chunk0[s] = (int32_t)chunk_start.size();
-        seg_n[s] = (int32_t)(off[s + 1] - off[s]);
-        int64_t at = off[s];
-        while (at < off[s + 1]) {
-            int64_t end = (at / kChunk + 1) * kChunk;
-            if (end > off[s + 1]) end = off[s + 1];
-            chunk_start.push_back((int32_t)at);
-            chunk_seg.push_back(s);
-            at = end;
-        }
-    }
-    const int T = (int)chunk_start.size();
-    seg_chunk0[S] = T;
-    chunk_start.push_back((int32_t)d);
-    chunk_seg.push_back(0);
-
-    // Static partition of the chunks over the CTAs (contiguous runs), balanced by elements plus a
-    // per-chunk overhead.
-    std::vector<int32_t> cta_chunk0(G + 1, T);
-    {
-        const double per_chunk = 128.0;
-        double total = 0.0;
-        for (int t = 0; t < T; ++t) total += (chunk_start[t + 1] - chunk_start[t]) + per_chunk;
-        double acc = 0.0;
-        int cta = 0;
-        cta_chunk0[0] = 0;
-        for (int t = 0; t < T; ++t) {
-            // chunk t goes to the CTA whose share contains the chunk's midpoint
-            const double w = (chunk_start[t + 1] - chunk_start[t]) + per_chunk;
-            const double mid = acc + 0.5 * w;
-            int want = (int)(mid / total * G);
-            if (want > G - 1) want = G - 1;
-            while (cta < want) cta_chunk0[++cta] = t;
-            acc += w;
-        }
-        while (cta < G) cta_chunk0[++cta] = T;
-    }
-    // number of CTA runs that hold chunks of each segment (arrivals expected per statistics phase),
-    // and the per-CTA descriptor {first chunk, end chunk, first segment, number of segments spanned}
-    std::vector<int4> cta_desc(G + 1, make_int4(T, T, 0, 0));
-    for (int g = 0; g < G; ++g) {
-        int prev = -1;
-        for (int t = cta_chunk0[g]; t < cta_chunk0[g + 1]; ++t)
-            if (chunk_seg[t] != prev) { prev = chunk_seg[t]; ++seg_runs[prev]; }
-        const int a = cta_chunk0[g], b = cta_chunk0[g + 1];
-        cta_desc[g] = a < b ? make_int4(a, b, chunk_seg[a], chunk_seg[b - 1] - chunk_seg[a] + 1) : make_int4(a, a, 0, 0);
-    }
+    const size_t cap = (size_t)max_chunks(d, S) + 1;
+    std::vector<int32_t> chunk_start(cap), chunk_seg(cap), seg_chunk0(S + 1), seg_n(S + 1), seg_runs(S + 1),
+        cta_chunk0(G + 1);
+    std::vector<int4> cta_desc(G + 1);
+    const int T = compute_tables(off, S, G, HostTables{chunk_start.data(), chunk_seg.data(), seg_chunk0.data(),
+                                                       seg_n.data(), seg_runs.data(), cta_chunk0.data(),
+                                                       cta_desc.data()});
 
     const Layout L = make_layout(d, S, T, G);
     if (c->ws && c->ws_bytes < L.total) {
@@ -226,6 +276,17 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
         fresh = true;
     }
     const bool same_segments = c->tables_valid && c->S == S;
+    // A reset that no call has consumed yet ("the residual is empty") outlives the rebuild.
+    Control ctl_host;
+    std::memset(&ctl_host, 0, sizeof(Control));
+    if (c->tables_valid && !fresh) {
+        Control old;
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return e;
+        if ((e = cudaMemcpy(&old, (char*)c->ws + c->L.ctl, sizeof(Control), cudaMemcpyDeviceToHost)) != cudaSuccess)
+            return e;
+        ctl_host.residual_is_zero = old.residual_is_zero;
+    }
+    c->tables_valid = false;               // until the uploads below have succeeded
     // keep adaptation state across a table rebuild only when the segment count is unchanged
     std::vector<SegDev> seg_host(S + 1);
     if (same_segments && !fresh) {
@@ -252,7 +313,7 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.seg_runs, seg_runs.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
-    if ((e = cudaMemset(base + L.ctl, 0, sizeof(Control))) != cudaSuccess) return e;
+    if ((e = up(L.ctl, &ctl_host, sizeof(Control))) != cudaSuccess) return e;
     // (the call numbering restarts: no run's published count may carry a number of the old numbering)
     if ((e = cudaMemset(base + L.cta_total, 0, sizeof(unsigned long long) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
@@ -283,21 +344,11 @@ cudaError_t launch_persistent(const void* fn, int grid, void** kargs, cudaStream
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), kargs, 0, stream);
 }
 
-int compress_impl(Context* c, const float* grad, float* residual, const int64_t* off, int S, float delta, int sid,
-                  int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
-                  const Params& prm) {
-    cudaError_t e;
-    const bool same = c->tables_valid && c->S == S &&
-                      std::memcmp(c->offsets.data(), off, sizeof(int64_t) * (S + 1)) == 0;
-    if (!same) {
-        // allocation, uploads and a stream synchronisation: not something a capturing stream can record
-        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-        if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return (int)e;
-        if (cap != cudaStreamCaptureStatusNone) return SIDCO_E_CAPTURE;
-        if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
-    }
-    char* base = (char*)c->ws;
-    const Layout& L = c->L;
+// Fill the kernel's argument block for a workspace at `base` laid out as `L` and enqueue the persistent kernel.
+// Used by every entry point, so that they cannot drift apart.
+int launch_compress(char* base, const Layout& L, int T, int S, int G, const float* grad, float* residual, float delta,
+                    int sid, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
+                    const Params& prm) {
     Args a{};
     a.grad = grad;
     a.residual = residual;
@@ -332,22 +383,40 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
     a.Q = prm.Q;
     a.sid = sid;
     a.max_stages = max_stages;
-    a.C = c->T;
-    a.S = c->S;
-    a.G = c->G;
+    a.C = T;
+    a.S = S;
+    a.G = G;
     a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
-    // SIDCO_SPEC=0 switches the candidate pre-selection off (the result is the same either way)
-    static const bool spec_on = [] { const char* e = getenv("SIDCO_SPEC"); return !(e && e[0] == '0'); }();
-    a.spec_enable = spec_on ? 1 : 0;
+    const Hooks& h = hooks();
+    a.spec_enable = h.spec_enable;           // (the result is the same with or without the pre-selection)
+    a.spin_limit = h.spin_limit;
+    a.drop_pub_seg = h.drop_pub_seg;
 
     void* kargs[] = {(void*)&a};
     const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
                      : sid == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
-    e = launch_persistent(fn, c->G, kargs, stream);
+    const cudaError_t e = launch_persistent(fn, G, kargs, stream);
     if (e != cudaSuccess) return (int)e;
     g_launches.fetch_add(1);
     return 0;
+}
+
+int compress_impl(Context* c, const float* grad, float* residual, const int64_t* off, int S, float delta, int sid,
+                  int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
+                  const Params& prm) {
+    cudaError_t e;
+    const bool same = c->tables_valid && c->S == S &&
+                      std::memcmp(c->offsets.data(), off, sizeof(int64_t) * (S + 1)) == 0;
+    if (!same) {
+        // allocation, uploads and a stream synchronisation: not something a capturing stream can record
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return (int)e;
+        if (cap != cudaStreamCaptureStatusNone) return SIDCO_E_CAPTURE;
+        if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
+    }
+    return launch_compress((char*)c->ws, c->L, c->T, c->S, c->G, grad, residual, delta, sid, max_stages, out_idx,
+                           out_val, out_k, stream, prm);
 }
 
 Context* find_or_create(const void* key, int dev) {
@@ -416,56 +485,6 @@ struct StaticContext {
 constexpr int kMaxDevices = 64;
 StaticContext g_static[kMaxDevices];
 
-// Same tables as build_tables(), written into the fixed host arrays of the static context.
-void fill_static_tables(StaticContext& c, const int64_t* off, int S, int G) {
-    int T = 0;
-    for (int s = 0; s < S; ++s) {
-        c.seg_chunk0[s] = T;
-        c.seg_n[s] = (int32_t)(off[s + 1] - off[s]);
-        c.seg_runs[s] = 0;
-        int64_t at = off[s];
-        while (at < off[s + 1]) {
-            int64_t end = (at / kChunk + 1) * kChunk;
-            if (end > off[s + 1]) end = off[s + 1];
-            c.chunk_start[T] = (int32_t)at;
-            c.chunk_seg[T] = s;
-            ++T;
-            at = end;
-        }
-    }
-    c.seg_chunk0[S] = T;
-    c.seg_n[S] = 0;
-    c.seg_runs[S] = 0;
-    c.chunk_start[T] = (int32_t)off[S];
-    c.chunk_seg[T] = 0;
-    const double per_chunk = 128.0;
-    double total = 0.0;
-    for (int t = 0; t < T; ++t) total += (c.chunk_start[t + 1] - c.chunk_start[t]) + per_chunk;
-    double acc = 0.0;
-    int cta = 0;
-    c.cta_chunk0[0] = 0;
-    for (int t = 0; t < T; ++t) {
-        const double w = (c.chunk_start[t + 1] - c.chunk_start[t]) + per_chunk;
-        int want = (int)((acc + 0.5 * w) / total * G);
-        if (want > G - 1) want = G - 1;
-        while (cta < want) c.cta_chunk0[++cta] = t;
-        acc += w;
-    }
-    while (cta < G) c.cta_chunk0[++cta] = T;
-    for (int g = 0; g < G; ++g) {
-        int prev = -1;
-        for (int t = c.cta_chunk0[g]; t < c.cta_chunk0[g + 1]; ++t)
-            if (c.chunk_seg[t] != prev) { prev = c.chunk_seg[t]; ++c.seg_runs[prev]; }
-        const int a = c.cta_chunk0[g], b = c.cta_chunk0[g + 1];
-        c.cta_desc[g] = a < b ? make_int4(a, b, c.chunk_seg[a], c.chunk_seg[b - 1] - c.chunk_seg[a] + 1)
-                              : make_int4(a, a, 0, 0);
-    }
-    c.T = T;
-    c.S = S;
-    c.G = G;
-    for (int s = 0; s <= S; ++s) c.offsets[s] = off[s];
-}
-
 }  // namespace
 
 extern "C" {
@@ -497,8 +516,21 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
     const bool same = c.tables_valid && c.key == residual && c.S == n_segs &&
                       std::memcmp(c.offsets, seg_offsets, sizeof(int64_t) * (n_segs + 1)) == 0;
     if (!same) {
-        // New residual or segment table: rebuild the tables and start the adaptation state afresh.
-        fill_static_tables(c, seg_offsets, n_segs, di->grid);
+        // New residual or segment table: rebuild the tables and start the adaptation state afresh.  The uploads
+        // and the synchronisation below are not something a capturing stream can record.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if ((e = cudaStreamIsCapturing(stream, &cap)) != cudaSuccess) return (int)e;
+        if (cap != cudaStreamCaptureStatusNone) return SIDCO_E_CAPTURE;
+        // From here until the last upload has completed the context describes no usable tables.
+        c.tables_valid = false;
+        c.key = nullptr;
+        const int G = launch_grid(*di);
+        if (G > kMaxGrid) return SIDCO_E_SIZE;
+        c.T = compute_tables(seg_offsets, n_segs, G, HostTables{c.chunk_start, c.chunk_seg, c.seg_chunk0, c.seg_n,
+                                                                c.seg_runs, c.cta_chunk0, c.cta_desc});
+        c.S = n_segs;
+        c.G = G;
+        for (int s = 0; s <= n_segs; ++s) c.offsets[s] = seg_offsets[s];
         c.L = make_layout(d, n_segs, c.T, c.G);
         if (c.L.total > kStaticBytes) return SIDCO_E_SIZE;
         for (int s = 0; s <= n_segs; ++s) {
@@ -516,67 +548,22 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = up(L.seg_runs, c.seg_runs, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.cta_desc, c.cta_desc, sizeof(int4) * (c.G + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        // The array keeps whatever the last call left.  What must start at zero (the control block: finished-CTA
+        // count, call number, time-out flag; the published run counts; the per-chunk counts) is cleared here,
+        // when this residual and segment table are first seen; from then on it is state that is meant to
+        // persist, and everything else is rewritten before it is read.
         if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.cta_total, 0, sizeof(unsigned long long) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.side_cnt, 0, sizeof(int32_t) * (c.T + 1), stream)) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.chunk_cnt, 0, sizeof(int32_t) * (c.T + 1), stream)) != cudaSuccess) return (int)e;
         // the uploads read the fixed host arrays: let them finish before those can change again
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;
         c.key = residual;
         c.tables_valid = true;
     }
-    const Layout& L = c.L;
-    // The array keeps whatever the last call left.  What must start at zero (the control block: barrier
-    // arrivals, call number, time-out flag; and the segment records) was cleared with the upload above, when
-    // this residual and segment table were first seen; from then on it is state that is meant to persist,
-    // and everything else is rewritten before it is read.
-    unsigned char* base = c.base;
-    Args a{};
-    a.grad = grad;
-    a.residual = residual;
-    a.out_idx = out_idx;
-    a.out_val = out_val;
-    a.out_k = out_k;
-    a.chunk_start = (const int32_t*)(base + L.chunk_start);
-    a.chunk_seg = (const int32_t*)(base + L.chunk_seg);
-    a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
-    a.seg_n = (const int32_t*)(base + L.seg_n);
-    a.seg_runs = (const int32_t*)(base + L.seg_runs);
-    a.cta_desc = (const int4*)(base + L.cta_desc);
-    a.part = (double*)(base + L.part);
-    a.part_n = (int32_t*)(base + L.part_n);
-    a.side_cnt = (int32_t*)(base + L.side_cnt);
-    a.chunk_cnt = (int32_t*)(base + L.chunk_cnt);
-    a.side_idx = (int32_t*)(base + L.side_idx);
-    a.side_val = (float*)(base + L.side_val);
-    a.stage_idx = (int32_t*)(base + L.stage_idx);
-    a.stage_val = (float*)(base + L.stage_val);
-    a.cta_pub = (unsigned long long*)(base + L.cta_total);
-    a.cand = base + L.cand;
-    a.cta_dir = (int32_t*)(base + L.cta_dir);
-    a.cta_ns = (unsigned long long*)(base + L.cta_ns);
-    a.seg = (SegDev*)(base + L.seg);
-    a.ctl = (Control*)(base + L.ctl);
-    a.delta = (double)delta;
-    a.delta1 = g_params.delta1;
-    fill_ln_tables(a, (double)delta, g_params.delta1);
-    a.eps_H = g_params.eps_H;
-    a.eps_L = g_params.eps_L;
-    a.Q = g_params.Q;
-    a.sid = sid_type;
-    a.max_stages = max_stages;
-    a.C = c.T;
-    a.S = c.S;
-    a.G = c.G;
-    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
-    a.spec_enable = 1;
-    void* kargs[] = {(void*)&a};
-    const void* fn = sid_type == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
-                     : sid_type == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
-                                     : (const void*)sidco::sidco_persistent_kernel<2>;
-    e = launch_persistent(fn, c.G, kargs, stream);
-    if (e != cudaSuccess) return (int)e;
-    g_launches.fetch_add(1);
-    return 0;
+    return launch_compress((char*)c.base, c.L, c.T, c.S, c.G, grad, residual, delta, sid_type, max_stages, out_idx,
+                           out_val, out_k, stream, g_params);
 }
 
 int sidco_compress_host(const float* grad, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
@@ -726,6 +713,10 @@ int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs) {
 }
 
 int sidco_get_phase_times(const float* residual, double* us_out) {
+#ifndef SIDCO_PROFILE
+    (void)residual; (void)us_out;
+    return SIDCO_E_UNSUPPORTED;
+#else
     if (!us_out) return SIDCO_E_NULL;
     std::lock_guard<std::mutex> lock(g_mu);
     auto it = g_ctx.find(residual);
@@ -744,11 +735,16 @@ int sidco_get_phase_times(const float* residual, double* us_out) {
     us_out[8] = us(1, 8);      // stage-2 sweep of CTA 0 alone (meaningless if no segment used M >= 2)
     us_out[9] = us(8, 9);
     us_out[10] = us(10, 11);   // arrivals and fits of the last refit stage
-    us_out[11] = us(4, 12) < 0 ? us(3, 12) : us(3, 12);   // survivor staging sweep of CTA 0 alone
+    us_out[11] = us(3, 12);    // survivor staging sweep of CTA 0 alone
     return 0;
+#endif
 }
 
 int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_ctas) {
+#ifndef SIDCO_PROFILE
+    (void)residual; (void)us_out; (void)max_ctas;
+    return SIDCO_E_UNSUPPORTED;
+#else
     if (!us_out) return SIDCO_E_NULL;
     std::lock_guard<std::mutex> lock(g_mu);
     auto it = g_ctx.find(residual);
@@ -765,6 +761,29 @@ int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_cta
     const int n = c->G < max_ctas ? c->G : max_ctas;
     for (int i = 0; i < 4 * n; ++i) us_out[i] = (double)(long long)(ns[i] - ctl.t_ns[0]) * 1e-3;
     return n;
+#endif
+}
+
+int sidco_set_test_hooks(int grid, int spec_enable, long long spin_limit, int drop_publication_seg) {
+    if (grid < 0 || spin_limit < 0) return SIDCO_E_PARAMS;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Hooks& h = hooks();
+    h.grid = grid;
+    h.spec_enable = spec_enable ? 1 : 0;
+    h.spin_limit = spin_limit ? spin_limit : sidco::kSpinLimit;
+    h.drop_pub_seg = drop_publication_seg;
+    return 0;
+}
+
+int sidco_build_flags(void) {
+    int f = 0;
+#ifdef SIDCO_PROFILE
+    f |= SIDCO_BUILD_PROFILE;
+#endif
+#ifdef SIDCO_BOUNDS_CHECK
+    f |= SIDCO_BUILD_BOUNDS_CHECK;
+#endif
+    return f;
 }
 
 int sidco_state_save(const float* residual, int64_t* blob, int n_segs) {
@@ -844,12 +863,13 @@ const char* sidco_error_string(int code) {
         case SIDCO_E_SIZE: return "size beyond the limit of this entry point";
         case SIDCO_E_CAPTURE:
             return "first call for this residual and segment table must be made before stream capture begins";
+        case SIDCO_E_UNSUPPORTED: return "not available in this build of the library";
         default: break;
     }
     if (code > 0) return cudaGetErrorString((cudaError_t)code);
     return "unknown error";
 }
 
-int sidco_version(void) { return 100; }
+int sidco_version(void) { return 200; }
 
 }  // extern "C"

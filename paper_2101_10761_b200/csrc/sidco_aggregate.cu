@@ -1,0 +1,239 @@
+// Aggregation of N workers' sparse gradients into the dense mean (the collective step of the paper's
+// sparsified distributed synchronous SGD: G = (1/N) * sum_n Sparsify(g_n, delta)), for sm_100a.
+//
+// The lists have been gathered into local memory already (padded to a common stride); this kernel turns
+// them into the dense vector.  Almost all of the output is zeros, so the kernel is a store stream with a
+// sparse correction: every CTA owns a contiguous range of the output; a few of its warps locate the range in
+// each worker's ascending index list (warp-wide 32-ary search) and copy those entries into shared memory
+// while the other warps already write zeros over the range with 32-byte stores; after one CTA barrier the
+// entries are put in place.  A position that several workers sent is written once, by the entry of the first
+// worker that has it: that thread looks the position up in the later workers' lists (binary search in shared
+// memory) and adds their values in worker order in fp64, so the result does not depend on scheduling.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "../../include/sidco.h"
+#include "sidco_internal.h"
+
+namespace sidco_agg {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxWorkers = SIDCO_AGG_MAX_WORKERS;
+constexpr int kSmemEntries = 11264;            // (index, value) pairs of one CTA range kept in shared memory: 88 KB
+constexpr unsigned kFull = 0xffffffffu;
+
+struct Args {
+    const int32_t* idx_all;      // [n_workers][stride]
+    const float* val_all;        // [n_workers][stride]
+    const int32_t* counts;       // [n_workers]
+    float* out;                  // [d]
+    int32_t* status;             // optional
+    long long stride, d;
+    long long per_cta;           // elements per CTA range (a multiple of 8)
+    int n_workers;
+    int vec_ok;                  // out is 32-byte aligned
+};
+
+// First position in [a, b) of the ascending list whose index is >= target (b if none), found by the whole
+// warp: 32 probes per round.
+__device__ __forceinline__ long long warp_lower_bound(const int32_t* __restrict__ list, long long a, long long b,
+                                                      long long target) {
+    const int lane = threadIdx.x & 31;
+    while (b - a > 32) {
+        const long long step = (b - a + 31) / 32;
+        const long long p = a + lane * step;
+        const bool less = p < b && (long long)__ldg(list + p) < target;
+        const int m = __popc(__ballot_sync(kFull, less));          // probes below the target: a prefix of the lanes
+        if (m == 0) { b = a; break; }
+        const long long na = a + (long long)(m - 1) * step + 1;
+        const long long nb = a + (long long)m * step;
+        a = na;
+        b = nb < b ? nb : b;
+    }
+    const bool less = a + lane < b && (long long)__ldg(list + a + lane) < target;
+    return a + __popc(__ballot_sync(kFull, less));
+}
+
+// Position of `target` in the ascending list [0, n), or -1.
+template <class Ptr>
+__device__ __forceinline__ int find_index(Ptr list, int n, int target) {
+    int a = 0, b = n;
+    while (a < b) {
+        const int mid = (a + b) >> 1;
+        if (list[mid] < target) a = mid + 1; else b = mid;
+    }
+    return (a < n && list[a] == target) ? a : -1;
+}
+
+__global__ void __launch_bounds__(kThreads, 2) sidco_aggregate_kernel(const __grid_constant__ Args A) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw);
+    float* s_val = reinterpret_cast<float*>(smem_raw + sizeof(int32_t) * kSmemEntries);
+    __shared__ long long s_begin[kMaxWorkers];       // first entry of the range in worker w's list
+    __shared__ int s_cnt[kMaxWorkers];               // entries of the range in worker w's list
+    __shared__ int s_off[kMaxWorkers + 1];           // prefix sums of s_cnt
+    __shared__ int s_flags;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long lo = (long long)blockIdx.x * A.per_cta;
+    long long hi = lo + A.per_cta;
+    if (hi > A.d) hi = A.d;
+    if (lo >= hi) return;
+    if (threadIdx.x == 0) s_flags = 0;
+    __syncthreads();
+    const int N = A.n_workers;
+
+    // ---- where the range lies in every worker's list (warps take workers in turn)
+    for (int w = warp; w < N; w += kWarps) {
+        long long cnt = __ldg(A.counts + w);
+        int flag = 0;
+        if (cnt < 0) { cnt = 0; flag = SIDCO_AGG_ST_COUNT; }
+        if (cnt > A.stride) { cnt = A.stride; flag = SIDCO_AGG_ST_COUNT; }
+        const int32_t* list = A.idx_all + (long long)w * A.stride;
+        const long long b = warp_lower_bound(list, 0, cnt, lo);
+        const long long e = warp_lower_bound(list, b, cnt, hi);
+        if (lane == 0) {
+            s_begin[w] = b;
+            s_cnt[w] = (int)(e - b);
+            if (flag) atomicOr(&s_flags, flag);
+        }
+    }
+
+    // ---- zeros over the range
+    {
+        float* out = A.out;
+        if (A.vec_ok) {
+            // lo is a multiple of 8 and out is 32-byte aligned: whole 32-byte stores up to the last multiple of 8
+            const long long n_vec = (hi - lo) >> 3;
+            float4* o4 = reinterpret_cast<float4*>(out + lo);
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (long long v = threadIdx.x; v < n_vec; v += kThreads) {
+                o4[2 * v] = z;
+                o4[2 * v + 1] = z;
+            }
+            for (long long i = lo + (n_vec << 3) + threadIdx.x; i < hi; i += kThreads) out[i] = 0.0f;
+        } else {
+            for (long long i = lo + threadIdx.x; i < hi; i += kThreads) out[i] = 0.0f;
+        }
+    }
+    __syncthreads();      // the searches are done, and every zero of this range is ordered before the values below
+
+    if (threadIdx.x == 0) {
+        int o = 0;
+        for (int w = 0; w < N; ++w) { s_off[w] = o; o += s_cnt[w]; }
+        s_off[N] = o;
+    }
+    __syncthreads();
+    const int E = s_off[N];
+    if (E == 0) {
+        if (threadIdx.x == 0 && s_flags && A.status) atomicOr(A.status, s_flags);
+        return;
+    }
+    const bool in_smem = E <= kSmemEntries;
+    if (in_smem) {
+        for (int w = 0; w < N; ++w) {
+            const int32_t* gi = A.idx_all + (long long)w * A.stride + s_begin[w];
+            const float* gv = A.val_all + (long long)w * A.stride + s_begin[w];
+            for (int i = threadIdx.x; i < s_cnt[w]; i += kThreads) {
+                s_idx[s_off[w] + i] = __ldg(gi + i);
+                s_val[s_off[w] + i] = __ldg(gv + i);
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- the sparse correction: one thread per entry; the first worker that has a position writes it
+    const double inv_scale = (double)N;
+    int bad = 0;
+    for (int f = threadIdx.x; f < E; f += kThreads) {
+        int w = 0;
+        while (f >= s_off[w + 1]) ++w;
+        const int i = f - s_off[w];
+        int idx;
+        float val;
+        if (in_smem) { idx = s_idx[f]; val = s_val[f]; }
+        else {
+            idx = __ldg(A.idx_all + (long long)w * A.stride + s_begin[w] + i);
+            val = __ldg(A.val_all + (long long)w * A.stride + s_begin[w] + i);
+        }
+        if (idx < lo || idx >= hi) { bad = 1; continue; }          // a list that is not ascending: skip, report
+        bool owner = true;
+        for (int u = 0; u < w && owner; ++u) {
+            const int hit = in_smem ? find_index(s_idx + s_off[u], s_cnt[u], idx)
+                                    : find_index(A.idx_all + (long long)u * A.stride + s_begin[u], s_cnt[u], idx);
+            owner = hit < 0;
+        }
+        if (!owner) continue;
+        double sum = 0.0 + (double)val;
+        for (int u = w + 1; u < N; ++u) {
+            if (in_smem) {
+                const int hit = find_index(s_idx + s_off[u], s_cnt[u], idx);
+                if (hit >= 0) sum += (double)s_val[s_off[u] + hit];
+            } else {
+                const int32_t* gi = A.idx_all + (long long)u * A.stride + s_begin[u];
+                const int hit = find_index(gi, s_cnt[u], idx);
+                if (hit >= 0) sum += (double)__ldg(A.val_all + (long long)u * A.stride + s_begin[u] + hit);
+            }
+        }
+        A.out[idx] = (float)(sum / inv_scale);
+    }
+    if (bad) atomicOr(&s_flags, SIDCO_AGG_ST_ORDER);
+    __syncthreads();
+    if (threadIdx.x == 0 && s_flags && A.status) atomicOr(A.status, s_flags);
+}
+
+}  // namespace sidco_agg
+
+extern "C" {
+
+int sidco_aggregate(const int32_t* idx_all, const float* val_all, const int32_t* counts, int n_workers,
+                    int64_t stride, int64_t d, float* out_dense, int32_t* status, void* stream_v) {
+    if (!idx_all || !val_all || !counts || !out_dense) return SIDCO_E_NULL;
+    if (n_workers < 1 || n_workers > SIDCO_AGG_MAX_WORKERS) return SIDCO_E_PARAMS;
+    if (stride < 0 || d < 0 || d > (int64_t)2147483647 - 65536) return SIDCO_E_SIZE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    cudaError_t e;
+    if (status && (e = cudaMemsetAsync(status, 0, sizeof(int32_t), stream)) != cudaSuccess) return (int)e;
+    if (d == 0) return 0;
+    static int sm_count[64] = {0};
+    static std::mutex mu;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= 64) return SIDCO_E_SIZE;
+    std::lock_guard<std::mutex> lock(mu);
+    const size_t smem = (sizeof(int32_t) + sizeof(float)) * sidco_agg::kSmemEntries;
+    if (!sm_count[dev]) {
+        int n = 0;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return (int)e;
+        if ((e = cudaFuncSetAttribute(sidco_agg::sidco_aggregate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)smem)) != cudaSuccess)
+            return (int)e;
+        sm_count[dev] = n;
+    }
+    sidco_agg::Args a{};
+    a.idx_all = idx_all;
+    a.val_all = val_all;
+    a.counts = counts;
+    a.out = out_dense;
+    a.status = status;
+    a.stride = stride;
+    a.d = d;
+    a.n_workers = n_workers;
+    a.vec_ok = (((uintptr_t)out_dense) & 31u) == 0;
+    // two CTAs per SM; ranges are multiples of 256 elements, and no smaller than 4096
+    long long grid = 2ll * sm_count[dev];
+    long long per = (d + grid - 1) / grid;
+    if (per < 4096) per = 4096;
+    per = (per + 255) / 256 * 256;
+    grid = (d + per - 1) / per;
+    a.per_cta = per;
+    sidco_agg::sidco_aggregate_kernel<<<(unsigned)grid, sidco_agg::kThreads, smem, stream>>>(a);
+    if ((e = cudaGetLastError()) != cudaSuccess) return (int)e;
+    sidco_internal::note_launch();
+    return 0;
+}
+
+}  // extern "C"

@@ -48,6 +48,14 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Device timestamps at phase boundaries (sidco_get_phase_times, sidco_get_cta_sweep_times) exist only in a
+// build with -DSIDCO_PROFILE; the default build carries none of them.
+#ifdef SIDCO_PROFILE
+#define SIDCO_STAMP(...) do { __VA_ARGS__; } while (0)
+#else
+#define SIDCO_STAMP(...) do { } while (0)
+#endif
+
 namespace sidco {
 
 constexpr int kThreads = 1024;
@@ -64,7 +72,7 @@ constexpr int kCoopItems = 4096;                  // flagged slots one pass can 
 constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
-constexpr long long kSpinLimit = 1ll << 22;       // bounded waits: ~1 s with the back-off below
+constexpr long long kSpinLimit = 1ll << 22;       // default bound of the waits: ~1 s with the back-off below
 static_assert(kWarps == 32, "block_tree and the scans assume 32 warps per CTA");
 
 enum { kSidExp = 0, kSidGamma = 1, kSidGpd = 2 };
@@ -145,6 +153,9 @@ struct Args {
     int C, S, G;
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
+    long long spin_limit;        // polls after which a bounded wait gives up (kSpinLimit unless a test shortens it)
+    int drop_pub_seg;            // test hook: the published words of this segment are withheld (-1: none), so that
+                                 // the runs waiting for them run into the bound
 };
 
 // ----------------------------------------------------------------------------
@@ -213,7 +224,7 @@ __device__ __forceinline__ float wait_ready_thread(const Args& A, unsigned call_
         // (the time-out flag is looked at now and then only: a second dependent load in every round would
         // double the time it takes to notice the word)
         if ((++spins & 15) == 0 && ld_volatile(&A.ctl->timeout)) break;
-        if (spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+        if (spins > A.spin_limit) { atomicExch(&A.ctl->timeout, 1); break; }
         __nanosleep(spins < 16 ? 20 : 100);
     }
     return __uint_as_float((unsigned)(w >> 32));
@@ -427,11 +438,13 @@ __device__ __forceinline__ void record_stage(SegDev* sg, int stage, const Fit& f
 // stored afterwards (record_stage).  If another stage follows, its sweep shifts by eta, which is therefore
 // stored before the word and released with it.  The word of a last stage carries all that its readers need
 // (they go on to read only their own run's data), so it is a plain strong store with no fence to wait for.
-__device__ inline Fit publish_stage(unsigned call_id, SegDev* sg, int stages, bool last, double eta) {
+__device__ inline Fit publish_stage(const Args& A, unsigned call_id, SegDev* sg, int stages, bool last, double eta) {
     Fit f{eta, last ? __double2float_ru(eta) : __double2float_rd(eta), stages, last, 0, 0, 0, false};
     const unsigned long long word = ((unsigned long long)__float_as_uint(f.thr) << 32) |
                                     (unsigned long long)(call_id * 16u + (unsigned)stages);
-    if (last) {
+    if (A.drop_pub_seg >= 0 && sg == A.seg + A.drop_pub_seg) {
+        // (test hook: nothing is published)
+    } else if (last) {
         st_relaxed_u64(&sg->pub, word);
     } else {
         sg->eta[stages - 1] = eta;
@@ -486,7 +499,7 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
         }
     }
     // an empty segment takes part in no later phase: all its stages count as fitted here
-    Fit f = publish_stage(T.call_id, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
+    Fit f = publish_stage(A, T.call_id, sg, n == 0 ? M_eff : 1, n == 0 || M_eff == 1, eta);
     f.M_eff = M_eff;
     f.status = status;
     f.empty = n == 0;
@@ -507,7 +520,7 @@ __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, d
         else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, T.ln[slot], T.ln_inv[slot], status);
         eta = prev + inc;
     }
-    Fit f = publish_stage(T.call_id, sg, m + 1, m + 1 == M_eff, eta);
+    Fit f = publish_stage(A, T.call_id, sg, m + 1, m + 1 == M_eff, eta);
     f.M_eff = M_eff;
     f.status = status;
     f.n_e = n_e;
@@ -771,7 +784,7 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
         v.M_eff = R.m_eff[i];
         long long spins = 0;
         while (R.ok[i] != tag) {                       // published by a thread of this CTA
-            if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+            if (++spins > A.spin_limit) { atomicExch(&A.ctl->timeout, 1); break; }
             __nanosleep(20);
         }
         __threadfence_block();
@@ -800,11 +813,11 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                                                int stamp_slot) {
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) {                                   // this CTA's sweep is over
+    SIDCO_STAMP(if (threadIdx.x == 0) {                       // this CTA's sweep is over
         const unsigned long long now = global_ns();
         A.cta_ns[4 * blockIdx.x + (stage < 2 ? stage : 2)] = now;
         if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
-    }
+    });
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // one warp: its first lane fits segment i2 of the run from its sums (M_state and r are that lane's),
     // publishes, and fills the CTA's own cache entry; all lanes then write the stage's record
@@ -931,8 +944,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     const int first_chunk = warp < c1 - c0 ? (p1_desc ? c1 - 1 - warp : c0 + warp) : -1;
     const Desc first_desc = fetch_desc(A, first_chunk, false);
     const int cap = stage_cap(A.delta, A.delta1);
-    const bool stamper = (cta == 0 && threadIdx.x == 0);
-    if (stamper) A.ctl->t_ns[0] = global_ns();
+    [[maybe_unused]] const bool stamper = (cta == 0 && threadIdx.x == 0);
+    SIDCO_STAMP(if (stamper) A.ctl->t_ns[0] = global_ns());
     if (threadIdx.x == 0) sm_mloc = 1;
     if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
@@ -1102,7 +1115,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     if (threadIdx.x == 0) sm_next = 0;
     __syncthreads();
     const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
-    if (stamper) A.ctl->t_ns[7] = A.ctl->t_ns[1] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
+    SIDCO_STAMP(if (stamper) A.ctl->t_ns[7] = A.ctl->t_ns[1] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns());
 
     // ------------------------------------------------------------------ P3: stage 2 from acc
     if (M_max_eff >= 2) {
@@ -1192,7 +1205,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         arrive_and_fit(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8);
         if (threadIdx.x == 0) sm_next = 0;
         __syncthreads();
-        if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns();
+        SIDCO_STAMP(if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns());
 
         // -------------------------------------------------------------- P4: stages 3..M from the side regions
         for (int m = 2; m < M_max_eff; ++m) {
@@ -1238,7 +1251,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             arrive_and_fit(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10);
             if (threadIdx.x == 0) sm_next = 0;
             __syncthreads();
-            if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns();
+            SIDCO_STAMP(if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns());
         }
     }
 
@@ -1272,7 +1285,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             const int i = tag & (kAllSlots - 1);
             long long spins = 0;
             while (R.ok[i] != 100) {                       // published by a thread of this CTA
-                if (++spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+                if (++spins > A.spin_limit) { atomicExch(&A.ctl->timeout, 1); break; }
                 __nanosleep(20);
             }
             __threadfence_block();
@@ -1550,8 +1563,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     }
     if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
     __syncthreads();
-    if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns();
-    if (stamper) A.ctl->t_ns[12] = global_ns();
+    SIDCO_STAMP(if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns());
+    SIDCO_STAMP(if (stamper) A.ctl->t_ns[12] = global_ns());
     // next call: start the first sweep where this call's last full sweep over acc ended
     if (threadIdx.x == 0) A.cta_dir[cta] = (2 * sm_resweep >= c1 - c0) ? (p1_desc ? 1 : 0) : (p1_desc ? 0 : 1);
 
@@ -1656,7 +1669,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 long long spins = 0;
                 while ((unsigned)((w = ld_relaxed_u64(&A.cta_pub[c])) >> 32) != call_id) {
                     if ((++spins & 15) == 0 && ld_volatile(&A.ctl->timeout)) break;
-                    if (spins > kSpinLimit) { atomicExch(&A.ctl->timeout, 1); break; }
+                    if (spins > A.spin_limit) { atomicExch(&A.ctl->timeout, 1); break; }
                     __nanosleep(spins < 64 ? 20 : 100);
                 }
                 below += (int)(unsigned)w;
@@ -1666,7 +1679,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             if (lane == 0) sm_base = below;
         }
         __syncthreads();
-        if (stamper) A.ctl->t_ns[4] = global_ns();
+        SIDCO_STAMP(if (stamper) A.ctl->t_ns[4] = global_ns());
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
         if (place_from_smem) {
@@ -1732,7 +1745,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         }
     }
 
-    if (stamper) A.ctl->t_ns[5] = global_ns();
+    SIDCO_STAMP(if (stamper) A.ctl->t_ns[5] = global_ns());
 }
 
 // Back to the state of a fresh residual: M = 1, counters and candidate thresholds cleared, the residual

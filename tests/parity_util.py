@@ -77,8 +77,7 @@ def check_parity(gpu, ora: O.Result, offsets, state=None, check_status=True):
         for m in range(rep.M_used):
             assert eta_close(dbg.eta[m], rep.eta[m]), f"seg {s} stage {m}: eta {dbg.eta[m]!r} vs {rep.eta[m]!r}"
         if check_status:
-            # bits 16 and 32 are informational (how the final selection read acc), not part of the method
-            assert dbg.status & 15 == rep.status, f"seg {s}: status {dbg.status} vs {rep.status}"
+            assert dbg.status == rep.status, f"seg {s}: status {dbg.status} vs {rep.status}"
         if state is not None:
             assert dbg.M_next == state[s].M and dbg.calls == state[s].calls and dbg.k_sum == state[s].k_sum, \
                 f"seg {s}: adaptation state ({dbg.M_next},{dbg.calls},{dbg.k_sum}) vs " \

@@ -176,10 +176,14 @@ def test_diagnostics_and_bookkeeping():
         before = B.sidco_launch_count()
         run.step(W.ragged_case(5, sizes, 1e-3), f32(0.01), O.SID_EXP, -3)
         assert B.sidco_launch_count() == before + 1           # the whole call is one kernel
-        ph = B.sidco_get_phase_times(run.res)
-        assert len(ph) == 12 and all(0.0 <= x < 1e5 for x in ph[:6]) and ph[5] >= ph[0] > 0
-        ct = B.sidco_get_cta_sweep_times(run.res)
-        assert ct.shape[1] == 4 and ct.shape[0] >= 1 and np.all(ct[:, 0] > 0)
+        # the product build takes no device timestamps: the profiling helpers say so
+        assert B.sidco_build_flags() == 0
+        with pytest.raises(B.SidcoError) as err:
+            B.sidco_get_phase_times(run.res)
+        assert err.value.code == -12
+        with pytest.raises(B.SidcoError) as err:
+            B.sidco_get_cta_sweep_times(run.res)
+        assert err.value.code == -12
         B.sidco_reset_state_async(run.res)
         assert B.sidco_launch_count() == before + 2
     finally:
@@ -187,4 +191,30 @@ def test_diagnostics_and_bookkeeping():
     with pytest.raises(B.SidcoError) as err:
         B.sidco_get_debug(run.res, 1)                          # released: no state for this pointer
     assert err.value.code == -7
-    assert B.sidco_version() >= 100 and "delta" in B.sidco_error_string(-3)
+    assert B.sidco_version() >= 200 and "delta" in B.sidco_error_string(-3)
+
+
+def test_profile_build_reports_phase_times():
+    """The -DSIDCO_PROFILE build of the same sources (loaded in a child process) stamps the phases."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import sys, numpy as np
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+from paper_2101_10761_b200 import binding as B, workloads as W
+from parity_util import GpuRun, f32
+assert B.sidco_build_flags() & B.BUILD_PROFILE
+sizes = [300000]
+run = GpuRun(W.offsets_from_sizes(sizes))
+run.step(W.ragged_case(5, sizes, 1e-3), f32(0.01), 0, -3)
+ph = B.sidco_get_phase_times(run.res)
+assert len(ph) == 12 and all(0.0 <= x < 1e5 for x in ph[:6]) and ph[5] >= ph[0] > 0, ph
+ct = B.sidco_get_cta_sweep_times(run.res)
+assert ct.shape[1] == 4 and ct.shape[0] >= 1 and np.all(ct[:, 0] > 0)
+run.close()
+print("profile ok")
+''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SIDCO_LIB_VARIANT="profile")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "profile ok" in r.stdout, (r.stdout[-1000:], r.stderr[-3000:])
