@@ -668,12 +668,123 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-def bench_aggregate(torch, B, wl, head, dev, peak):
-    return None
+def bench_aggregate(torch, B, wl, head, dev, peak, n_workers=8):
+    """The step after compress: sidco_aggregate on the lists of n_workers compress calls (each worker its own
+    draw of the workload, single stage), three output buffers in rotation so that the 4 d bytes written per
+    call do not stay in the L2."""
+    d, S = wl.d, wl.n_segs
+    lists = []
+    res = torch.zeros(d, dtype=torch.float32, device=dev)
+    k_buf = torch.zeros(S + 1, dtype=torch.int32, device=dev)
+    for w in range(n_workers):
+        g = torch.from_numpy(wl.draw(100 + w)).to(dev)
+        res.zero_()
+        B.sidco_compress(g, res, wl.seg_offsets, DELTA, 0, -1, head.out_idx, head.out_val, k_buf)
+        torch.cuda.synchronize()
+        k = int(k_buf[S])
+        lists.append((head.out_idx[:k].clone(), head.out_val[:k].clone()))
+        del g
+    B.sidco_release(res)
+    del res
+    counts = torch.tensor([int(i.numel()) for i, _ in lists], dtype=torch.int32, device=dev)
+    stride = (int(counts.max()) + 7) // 8 * 8
+    idx_all = torch.zeros(n_workers * stride, dtype=torch.int32, device=dev)
+    val_all = torch.zeros(n_workers * stride, dtype=torch.float32, device=dev)
+    for w, (i, v) in enumerate(lists):
+        idx_all[w * stride:w * stride + i.numel()] = i
+        val_all[w * stride:w * stride + v.numel()] = v
+    outs = [torch.empty(d, dtype=torch.float32, device=dev) for _ in range(3)]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for w in range(6):
+        B.sidco_aggregate(idx_all, val_all, counts, n_workers, stride, d, outs[w % 3], status)
+    torch.cuda.synchronize()
+    times = []
+    n = 30
+    for _ in range(7):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for w in range(n):
+            B.sidco_aggregate(idx_all, val_all, counts, n_workers, stride, d, outs[w % 3], None)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / n)
+    ms = statistics.median(times)
+    nbytes = 8 * int(counts.sum()) + 4 * d
+    return {"workload": f"{n_workers} workers' lists from config {CONFIG} (EXP, one stage, delta {DELTA:g}), d={d}",
+            "entries_total": int(counts.sum()), "ms_per_call": ms, "status": int(status.item()),
+            "roofline": {"bound": "hbm", "achieved": nbytes / ms / 1e6, "peak": peak, "unit": "GB/s",
+                         "frac": nbytes / ms / 1e6 / peak, "algorithmic_bytes_per_launch": nbytes,
+                         "bytes_note": "8 bytes per gathered (index, value) pair read + 4 d bytes written",
+                         "traffic": None},
+            "l2": "three output buffers (3 x 4 d bytes) in rotation"}
+
+
+SWEEP_SIZES = [
+    ("0.26M", 262_144), ("2.6M", 2_621_440), ("26M", 26_214_400), ("lstm-an4 43.5M", 43_476_256),
+    ("vgg19 143.7M", 143_652_544), ("260M", 262_144_000),
+]
 
 
 def bench_sweep(torch, B, dev, peak, args):
-    return None
+    """Size sweep of the paper's synthetic micro-benchmark: single-segment Laplace tensors of 0.26 / 2.6 /
+    26 / 260 million elements and the two remaining model sizes of its Table 1 (as one segment each), fp32 and
+    bf16 gradients, delta = 1e-3, EXP, one stage.  Steady-state calls (residual carried, no resets), warm
+    (back to back) and cold (L2 flushed before every call, timed by subtracting the flush-only loop)."""
+    out = []
+    gen = torch.Generator(device=dev)
+    flush = torch.zeros(FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
+    for name, d in SWEEP_SIZES:
+        n_bufs = 4 if d <= 50_000_000 else 2
+        grads = []
+        for b in range(n_bufs):
+            gen.manual_seed(7000 + b)
+            u = torch.rand(d, device=dev, generator=gen) - 0.5
+            grads.append(-1e-3 * torch.sign(u) * torch.log1p(-2.0 * u.abs()))      # Laplace(0, 1e-3)
+            del u
+        off = np.array([0, d], dtype=np.int64)
+        res = torch.zeros(d, dtype=torch.float32, device=dev)
+        out_idx = torch.empty(d, dtype=torch.int32, device=dev)
+        out_val = torch.empty(d, dtype=torch.float32, device=dev)
+        out_k = torch.zeros(2, dtype=torch.int32, device=dev)
+        row = {"name": name, "d": d}
+        for dtype in ("f32", "bf16"):
+            gs = grads if dtype == "f32" else [g.to(torch.bfloat16) for g in grads]
+            call = B.sidco_compress if dtype == "f32" else B.sidco_compress_bf16
+            per_elem = 12 if dtype == "f32" else 10
+            res.zero_()
+
+            def loop(n, with_flush, with_call=True):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(n):
+                    if with_flush:
+                        flush.add_(1)
+                    if with_call:
+                        call(gs[i % n_bufs], res, off, DELTA, 0, -1, out_idx, out_val, out_k)
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / n
+
+            loop(12, False)
+            n = 200 if d < 10_000_000 else (60 if d < 100_000_000 else 24)
+            warm = statistics.median(loop(n, False) for _ in range(5))
+            cold = statistics.median(loop(n, True) - loop(n, True, False) for _ in range(3))
+            k_hat = int(out_k[1])
+            nbytes = per_elem * d + 8 * k_hat
+            row[dtype] = {"k_hat": k_hat, "warm_us": round(warm * 1e3, 2), "cold_us": round(cold * 1e3, 2),
+                          "warm_GBps": round(nbytes / warm / 1e6, 1), "cold_GBps": round(nbytes / cold / 1e6, 1),
+                          "warm_frac": round(nbytes / warm / 1e6 / peak, 4),
+                          "cold_frac": round(nbytes / cold / 1e6 / peak, 4),
+                          "bytes_per_element": per_elem}
+            if dtype == "bf16":
+                del gs
+        B.sidco_release(res)
+        del res, out_idx, out_val, grads
+        torch.cuda.empty_cache()
+        out.append(row)
+    return {"rows": out, "config": "single segment, Laplace(0, 1e-3) drawn on the device (seeds 7000..), delta 1e-3, "
+                                   "EXP, fixed one stage, residual carried; every call launched directly",
+            "cold_method": "(loop of flush + call) - (loop of flush alone), per call"}
 
 
 def main():

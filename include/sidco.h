@@ -114,6 +114,20 @@ int sidco_compress(const float* grad, float* residual, const int64_t* seg_offset
                    int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
 
 /*
+ * sidco_compress_bf16 - sidco_compress with the gradient stored as bf16 (the error-compensation memory, the
+ * thresholds and the outputs stay fp32).  Step 1 becomes acc_j = (float)grad_j + residual_j, the bf16 value
+ * widened exactly; everything after it is unchanged.  This is the mixed-precision variant of the paper's
+ * synthetic-tensor micro-benchmark (appendix, compression overhead on tensors of 0.26 to 260 million elements)
+ * for frameworks that keep gradients in bf16: the call reads 2 bytes per gradient element instead of 4.
+ * grad_bf16   device, uint16[d] holding bf16 bit patterns, read only; 16-byte alignment (together with a
+ *             32-byte aligned residual) gives the vectorised path.
+ * State is keyed by `residual` as in sidco_compress, and the two entry points may be mixed on one residual.
+ */
+int sidco_compress_bf16(const uint16_t* grad_bf16, float* residual, const int64_t* seg_offsets, int n_segs,
+                        float delta, int sid_type, int max_stages,
+                        int32_t* out_idx, float* out_val, int32_t* out_k, void* stream);
+
+/*
  * sidco_compress_host - the same operation with HOST buffers (pinned memory gives full copy speed).
  * Copies grad and residual to device staging buffers owned by the library, runs sidco_compress,
  * copies residual, out_k and the first out_k[n_segs] entries of out_idx/out_val back, and

@@ -295,5 +295,12 @@ def sidco_compress(grad: np.ndarray, residual: np.ndarray, seg_offsets, delta: f
     return Result(idx=idx, val=val, out_k=out_k, residual=new_res, acc=acc, report=reports)
 
 
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """A gradient stored as bf16 enters the error-compensation add widened exactly: bf16 is the upper half
+    of an fp32, so the value is the 16 bits followed by 16 zero bits.  (Mixed-precision variant of the
+    synthetic-tensor micro-benchmark; the method itself is unchanged.)"""
+    return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
 def new_state(n_segs: int) -> List[SegState]:
     return [SegState() for _ in range(n_segs)]

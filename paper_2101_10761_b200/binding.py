@@ -43,7 +43,7 @@ EXPORTS = [
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
-    "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate",
+    "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate", "sidco_compress_bf16",
 ]
 
 _lib = None
@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
     L.sidco_compress_host.restype = i32
     L.sidco_compress_static.argtypes = compress_sig
     L.sidco_compress_static.restype = i32
+    L.sidco_compress_bf16.argtypes = compress_sig
+    L.sidco_compress_bf16.restype = i32
     L.sidco_workspace_bytes.argtypes = [i64, i32]
     L.sidco_workspace_bytes.restype = C.c_size_t
     L.sidco_set_workspace.argtypes = [vp, vp, C.c_size_t]
@@ -148,6 +150,16 @@ def sidco_compress(grad, residual, seg_offsets, delta: float, sid_type: int, max
                               _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
     if rc:
         raise SidcoError(rc, "sidco_compress")
+
+
+def sidco_compress_bf16(grad_bf16, residual, seg_offsets, delta: float, sid_type: int, max_stages: int,
+                        out_idx, out_val, out_k, stream=None) -> None:
+    """sidco_compress with a bf16 gradient (torch.bfloat16 tensor, or uint16 bit patterns); fp32 residual."""
+    arr, p, n = _offsets(seg_offsets)
+    rc = lib().sidco_compress_bf16(_ptr(grad_bf16), _ptr(residual), p, n, delta, sid_type, max_stages,
+                                   _ptr(out_idx), _ptr(out_val), _ptr(out_k), _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_compress_bf16")
 
 
 def sidco_compress_host(grad, residual, seg_offsets, delta: float, sid_type: int, max_stages: int,

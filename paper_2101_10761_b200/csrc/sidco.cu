@@ -39,7 +39,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_desc;
-    size_t part, part_n, side_cnt, chunk_cnt, side_idx, side_val, stage_idx, stage_val, cta_total, cand, cta_dir, cta_ns, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cand, cta_dir, cta_ns, seg, ctl;
     size_t total;
 };
 
@@ -57,8 +57,8 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.part_n = take(sizeof(int32_t) * (size_t)(T + 1));
     L.side_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
     L.chunk_cnt = take(sizeof(int32_t) * (size_t)(T + 1));
-    L.side_idx = take(sizeof(int32_t) * (size_t)(d + 4));
-    L.side_val = take(sizeof(float) * (size_t)(d + 4));
+    L.side_val = take(sizeof(float) * (size_t)kChunk * (size_t)(T + 1));
+    L.side_mask = take(sizeof(unsigned) * 32 * (size_t)(T + 1));
     L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
     L.stage_val = take(sizeof(float) * (size_t)(d + 4));
     L.cta_total = take(sizeof(unsigned long long) * (size_t)(G + 1));
@@ -129,7 +129,11 @@ namespace {
 
 template <int SID>
 cudaError_t occupancy(int* out) {
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sidco::sidco_persistent_kernel<SID>, kThreads, 0);
+    cudaError_t e = cudaFuncSetAttribute(sidco::sidco_persistent_kernel<SID>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         sidco::kDynSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sidco::sidco_persistent_kernel<SID>, kThreads,
+                                                         sidco::kDynSmemBytes);
 }
 
 cudaError_t device_info(int dev, DeviceInfo** out) {
@@ -317,7 +321,6 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     // (the call numbering restarts: no run's published count may carry a number of the old numbering)
     if ((e = cudaMemset(base + L.cta_total, 0, sizeof(unsigned long long) * (G + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.cta_dir, 0, sizeof(int32_t) * (G + 1))) != cudaSuccess) return e;
-    if ((e = cudaMemset(base + L.side_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
     if ((e = cudaMemset(base + L.chunk_cnt, 0, sizeof(int32_t) * (T + 1))) != cudaSuccess) return e;
 
     c->L = L;
@@ -341,14 +344,14 @@ void fill_ln_tables(Args& a, double delta, double delta1) {
 
 // Cooperative launch: all CTAs of the persistent kernel are co-resident.
 cudaError_t launch_persistent(const void* fn, int grid, void** kargs, cudaStream_t stream) {
-    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), kargs, 0, stream);
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), kargs, sidco::kDynSmemBytes, stream);
 }
 
 // Fill the kernel's argument block for a workspace at `base` laid out as `L` and enqueue the persistent kernel.
 // Used by every entry point, so that they cannot drift apart.
 int launch_compress(char* base, const Layout& L, int T, int S, int G, const float* grad, float* residual, float delta,
                     int sid, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
-                    const Params& prm) {
+                    const Params& prm, bool grad_bf16 = false) {
     Args a{};
     a.grad = grad;
     a.residual = residual;
@@ -363,10 +366,10 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
     a.cta_desc = (const int4*)(base + L.cta_desc);
     a.part = (double*)(base + L.part);
     a.part_n = (int32_t*)(base + L.part_n);
-    a.side_cnt = (int32_t*)(base + L.side_cnt);
     a.chunk_cnt = (int32_t*)(base + L.chunk_cnt);
-    a.side_idx = (int32_t*)(base + L.side_idx);
     a.side_val = (float*)(base + L.side_val);
+    a.side_mask = (unsigned*)(base + L.side_mask);
+    a.side_cnt = (int32_t*)(base + L.side_cnt);
     a.stage_idx = (int32_t*)(base + L.stage_idx);
     a.stage_val = (float*)(base + L.stage_val);
     a.cta_pub = (unsigned long long*)(base + L.cta_total);
@@ -386,7 +389,9 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
     a.C = T;
     a.S = S;
     a.G = G;
-    a.vec_ok = ((((uintptr_t)grad) | ((uintptr_t)residual)) & 31u) == 0;     // 256-bit accesses
+    // 256-bit accesses to the residual and an fp32 gradient, 128-bit ones to a bf16 gradient
+    a.vec_ok = (((uintptr_t)residual & 31u) | ((uintptr_t)grad & (grad_bf16 ? 15u : 31u))) == 0;
+    a.grad_bf16 = grad_bf16 ? 1 : 0;
     const Hooks& h = hooks();
     a.spec_enable = h.spec_enable;           // (the result is the same with or without the pre-selection)
     a.spin_limit = h.spin_limit;
@@ -404,7 +409,7 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
 
 int compress_impl(Context* c, const float* grad, float* residual, const int64_t* off, int S, float delta, int sid,
                   int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
-                  const Params& prm) {
+                  const Params& prm, bool grad_bf16 = false) {
     cudaError_t e;
     const bool same = c->tables_valid && c->S == S &&
                       std::memcmp(c->offsets.data(), off, sizeof(int64_t) * (S + 1)) == 0;
@@ -416,7 +421,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
         if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
     }
     return launch_compress((char*)c->ws, c->L, c->T, c->S, c->G, grad, residual, delta, sid, max_stages, out_idx,
-                           out_val, out_k, stream, prm);
+                           out_val, out_k, stream, prm, grad_bf16);
 }
 
 Context* find_or_create(const void* key, int dev) {
@@ -449,6 +454,23 @@ int sidco_compress(const float* grad, float* residual, const int64_t* seg_offset
     Context* c = find_or_create(residual, dev);
     return compress_impl(c, grad, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k,
                          (cudaStream_t)stream, g_params);
+}
+
+int sidco_compress_bf16(const uint16_t* grad_bf16, float* residual, const int64_t* seg_offsets, int n_segs, float delta,
+                        int sid_type, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, void* stream) {
+    int rc = check_args(grad_bf16, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx, out_val, out_k);
+    if (rc) return rc;
+    const int64_t d = seg_offsets[n_segs];
+    const char* g0 = (const char*)grad_bf16;
+    const char* r0 = (const char*)residual;
+    if ((g0 < r0 + 4 * d) && (r0 < g0 + 2 * d) && d > 0) return SIDCO_E_ALIAS;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    std::lock_guard<std::mutex> lock(g_mu);
+    Context* c = find_or_create(residual, dev);
+    return compress_impl(c, (const float*)grad_bf16, residual, seg_offsets, n_segs, delta, sid_type, max_stages, out_idx,
+                         out_val, out_k, (cudaStream_t)stream, g_params, true);
 }
 
 }  // extern "C"
@@ -555,7 +577,6 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = cudaMemsetAsync(c.base + L.cta_dir, 0, sizeof(int32_t) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.ctl, 0, sizeof(Control), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.cta_total, 0, sizeof(unsigned long long) * (c.G + 1), stream)) != cudaSuccess) return (int)e;
-        if ((e = cudaMemsetAsync(c.base + L.side_cnt, 0, sizeof(int32_t) * (c.T + 1), stream)) != cudaSuccess) return (int)e;
         if ((e = cudaMemsetAsync(c.base + L.chunk_cnt, 0, sizeof(int32_t) * (c.T + 1), stream)) != cudaSuccess) return (int)e;
         // the uploads read the fixed host arrays: let them finish before those can change again
         if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return (int)e;

@@ -4,11 +4,12 @@
 // The lists have been gathered into local memory already (padded to a common stride); this kernel turns
 // them into the dense vector.  Almost all of the output is zeros, so the kernel is a store stream with a
 // sparse correction: every CTA owns a contiguous range of the output; a few of its warps locate the range in
-// each worker's ascending index list (warp-wide 32-ary search) and copy those entries into shared memory
-// while the other warps already write zeros over the range with 32-byte stores; after one CTA barrier the
-// entries are put in place.  A position that several workers sent is written once, by the entry of the first
-// worker that has it: that thread looks the position up in the later workers' lists (binary search in shared
-// memory) and adds their values in worker order in fp64, so the result does not depend on scheduling.
+// each worker's ascending index list (warp-wide 32-ary search) while the other warps already write zeros over
+// the range; after one CTA barrier the range's entries are copied into shared memory, a bitmap over the range
+// finds the positions that more than one worker sent, and the entries are put in place.  Such a shared position
+// is written once, by the entry of the first worker that has it: that thread looks the position up in the
+// later workers' lists (binary search) and adds their values in worker order in fp64, so the result does not
+// depend on scheduling.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -22,7 +23,9 @@ namespace sidco_agg {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxWorkers = SIDCO_AGG_MAX_WORKERS;
-constexpr int kSmemEntries = 11264;            // (index, value) pairs of one CTA range kept in shared memory: 88 KB
+constexpr int kSmemEntries = 6144;             // (index, value) pairs of one CTA range kept in shared memory: 48 KB
+constexpr int kMaxRange = 131072;              // elements of one CTA range: two bitmaps of that many bits, 32 KB
+constexpr int kFillBlock = 2048;               // elements one warp zero-fills per turn (8 KB)
 constexpr unsigned kFull = 0xffffffffu;
 
 struct Args {
@@ -32,9 +35,9 @@ struct Args {
     float* out;                  // [d]
     int32_t* status;             // optional
     long long stride, d;
-    long long per_cta;           // elements per CTA range (a multiple of 8)
+    long long per_cta;           // elements per CTA range (a multiple of kFillBlock, at most kMaxRange)
     int n_workers;
-    int vec_ok;                  // out is 32-byte aligned
+    int vec_ok;                  // out is 16-byte aligned
 };
 
 // First position in [a, b) of the ascending list whose index is >= target (b if none), found by the whole
@@ -72,17 +75,20 @@ __global__ void __launch_bounds__(kThreads, 2) sidco_aggregate_kernel(const __gr
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw);
     float* s_val = reinterpret_cast<float*>(smem_raw + sizeof(int32_t) * kSmemEntries);
+    unsigned* s_seen = reinterpret_cast<unsigned*>(smem_raw + (sizeof(int32_t) + sizeof(float)) * kSmemEntries);
+    unsigned* s_dup = s_seen + kMaxRange / 32;      // position sent by more than one worker
     __shared__ long long s_begin[kMaxWorkers];       // first entry of the range in worker w's list
     __shared__ int s_cnt[kMaxWorkers];               // entries of the range in worker w's list
     __shared__ int s_off[kMaxWorkers + 1];           // prefix sums of s_cnt
-    __shared__ int s_flags;
+    __shared__ int s_flags, s_next;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long lo = (long long)blockIdx.x * A.per_cta;
     long long hi = lo + A.per_cta;
     if (hi > A.d) hi = A.d;
     if (lo >= hi) return;
-    if (threadIdx.x == 0) s_flags = 0;
+    if (threadIdx.x == 0) { s_flags = 0; s_next = 0; }
+    for (int i = threadIdx.x; i < 2 * (kMaxRange / 32); i += kThreads) s_seen[i] = 0u;
     __syncthreads();
     const int N = A.n_workers;
 
@@ -102,21 +108,26 @@ __global__ void __launch_bounds__(kThreads, 2) sidco_aggregate_kernel(const __gr
         }
     }
 
-    // ---- zeros over the range
+    // ---- zeros over the range: warps take 8 KB blocks in turn (the warps that searched join late and take
+    // fewer); every store instruction of a warp covers 512 contiguous bytes
     {
         float* out = A.out;
-        if (A.vec_ok) {
-            // lo is a multiple of 8 and out is 32-byte aligned: whole 32-byte stores up to the last multiple of 8
-            const long long n_vec = (hi - lo) >> 3;
-            float4* o4 = reinterpret_cast<float4*>(out + lo);
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (long long v = threadIdx.x; v < n_vec; v += kThreads) {
-                o4[2 * v] = z;
-                o4[2 * v + 1] = z;
+        const int n_blocks = (int)((hi - lo + kFillBlock - 1) / kFillBlock);
+        for (;;) {
+            int blk = 0;
+            if (lane == 0) blk = atomicAdd(&s_next, 1);
+            blk = __shfl_sync(kFull, blk, 0);
+            if (blk >= n_blocks) break;
+            const long long b0 = lo + (long long)blk * kFillBlock;
+            const long long b1 = b0 + kFillBlock < hi ? b0 + kFillBlock : hi;
+            if (A.vec_ok && b1 - b0 == kFillBlock) {
+                float4* o4 = reinterpret_cast<float4*>(out + b0);
+                const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                #pragma unroll
+                for (int k = 0; k < kFillBlock / 128; ++k) o4[k * 32 + lane] = z;
+            } else {
+                for (long long i = b0 + lane; i < b1; i += 32) out[i] = 0.0f;
             }
-            for (long long i = lo + (n_vec << 3) + threadIdx.x; i < hi; i += kThreads) out[i] = 0.0f;
-        } else {
-            for (long long i = lo + threadIdx.x; i < hi; i += kThreads) out[i] = 0.0f;
         }
     }
     __syncthreads();      // the searches are done, and every zero of this range is ordered before the values below
@@ -133,6 +144,16 @@ __global__ void __launch_bounds__(kThreads, 2) sidco_aggregate_kernel(const __gr
         return;
     }
     const bool in_smem = E <= kSmemEntries;
+    auto entry = [&](int f, int& w, int& idx, float& val) {
+        w = 0;
+        while (f >= s_off[w + 1]) ++w;
+        if (in_smem) { idx = s_idx[f]; val = s_val[f]; }
+        else {
+            const long long at = (long long)w * A.stride + s_begin[w] + (f - s_off[w]);
+            idx = __ldg(A.idx_all + at);
+            val = __ldg(A.val_all + at);
+        }
+    };
     if (in_smem) {
         for (int w = 0; w < N; ++w) {
             const int32_t* gi = A.idx_all + (long long)w * A.stride + s_begin[w];
@@ -145,40 +166,49 @@ __global__ void __launch_bounds__(kThreads, 2) sidco_aggregate_kernel(const __gr
         __syncthreads();
     }
 
-    // ---- the sparse correction: one thread per entry; the first worker that has a position writes it
-    const double inv_scale = (double)N;
+    // ---- which positions were sent by more than one worker
     int bad = 0;
     for (int f = threadIdx.x; f < E; f += kThreads) {
-        int w = 0;
-        while (f >= s_off[w + 1]) ++w;
-        const int i = f - s_off[w];
-        int idx;
+        int w, idx;
         float val;
-        if (in_smem) { idx = s_idx[f]; val = s_val[f]; }
-        else {
-            idx = __ldg(A.idx_all + (long long)w * A.stride + s_begin[w] + i);
-            val = __ldg(A.val_all + (long long)w * A.stride + s_begin[w] + i);
-        }
-        if (idx < lo || idx >= hi) { bad = 1; continue; }          // a list that is not ascending: skip, report
-        bool owner = true;
-        for (int u = 0; u < w && owner; ++u) {
-            const int hit = in_smem ? find_index(s_idx + s_off[u], s_cnt[u], idx)
-                                    : find_index(A.idx_all + (long long)u * A.stride + s_begin[u], s_cnt[u], idx);
-            owner = hit < 0;
-        }
-        if (!owner) continue;
+        entry(f, w, idx, val);
+        if (idx < lo || idx >= hi) { bad = 1; continue; }          // a list that is not ascending: skipped, reported
+        const unsigned r = (unsigned)(idx - lo), bit = 1u << (r & 31);
+        if (atomicOr(&s_seen[r >> 5], bit) & bit) atomicOr(&s_dup[r >> 5], bit);
+    }
+    __syncthreads();
+
+    // ---- the sparse correction, one thread per entry.  A position only one worker sent is that value over N.
+    // A position several workers sent is written once, by the entry of the first worker that has it: that
+    // thread looks it up in the later workers' lists and adds their values in worker order in fp64.
+    const double n_workers = (double)N;
+    for (int f = threadIdx.x; f < E; f += kThreads) {
+        int w, idx;
+        float val;
+        entry(f, w, idx, val);
+        if (idx < lo || idx >= hi) continue;
+        const unsigned r = (unsigned)(idx - lo);
         double sum = 0.0 + (double)val;
-        for (int u = w + 1; u < N; ++u) {
-            if (in_smem) {
-                const int hit = find_index(s_idx + s_off[u], s_cnt[u], idx);
-                if (hit >= 0) sum += (double)s_val[s_off[u] + hit];
-            } else {
-                const int32_t* gi = A.idx_all + (long long)u * A.stride + s_begin[u];
-                const int hit = find_index(gi, s_cnt[u], idx);
-                if (hit >= 0) sum += (double)__ldg(A.val_all + (long long)u * A.stride + s_begin[u] + hit);
+        if ((s_dup[r >> 5] >> (r & 31)) & 1u) {
+            bool owner = true;
+            for (int u = 0; u < w && owner; ++u) {
+                const int hit = in_smem ? find_index(s_idx + s_off[u], s_cnt[u], idx)
+                                        : find_index(A.idx_all + (long long)u * A.stride + s_begin[u], s_cnt[u], idx);
+                owner = hit < 0;
+            }
+            if (!owner) continue;
+            for (int u = w + 1; u < N; ++u) {
+                if (in_smem) {
+                    const int hit = find_index(s_idx + s_off[u], s_cnt[u], idx);
+                    if (hit >= 0) sum += (double)s_val[s_off[u] + hit];
+                } else {
+                    const int32_t* gi = A.idx_all + (long long)u * A.stride + s_begin[u];
+                    const int hit = find_index(gi, s_cnt[u], idx);
+                    if (hit >= 0) sum += (double)__ldg(A.val_all + (long long)u * A.stride + s_begin[u] + hit);
+                }
             }
         }
-        A.out[idx] = (float)(sum / inv_scale);
+        A.out[idx] = (float)(sum / n_workers);
     }
     if (bad) atomicOr(&s_flags, SIDCO_AGG_ST_ORDER);
     __syncthreads();
@@ -204,7 +234,7 @@ int sidco_aggregate(const int32_t* idx_all, const float* val_all, const int32_t*
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return (int)e;
     if (dev < 0 || dev >= 64) return SIDCO_E_SIZE;
     std::lock_guard<std::mutex> lock(mu);
-    const size_t smem = (sizeof(int32_t) + sizeof(float)) * sidco_agg::kSmemEntries;
+    const size_t smem = (sizeof(int32_t) + sizeof(float)) * sidco_agg::kSmemEntries + 2 * (sidco_agg::kMaxRange / 8);
     if (!sm_count[dev]) {
         int n = 0;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return (int)e;
@@ -222,12 +252,12 @@ int sidco_aggregate(const int32_t* idx_all, const float* val_all, const int32_t*
     a.stride = stride;
     a.d = d;
     a.n_workers = n_workers;
-    a.vec_ok = (((uintptr_t)out_dense) & 31u) == 0;
-    // two CTAs per SM; ranges are multiples of 256 elements, and no smaller than 4096
+    a.vec_ok = (((uintptr_t)out_dense) & 15u) == 0;
+    // two CTAs per SM when the vector is small enough for that; ranges are multiples of the fill block
     long long grid = 2ll * sm_count[dev];
     long long per = (d + grid - 1) / grid;
-    if (per < 4096) per = 4096;
-    per = (per + 255) / 256 * 256;
+    per = (per + sidco_agg::kFillBlock - 1) / sidco_agg::kFillBlock * sidco_agg::kFillBlock;
+    if (per > sidco_agg::kMaxRange) per = sidco_agg::kMaxRange;
     grid = (d + per - 1) / per;
     a.per_cta = per;
     sidco_agg::sidco_aggregate_kernel<<<(unsigned)grid, sidco_agg::kThreads, smem, stream>>>(a);

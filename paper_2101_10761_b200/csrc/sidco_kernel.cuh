@@ -25,8 +25,11 @@
 //   P3  (segments with M >= 2) statistics of the shifted peaks |x| - eta_1 over
 //       the exceedances |x| > eta_1 (Lemma 2 / Corollary 2.1) and fit of eta_2.
 //       Two-stage segments record slot flags here (as P1 does for one stage);
-//       segments with more stages compact their exceedances, in order, into the
-//       chunk's side region
+//       segments with more stages copy their exceedances into the chunk's side
+//       region, lane by lane (each lane keeps the values it holds, and a 32-bit mask
+//       says which of its 32 elements they are), with no ordering work at all: the
+//       later statistics need no order, and the few final survivors get theirs back
+//       from the mask
 //   P4  (m = 3..M) statistics of side-region entries above eta_{m-1}; fit eta_m
 //   P5a survivors |x| >= eta_M staged per chunk in ascending order, selected
 //       residual entries zeroed.  A block-wide pass lists the flagged slots of
@@ -117,7 +120,7 @@ struct Control {
 };
 
 struct Args {
-    const float* grad;
+    const float* grad;           // fp32 gradient, or bf16 (two bytes per element) if grad_bf16 is set
     float* residual;
     int32_t* out_idx;
     float* out_val;
@@ -132,10 +135,10 @@ struct Args {
     // scratch
     double* part;                // [C][3] per-chunk partial sums
     int32_t* part_n;             // [C] per-chunk partial counts
-    int32_t* side_cnt;           // [C] stage-2 exceedances stored for the chunk
     int32_t* chunk_cnt;          // [C] final survivors staged for the chunk
-    int32_t* side_idx;           // [d]
-    float* side_val;             // [d]
+    float* side_val;             // [C][kChunk] side regions: the kept values of chunk c, dense, in index order
+    unsigned* side_mask;         // [C][32] per lane: which of its elements (bit 8 j + component) the side region holds
+    int32_t* side_cnt;           // [C] entries in the chunk's side region
     int32_t* stage_idx;          // [d]
     float* stage_val;            // [d]
     unsigned long long* cta_pub; // [G] {call number, survivors of the run}: published once the run's selection is done
@@ -153,6 +156,7 @@ struct Args {
     int C, S, G;
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
+    int grad_bf16;               // grad points to bf16 values, widened exactly to fp32 before the add
     long long spin_limit;        // polls after which a bounded wait gives up (kSpinLimit unless a test shortens it)
     int drop_pub_seg;            // test hook: the published words of this segment are withheld (-1: none), so that
                                  // the runs waiting for them run into the bound
@@ -557,6 +561,25 @@ __device__ __forceinline__ void st8_evict_last(float* p, const F8& r) {
                  : "memory");
 }
 
+// Eight gradient elements starting at element e (read once: evict_first).  A bf16 gradient is widened exactly
+// (bf16 is the upper half of an fp32).
+__device__ __forceinline__ F8 ld8_grad(const float* grad, int e, bool bf16) {
+    if (!bf16) return ld8_evict_first(grad + e);
+    // (the eviction-priority qualifier exists for 256-bit accesses only: a streaming 128-bit load here)
+    const uint4 w = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(grad) + e));
+    const unsigned w0 = w.x, w1 = w.y, w2 = w.z, w3 = w.w;
+    F8 r;
+    r.v[0] = __uint_as_float(w0 << 16); r.v[1] = __uint_as_float(w0 & 0xffff0000u);
+    r.v[2] = __uint_as_float(w1 << 16); r.v[3] = __uint_as_float(w1 & 0xffff0000u);
+    r.v[4] = __uint_as_float(w2 << 16); r.v[5] = __uint_as_float(w2 & 0xffff0000u);
+    r.v[6] = __uint_as_float(w3 << 16); r.v[7] = __uint_as_float(w3 & 0xffff0000u);
+    return r;
+}
+__device__ __forceinline__ float ld1_grad(const float* grad, int e, bool bf16) {
+    if (!bf16) return __ldcs(grad + e);
+    return __uint_as_float((unsigned)__ldcs(reinterpret_cast<const unsigned short*>(grad) + e) << 16);
+}
+
 // Error-compensation memory accesses: `keep` asks for L2 residency.  Segments with three or more stages
 // go without it, because their side regions (re-read by every later stage) need the L2 more.
 __device__ __forceinline__ F8 ld8_res(const float* p, bool keep) {
@@ -673,20 +696,75 @@ struct ChunkQueue {
     }
 };
 
+constexpr int kSidePre = 1;                       // 16-byte pieces of a side region fetched with the descriptor
+constexpr int kSidePre4 = 2;                      // the same in the sweeps that read nothing but side regions
+constexpr int kDynSmemBytes = kWarps * kChunk * (int)sizeof(float);   // per-warp staging of one chunk's side region
+
+// Positions of a lane's kept elements in the chunk's dense, index-ordered side region.  `mask` has bit
+// 8 j + c set for component c of slot j; chunk order is slot, lane, component.  pos[j] is where this lane's
+// first kept element of slot j goes; the return value is the number of kept elements in the whole chunk.
+__device__ __forceinline__ int side_positions(unsigned mask, int (&pos)[kSlots]) {
+    static_assert(kSlots == 4, "two packed scans cover four slots");
+    const int lane = threadIdx.x & 31;
+    const unsigned c01 = __popc(mask & 0xFFu) | (__popc((mask >> 8) & 0xFFu) << 16);
+    const unsigned c23 = __popc((mask >> 16) & 0xFFu) | (__popc(mask >> 24) << 16);
+    unsigned i01 = c01, i23 = c23;                 // inclusive scans over the lanes (a field holds at most 256)
+    #pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned a = __shfl_up_sync(kFull, i01, o), b = __shfl_up_sync(kFull, i23, o);
+        if (lane >= o) { i01 += a; i23 += b; }
+    }
+    const unsigned t01 = __shfl_sync(kFull, i01, 31), t23 = __shfl_sync(kFull, i23, 31);
+    const unsigned e01 = i01 - c01, e23 = i23 - c23;
+    const int t0 = t01 & 0xFFFFu, t1 = t01 >> 16, t2 = t23 & 0xFFFFu, t3 = t23 >> 16;
+    pos[0] = e01 & 0xFFFFu;
+    pos[1] = t0 + (e01 >> 16);
+    pos[2] = t0 + t1 + (e23 & 0xFFFFu);
+    pos[3] = t0 + t1 + t2 + (e23 >> 16);
+    return t0 + t1 + t2 + t3;
+}
+
 // Chunk descriptor, fetched one chunk ahead so that its loads overlap the current chunk's work.
 struct Desc {
-    int c, seg, lo, hi, side_n;
+    int c, seg, lo, hi;
+    int side_n;          // entries in the chunk's side region (phases that read side regions)
     unsigned flags;      // this lane's candidate slot flags (P5a only)
+    float4 pre[kSidePre];// entries 128 u + 4 lane .. + 3 of the side region, fetched with the descriptor and
+                         // without waiting for the count (entries beyond it are ignored)
 };
 
 __device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side, bool with_flags = false) {
-    Desc d{c, 0, 0, 0, 0, 0u};
+    Desc d;
+    d.c = c; d.seg = 0; d.lo = 0; d.hi = 0; d.side_n = 0; d.flags = 0u;
     if (c >= 0) {
         d.seg = __ldg(A.chunk_seg + c);
         d.lo = __ldg(A.chunk_start + c);
         d.hi = __ldg(A.chunk_start + c + 1);
-        if (with_side) d.side_n = ld_cg(A.side_cnt + c);
+        if (with_side) {
+            d.side_n = ld_cg(A.side_cnt + c);
+            const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + (threadIdx.x & 31);
+            #pragma unroll
+            for (int u = 0; u < kSidePre; ++u) d.pre[u] = __ldcg(side + 32 * u);
+        }
         if (with_flags) d.flags = __ldcg(A.cand + (size_t)c * 32 + (threadIdx.x & 31));
+    }
+    return d;
+}
+
+// Descriptor of the sweeps over side regions alone (stages 3..M).
+struct SideDesc {
+    int c, seg, side_n;
+    float4 pre[kSidePre4];
+};
+__device__ __forceinline__ SideDesc fetch_side_desc(const Args& A, int c) {
+    SideDesc d;
+    d.c = c; d.seg = 0; d.side_n = 0;
+    if (c >= 0) {
+        d.seg = __ldg(A.chunk_seg + c);
+        d.side_n = ld_cg(A.side_cnt + c);
+        const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + (threadIdx.x & 31);
+        #pragma unroll
+        for (int u = 0; u < kSidePre4; ++u) d.pre[u] = __ldcg(side + 32 * u);
     }
     return d;
 }
@@ -906,6 +984,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
 
 template <int SID>
 __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __grid_constant__ Args A) {
+    extern __shared__ __align__(16) float sm_stage[];        // [kWarps][kChunk] (kDynSmemBytes)
     __shared__ double sm_red[kWarps][3];
     __shared__ int sm_list[kThreads];
     __shared__ int sm_scan[kThreads];
@@ -935,6 +1014,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     const int4 run = __ldg(A.cta_desc + cta);          // {first chunk, end chunk, first segment, segments}
     const int c0 = run.x, c1 = run.y;
     const bool vec_ok = A.vec_ok != 0;
+    const bool g_bf16 = A.grad_bf16 != 0;
     const ChunkQueue queue{&sm_next, c0, c1};
     // Sweep directions.  Every full sweep over acc starts where the previous one (of this call or
     // of the last call) ended, so that it begins on the lines most recently left in L2.
@@ -1002,7 +1082,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     {
         int tau_seg = -1;
         float tau = -1.0f;
-        bool keep = true;          // ask for L2 residency of this segment's acc lines
+        const bool keep = true;    // ask for L2 residency of the acc lines
         Desc cur = first_desc;
         while (cur.c >= 0) {
             const Desc nxt = fetch_desc(A, queue.next(p1_desc), false);
@@ -1013,7 +1093,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 tau_seg = cur.seg;
                 const int m = stages_of(cur.seg);
                 tau = m == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments flag in P3
-                keep = m <= 2;
             }
             unsigned flags = 0;
 
@@ -1042,7 +1121,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     F8 g8[2], r8[2];
                     #pragma unroll
                     for (int j = 0; j < 2; ++j) {
-                        g8[j] = ld8_evict_first(A.grad + e0 + (b + j) * 256);
+                        g8[j] = ld8_grad(A.grad, e0 + (b + j) * 256, g_bf16);
                         if (!res_zero) r8[j] = ld8_res(A.residual + e0 + (b + j) * 256, keep);
                     }
                     #pragma unroll
@@ -1066,7 +1145,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     const int e = e0 + j * 256;
                     if (e + kComp <= lo || e >= hi) continue;
                     if (vec_ok && e >= lo && e + kComp <= hi) {
-                        const F8 g = ld8_evict_first(A.grad + e);
+                        const F8 g = ld8_grad(A.grad, e, g_bf16);
                         F8 r;
                         if (!res_zero) r = ld8_res(A.residual + e, keep);
                         #pragma unroll
@@ -1078,7 +1157,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     } else {
                         for (int cc = 0; cc < kComp; ++cc) {
                             if (e + cc >= lo && e + cc < hi) {
-                                const float a = __ldcs(A.grad + e + cc) + (res_zero ? 0.0f : A.residual[e + cc]);
+                                const float a = ld1_grad(A.grad, e + cc, g_bf16) + (res_zero ? 0.0f : A.residual[e + cc]);
                                 A.residual[e + cc] = a;
                                 accumulate(a);
                             }
@@ -1131,46 +1210,33 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     const int c = cur.c, lo = cur.lo, hi = cur.hi;
                     const int wb = lo & ~(kChunk - 1);
                     float v[kSlots][kComp];
-                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, sv.M_eff <= 2, v);
-                    unsigned mask = 0;
-                    #pragma unroll
-                    for (int j = 0; j < kSlots; ++j)
-                        #pragma unroll
-                        for (int cc = 0; cc < kComp; ++cc)
-                            if (fabsf(v[j][cc]) > sv.thr_gt) mask |= 1u << (8 * j + cc);
-                    mask &= valid;
+                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
+                    // Stage 2 is the last stage of a two-stage segment: nothing reads its exceedances again except
+                    // the final selection, which can work from slot flags (as after P1 for one stage).
+                    const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
+                    const bool flag_chunk = tau2 > 0.0f && vec_ok && lo == wb && hi == wb + kChunk;
+                    // (elements outside the chunk read as zero and the threshold is never negative, so they
+                    // pass no strict compare)
+                    unsigned mask = 0, flags = 0;
                     double sy = 0.0, sy2 = 0.0;
                     #pragma unroll
-                    for (int j = 0; j < kSlots; ++j)
+                    for (int j = 0; j < kSlots; ++j) {
+                        float big = 0.0f;
                         #pragma unroll
-                        for (int cc = 0; cc < kComp; ++cc)
-                        {
-                            // branch-free: entries below the threshold contribute an exact zero
-                            const bool in = (mask >> (8 * j + cc)) & 1u;
-                            const double y = in ? (double)fabsf(v[j][cc]) - sv.eta_prev : 0.0;
-                            sy += y;
-                            if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                        for (int cc = 0; cc < kComp; ++cc) {
+                            const float a = fabsf(v[j][cc]);
+                            big = fmaxf(big, a);
+                            if (a > sv.thr_gt) {
+                                const double y = (double)a - sv.eta_prev;
+                                sy += y;
+                                if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                                mask |= 1u << (8 * j + cc);
+                            }
                         }
-                    const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
-                    const bool full = vec_ok && lo == wb && hi == wb + kChunk;
-                    if (tau2 > 0.0f && full) {
-                        // Stage 2 is this segment's last: nothing reads the exceedances again except the
-                        // final selection, which can work from slot flags (as after P1 for one stage).
-                        unsigned flags = 0;
-                        #pragma unroll
-                        for (int j = 0; j < kSlots; ++j) {
-                            float big = 0.0f;
-                            #pragma unroll
-                            for (int cc = 0; cc < kComp; ++cc) big = fmaxf(big, fabsf(v[j][cc]));
-                            flags |= (unsigned)(big >= tau2) << j;
-                        }
+                        flags |= (unsigned)(big >= tau2) << j;
+                    }
+                    if (flag_chunk) {
                         A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
-                        Sums r = warp_tree(sy, sy2, __popc(mask));
-                        if (lane == 0) {
-                            A.part[3 * (size_t)c + 0] = r.a;
-                            A.part[3 * (size_t)c + 1] = r.b;
-                            A.part_n[c] = r.n;
-                        }
                     } else {
                         // The side region also takes the entries equal to eta_1: they are no exceedances (the
                         // statistics above leave them out), but if no later stage raises the threshold
@@ -1185,18 +1251,31 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                                     if (fabsf(v[j][cc]) == sv.thr_gt) keep_mask |= 1u << (8 * j + cc);
                             keep_mask &= valid;
                         }
-                        const int e0 = wb + lane * kComp;
-                        const int cnt = ordered_emit(keep_mask, lo, [&](int p, int j, int cc) {
-                            A.side_idx[p] = e0 + j * 256 + cc;
-                            A.side_val[p] = v[j][cc];
-                        });
-                        Sums r = warp_tree(sy, sy2, __popc(mask));
-                        if (lane == 0) {
-                            A.part[3 * (size_t)c + 0] = r.a;
-                            A.part[3 * (size_t)c + 1] = r.b;
-                            A.part_n[c] = r.n;          // exceedances (the next fit's count)
-                            A.side_cnt[c] = cnt;        // entries stored
+                        // The kept values go to the chunk's side region dense and in index order: every lane puts its
+                        // own at their positions in the warp's shared-memory staging area, and the warp copies the
+                        // area out with 16-byte stores.
+                        int pos[kSlots];
+                        const int kept = side_positions(keep_mask, pos);
+                        float* stage = sm_stage + warp * kChunk;
+                        #pragma unroll
+                        for (int j = 0; j < kSlots; ++j) {
+                            int q = pos[j];
+                            #pragma unroll
+                            for (int cc = 0; cc < kComp; ++cc)
+                                if ((keep_mask >> (8 * j + cc)) & 1u) stage[q++] = v[j][cc];
                         }
+                        __syncwarp();
+                        float4* side = reinterpret_cast<float4*>(A.side_val + (size_t)c * kChunk);
+                        for (int q = lane; 4 * q < kept; q += 32) side[q] = reinterpret_cast<const float4*>(stage)[q];
+                        __syncwarp();
+                        if (lane == 0) A.side_cnt[c] = kept;
+                        A.side_mask[(size_t)c * 32 + lane] = keep_mask;
+                    }
+                    Sums r = warp_tree(sy, sy2, __popc(mask));
+                    if (lane == 0) {
+                        A.part[3 * (size_t)c + 0] = r.a;
+                        A.part[3 * (size_t)c + 1] = r.b;
+                        A.part_n[c] = r.n;              // exceedances (the next fit's count)
                     }
                 }
                 cur = nxt;
@@ -1212,31 +1291,35 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             publish_params(A, R, m, m - 1, m);
             {
                 SegView sw;
-                Desc cur = fetch_desc(A, queue.next(false), true);
+                SideDesc cur = fetch_side_desc(A, queue.next(false));
                 while (cur.c >= 0) {
-                    const Desc nxt = fetch_desc(A, queue.next(false), true);
+                    const SideDesc nxt = fetch_side_desc(A, queue.next(false));
                     view_load(A, R, sw, cur.seg, m, m - 1, m, cap);
                     if (sw.M_eff > m) {
-                        // the side region is a compact list: lanes stride over its entries
+                        // the side region is a dense list: 16 bytes per lane and step, the first steps fetched
+                        // with the descriptor
                         const int c = cur.c, n = cur.side_n;
-                        const float* list = A.side_val + cur.lo;
+                        const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
                         double sy = 0.0, sy2 = 0.0;
                         int cnt = 0;
-                        for (int i0 = 0; i0 < n; i0 += 512) {
-                            float a[16];
+                        auto take = [&](const float4& x, int first) {
+                            const float a[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
                             #pragma unroll
-                            for (int u = 0; u < 16; ++u) {
-                                const int i = i0 + u * 32 + lane;
-                                a[u] = i < n ? fabsf(ld_cg(list + i)) : 0.0f;
-                            }
-                            #pragma unroll
-                            for (int u = 0; u < 16; ++u)
-                                if (a[u] > sw.thr_gt) {        // thr_gt >= 0, so padding zeros never pass
+                            for (int u = 0; u < 4; ++u)
+                                if (first + u < n && a[u] > sw.thr_gt) {
                                     const double y = (double)a[u] - sw.eta_prev;
                                     sy += y;
                                     if (SID != kSidExp) sy2 = fma(y, y, sy2);
                                     ++cnt;
                                 }
+                        };
+                        #pragma unroll
+                        for (int u = 0; u < kSidePre4; ++u) take(cur.pre[u], 128 * u + 4 * lane);
+                        for (int t = kSidePre4; 128 * t < n; t += 2) {
+                            const float4 x0 = __ldcg(side + 32 * t);
+                            const float4 x1 = 128 * (t + 1) < n ? __ldcg(side + 32 * (t + 1)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            take(x0, 128 * t + 4 * lane);
+                            take(x1, 128 * (t + 1) + 4 * lane);
                         }
                         Sums r = warp_tree(sy, sy2, cnt);
                         if (lane == 0) {
@@ -1482,9 +1565,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         SegView sv;
         bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
         int seg_count = 0;       // survivors of sv.seg not yet added to its counter
-        Desc cur = fetch_desc(A, n_rest == 0 ? -1 : next_chunk(), true, true);
+        const bool any_side = M_max_eff >= 2;      // some chunk of this run may have a side region
+        Desc cur = fetch_desc(A, n_rest == 0 ? -1 : next_chunk(), any_side, true);
         while (cur.c >= 0) {
-            const Desc nxt = fetch_desc(A, next_chunk(), true, true);
+            const Desc nxt = fetch_desc(A, next_chunk(), any_side, true);
             if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) add_seg_count(sv.seg, seg_count);
                 seg_count = 0;
@@ -1503,30 +1587,58 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             const bool from_side = seg_from_side && !(seg_two_flagged && vec_ok && lo == wb && cur.hi == wb + kChunk);
             int cnt = 0;
             if (from_side) {
-                // compact list of stage-2 exceedances: lanes stride over it, one ballot per 32 entries
+                // The side region is a dense list in index order.  Lanes read it 16 bytes at a time; a survivor is
+                // known by its position in the list, and the lane that holds the element at that position (found
+                // through the per-lane masks, only for chunks that have a survivor at all) marks it in a mask of
+                // the chunk's own layout, which gives the survivors their indices and their order.
                 const int n = cur.side_n;
-                const unsigned lt = (1u << lane) - 1u;
-                for (int i0 = 0; i0 < n; i0 += 512) {
-                    float x[16];
+                const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
+                unsigned surv = 0;
+                int pos[kSlots];
+                unsigned smask = 0;
+                bool have_pos = false;
+                auto take = [&](const float4& x, int first) {
+                    const float a[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
+                    unsigned hit = 0;
                     #pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        x[u] = i < n ? ld_cg(A.side_val + lo + i) : 0.0f;
+                    for (int u = 0; u < 4; ++u)
+                        if (first + u < n && a[u] >= sv.thr_ge) hit |= 1u << u;
+                    unsigned any = __ballot_sync(kFull, hit != 0);
+                    if (any == 0) return;
+                    if (!have_pos) {
+                        smask = __ldcg(A.side_mask + (size_t)c * 32 + lane);
+                        side_positions(smask, pos);
+                        have_pos = true;
                     }
-                    #pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        const int i = i0 + u * 32 + lane;
-                        const bool hit = i < n && fabsf(x[u]) >= sv.thr_ge;
-                        const unsigned b = __ballot_sync(kFull, hit);
-                        if (hit) {
-                            const int p = lo + cnt + __popc(b & lt);
-                            const int idx = ld_cg(A.side_idx + lo + i);
-                            A.stage_idx[p] = idx;
-                            A.stage_val[p] = x[u];
-                            A.residual[idx] = 0.0f;
+                    while (any) {
+                        const int src = __ffs(any) - 1;
+                        any &= any - 1u;
+                        unsigned h = __shfl_sync(kFull, hit, src);
+                        const int base = __shfl_sync(kFull, first, src);
+                        while (h) {
+                            const int p = base + __ffs(h) - 1;         // position in the list
+                            h &= h - 1u;
+                            // the lane whose elements of some slot cover position p
+                            #pragma unroll
+                            for (int j = 0; j < kSlots; ++j) {
+                                const unsigned byte = (smask >> (8 * j)) & 0xFFu;
+                                const int r = p - pos[j];
+                                if (r >= 0 && r < __popc(byte)) surv |= (1u << (8 * j)) << (__fns(byte, 0, r + 1));
+                            }
                         }
-                        cnt += __popc(b);
                     }
+                };
+                #pragma unroll
+                for (int u = 0; u < kSidePre; ++u) take(cur.pre[u], 128 * u + 4 * lane);
+                for (int t = kSidePre; 128 * t < n; ++t) take(__ldcg(side + 32 * t), 128 * t + 4 * lane);
+                if (__ballot_sync(kFull, surv != 0)) {
+                    const int e0 = wb + lane * kComp;
+                    cnt = ordered_emit(surv, lo, [&](int p, int j, int cc) {
+                        const int e = e0 + j * 256 + cc;
+                        A.stage_idx[p] = e;
+                        A.stage_val[p] = __ldcg(A.residual + e);
+                        A.residual[e] = 0.0f;
+                    });
                 }
             } else {
                 const int hi = cur.hi;

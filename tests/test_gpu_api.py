@@ -62,7 +62,7 @@ def test_caller_owned_workspace():
     off = W.offsets_from_sizes(sizes)
     d = int(off[-1])
     need = B.sidco_workspace_bytes(d, len(sizes))
-    assert need > 16 * d
+    assert need > 8 * d
     ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda:0")
     base = (ws.data_ptr() + 255) // 256 * 256
     run = GpuRun(off)

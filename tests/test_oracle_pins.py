@@ -449,3 +449,19 @@ def test_sign_symmetry():
     b = O.sidco_compress(-x, np.zeros_like(x), [0, n], 0.01, O.SID_GPD, -2)
     assert np.array_equal(a.idx, b.idx) and np.array_equal(a.val, -b.val)
     assert a.report[0].eta == b.report[0].eta
+
+
+# ------------------------------------------------------------------ bf16 gradients
+
+def test_bf16_widening_matches_an_independent_conversion():
+    import torch
+    r = rng(404)
+    bits = r.integers(0, 1 << 16, 20000).astype(np.uint16)
+    bits = bits[((bits >> 7) & 0xFF) != 0xFF]                 # finite values only (NaN payloads compare unequal)
+    want = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(torch.float32).numpy()
+    got = O.bf16_bits_to_f32(bits)
+    assert got.dtype == np.float32 and np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # and rounding an fp32 to bf16 and back changes it by at most half a bf16 ulp
+    x = r.standard_normal(1000).astype(np.float32)
+    xb = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.all(np.abs(O.bf16_bits_to_f32(xb) - x) <= np.abs(x) * 2.0 ** -8)
