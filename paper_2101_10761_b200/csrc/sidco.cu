@@ -39,7 +39,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_desc;
-    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cand, cta_dir, cta_ns, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, seg, ctl;
     size_t total;
 };
 
@@ -62,7 +62,6 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.stage_idx = take(sizeof(int32_t) * (size_t)(d + 4));
     L.stage_val = take(sizeof(float) * (size_t)(d + 4));
     L.cta_total = take(sizeof(unsigned long long) * (size_t)(G + 1));
-    L.cand = take(32 * (size_t)(T + 1));
     L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
     L.cta_ns = take(sizeof(unsigned long long) * 4 * (size_t)(G + 1));
     L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
@@ -373,7 +372,6 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
     a.stage_idx = (int32_t*)(base + L.stage_idx);
     a.stage_val = (float*)(base + L.stage_val);
     a.cta_pub = (unsigned long long*)(base + L.cta_total);
-    a.cand = (unsigned char*)(base + L.cand);
     a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.cta_ns = (unsigned long long*)(base + L.cta_ns);
     a.seg = (SegDev*)(base + L.seg);

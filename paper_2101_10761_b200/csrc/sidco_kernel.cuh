@@ -68,11 +68,11 @@ constexpr int kComp = 8;                          // elements per slot: one 32-b
 constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4)
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
 constexpr int kSegCache = 256;                    // segments of a CTA run whose table entries sit in shared memory
-constexpr int kOutCache = 1024;                   // survivors of a run kept in shared memory for the final placement
-constexpr int kCoopChunks = 4096;                 // chunks of a run the block-wide flagged-slot pass can cover
-constexpr int kCoopPass = kThreads / 2;           // chunks per pass of it (two threads per chunk)
-constexpr int kCoopItems = 4096;                  // flagged slots one pass can list
-constexpr float kSpecRatio = 0.8f;                // candidate threshold = this fraction of the last eta
+constexpr int kOutCache = 2048;                   // survivors of a run the shared-memory selection can hold
+constexpr int kSlotCap = 1536;                    // candidate slots (8 elements) of a run held in shared memory
+constexpr int kWinCap = 2048;                     // 1024-element windows of a run the shared-memory selection covers
+static_assert(kSlotCap * kComp >= 2 * kOutCache, "the ordered survivors reuse the candidate values' space");
+constexpr float kSpecRatio = 0.85f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr long long kSpinLimit = 1ll << 22;       // default bound of the waits: ~1 s with the back-off below
@@ -142,7 +142,6 @@ struct Args {
     int32_t* stage_idx;          // [d]
     float* stage_val;            // [d]
     unsigned long long* cta_pub; // [G] {call number, survivors of the run}: published once the run's selection is done
-    unsigned char* cand;         // [C][32] per-lane slot flags of full chunks: slot may hold a survivor
     int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
     unsigned long long* cta_ns;  // [G][4] globaltimer when the CTA finished its P1, P3, last P4, P5a sweep
     SegDev* seg;                 // [S]
@@ -580,6 +579,15 @@ __device__ __forceinline__ float ld1_grad(const float* grad, int e, bool bf16) {
     return __uint_as_float((unsigned)__ldcs(reinterpret_cast<const unsigned short*>(grad) + e) << 16);
 }
 
+// Asynchronous 16-byte copy from global to shared memory (completes in the background; see cp_async_wait_all).
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+}
+
 // Error-compensation memory accesses: `keep` asks for L2 residency.  Segments with three or more stages
 // go without it, because their side regions (re-read by every later stage) need the L2 more.
 __device__ __forceinline__ F8 ld8_res(const float* p, bool keep) {
@@ -678,15 +686,6 @@ struct ChunkQueue {
         if (k >= c1 - c0) return -1;
         return descending ? c1 - 1 - k : c0 + k;
     }
-    // As next(), but passes over the chunks whose bit is set in `done` (bit = chunk - c0, first n_done chunks).
-    __device__ __forceinline__ int next_undone(bool descending, const unsigned* done, int n_done) const {
-        for (;;) {
-            const int c = next(descending);
-            if (c < 0) return -1;
-            const int k = c - c0;
-            if (k >= n_done || !((done[k >> 5] >> (k & 31)) & 1u)) return c;
-        }
-    }
     // The next entry of a list of n chunk numbers (relative to c0) instead.
     __device__ __forceinline__ int next_listed(const int* list, int n) const {
         int k = 0;
@@ -698,12 +697,19 @@ struct ChunkQueue {
 
 constexpr int kSidePre = 1;                       // 16-byte pieces of a side region fetched with the descriptor
 constexpr int kSidePre4 = 2;                      // the same in the sweeps that read nothing but side regions
-constexpr int kDynSmemBytes = kWarps * kChunk * (int)sizeof(float);   // per-warp staging of one chunk's side region
+// Dynamic shared memory: per-warp staging of one slot row of a chunk's side region (stage-2 sweep only; the
+// survivor list and the window counters of the final selection lie over it), then the candidate slots.  (Kept
+// small on purpose: what shared memory takes, the L1 loses, and the first sweep's bandwidth suffers.)
+constexpr int kStageRow = kChunk / kSlots + 8;    // floats of staging per warp: one slot row plus the carried tail
+constexpr int kStageBytes = kWarps * kStageRow * (int)sizeof(float);
+constexpr int kDynSmemBytes = kStageBytes + kSlotCap * (kComp * (int)sizeof(float) + (int)sizeof(int) + 1);
+static_assert(kStageBytes >= kOutCache * 8 + kWinCap * 8, "survivor list and window counters fit over the staging area");
 
 // Positions of a lane's kept elements in the chunk's dense, index-ordered side region.  `mask` has bit
 // 8 j + c set for component c of slot j; chunk order is slot, lane, component.  pos[j] is where this lane's
-// first kept element of slot j goes; the return value is the number of kept elements in the whole chunk.
-__device__ __forceinline__ int side_positions(unsigned mask, int (&pos)[kSlots]) {
+// first kept element of slot j goes, base[j] where slot j's elements begin; the return value is the number of
+// kept elements in the whole chunk.
+__device__ __forceinline__ int side_positions(unsigned mask, int (&pos)[kSlots], int (&base)[kSlots]) {
     static_assert(kSlots == 4, "two packed scans cover four slots");
     const int lane = threadIdx.x & 31;
     const unsigned c01 = __popc(mask & 0xFFu) | (__popc((mask >> 8) & 0xFFu) << 16);
@@ -717,25 +723,25 @@ __device__ __forceinline__ int side_positions(unsigned mask, int (&pos)[kSlots])
     const unsigned t01 = __shfl_sync(kFull, i01, 31), t23 = __shfl_sync(kFull, i23, 31);
     const unsigned e01 = i01 - c01, e23 = i23 - c23;
     const int t0 = t01 & 0xFFFFu, t1 = t01 >> 16, t2 = t23 & 0xFFFFu, t3 = t23 >> 16;
+    base[0] = 0; base[1] = t0; base[2] = t0 + t1; base[3] = t0 + t1 + t2;      // where each slot's entries begin
     pos[0] = e01 & 0xFFFFu;
-    pos[1] = t0 + (e01 >> 16);
-    pos[2] = t0 + t1 + (e23 & 0xFFFFu);
-    pos[3] = t0 + t1 + t2 + (e23 >> 16);
-    return t0 + t1 + t2 + t3;
+    pos[1] = base[1] + (e01 >> 16);
+    pos[2] = base[2] + (e23 & 0xFFFFu);
+    pos[3] = base[3] + (e23 >> 16);
+    return base[3] + t3;
 }
 
 // Chunk descriptor, fetched one chunk ahead so that its loads overlap the current chunk's work.
 struct Desc {
     int c, seg, lo, hi;
     int side_n;          // entries in the chunk's side region (phases that read side regions)
-    unsigned flags;      // this lane's candidate slot flags (P5a only)
     float4 pre[kSidePre];// entries 128 u + 4 lane .. + 3 of the side region, fetched with the descriptor and
                          // without waiting for the count (entries beyond it are ignored)
 };
 
-__device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side, bool with_flags = false) {
+__device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side) {
     Desc d;
-    d.c = c; d.seg = 0; d.lo = 0; d.hi = 0; d.side_n = 0; d.flags = 0u;
+    d.c = c; d.seg = 0; d.lo = 0; d.hi = 0; d.side_n = 0;
     if (c >= 0) {
         d.seg = __ldg(A.chunk_seg + c);
         d.lo = __ldg(A.chunk_start + c);
@@ -746,7 +752,6 @@ __device__ __forceinline__ Desc fetch_desc(const Args& A, int c, bool with_side,
             #pragma unroll
             for (int u = 0; u < kSidePre; ++u) d.pre[u] = __ldcg(side + 32 * u);
         }
-        if (with_flags) d.flags = __ldcg(A.cand + (size_t)c * 32 + (threadIdx.x & 31));
     }
     return d;
 }
@@ -767,25 +772,6 @@ __device__ __forceinline__ SideDesc fetch_side_desc(const Args& A, int c) {
         for (int u = 0; u < kSidePre4; ++u) d.pre[u] = __ldcg(side + 32 * u);
     }
     return d;
-}
-
-// Load only the flagged slots of a full chunk of acc; the others read as zero.
-__device__ __forceinline__ unsigned load_flagged(const float* __restrict__ src, int wb, unsigned flags,
-                                                 float (&v)[kSlots][kComp]) {
-    const int e0 = wb + (threadIdx.x & 31) * kComp;
-    unsigned valid = 0;
-    #pragma unroll
-    for (int j = 0; j < kSlots; ++j) {
-        #pragma unroll
-        for (int c = 0; c < kComp; ++c) v[j][c] = 0.0f;
-        if (flags & (1u << j)) {
-            const F8 q = ld8_evict_last(src + e0 + j * 256);
-            #pragma unroll
-            for (int c = 0; c < kComp; ++c) v[j][c] = q.v[c];
-            valid |= 0xFFu << (8 * j);
-        }
-    }
-    return valid;
 }
 
 // Sum of the per-chunk partials q = first, first + stride, ... < q1, added in that order.  Loads are
@@ -886,11 +872,13 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
 // fitted at once; one shared with other runs is fitted by the run that arrives last.
 // The fitting thread also puts the result into this CTA's own parameter cache, tagged for the phase that
 // uses it next, so that the CTA does not wait for its own publication to come back through L2.
+template <class AfterSweep>
 __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
                                                int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3],
-                                               int stamp_slot) {
+                                               int stamp_slot, const AfterSweep& after_sweep) {
     __threadfence();
     __syncthreads();
+    after_sweep();       // (the CTA's sweep is over and its stores are fenced)
     SIDCO_STAMP(if (threadIdx.x == 0) {                       // this CTA's sweep is over
         const unsigned long long now = global_ns();
         A.cta_ns[4 * blockIdx.x + (stage < 2 ? stage : 2)] = now;
@@ -999,13 +987,22 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     __shared__ double sm_eta[kSegCache];
     __shared__ int sm_ok[kSegCache];
     __shared__ int sm_segk[kSegCache];      // survivors of the run per cached segment
-    __shared__ int sm_oidx[kOutCache];
-    __shared__ float sm_oval[kOutCache];
-    __shared__ unsigned short sm_items[kCoopItems];
-    __shared__ int sm_cseg[kCoopPass], sm_cbase[kCoopPass], sm_ccnt[kCoopPass];
-    __shared__ unsigned sm_done[kCoopChunks / 32];
-    __shared__ int sm_coop_total;
-    __shared__ int sm_any_tau;
+    __shared__ int sm_rest[kThreads];       // chunks (relative to c0) whose survivors the candidates do not cover
+    __shared__ int sm_nrest, sm_nslot, sm_nfetched, sm_nsurv, sm_scan_all;
+    __shared__ int sm_run_e[2];             // first element of the run and one past its last
+    // over the staging area (used after the last sweep that stages): the run's unordered survivor list and the
+    // per-window counters that put it in order
+    int* const sm_oidx = reinterpret_cast<int*>(sm_stage);
+    float* const sm_oval = sm_stage + kOutCache;
+    int* const sm_wcnt = reinterpret_cast<int*>(sm_stage) + 2 * kOutCache;
+    int* const sm_wfill = sm_wcnt + kWinCap;
+    // behind it: the candidate slots (their 8 values, first element, segment of the run); once the survivors are
+    // known, the space of the values takes the ordered list
+    float* const sm_slot_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sm_stage) + kStageBytes);
+    int* const sm_slot_e = reinterpret_cast<int*>(sm_slot_val + kSlotCap * kComp);
+    unsigned char* const sm_slot_seg = reinterpret_cast<unsigned char*>(sm_slot_e + kSlotCap);
+    int* const sm_cidx = reinterpret_cast<int*>(sm_slot_val);
+    float* const sm_cval = sm_slot_val + kOutCache;
     __shared__ unsigned sm_call;
     __shared__ int sm_reszero;
 
@@ -1027,9 +1024,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     [[maybe_unused]] const bool stamper = (cta == 0 && threadIdx.x == 0);
     SIDCO_STAMP(if (stamper) A.ctl->t_ns[0] = global_ns());
     if (threadIdx.x == 0) sm_mloc = 1;
-    if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_any_tau = 0; sm_coop_total = 0; }
+    if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_nrest = 0; sm_nslot = 0; sm_nfetched = 0; sm_nsurv = 0; sm_scan_all = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
-    if (threadIdx.x < kCoopChunks / 32) sm_done[threadIdx.x] = 0u;
+    if (threadIdx.x < 2) sm_run_e[threadIdx.x] = __ldg(A.chunk_start + (threadIdx.x ? c1 : c0));
     // What changes from call to call lives in the workspace (and is advanced by the CTA that finishes the call
     // last, long after every CTA has read it here).  The loads are issued now and their values handed to the
     // CTA after the table loop, whose own loads they overlap.
@@ -1053,7 +1050,6 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             sm_segn[i] = A.seg_n[run_seg_lo + i];
             const float tau = A.seg[run_seg_lo + i].spec_thr;
             sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
-            if (sm_tau[i] > 0.0f && q1 > q0) sm_any_tau = 1;
             sm_ok[i] = 0;
             sm_segk[i] = 0;
         }
@@ -1072,16 +1068,38 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // that precedes their last fit records which slots may hold survivors).  It depends on state the
     // previous call left behind, so every warp and every phase derives the same value.
     auto spec_tau = [&](int seg) -> float {
-        if (seg - R.seg_lo < kSegCache) return sm_tau[seg - R.seg_lo];
-        if (!A.spec_enable || stages_of(seg) > 2) return -1.0f;
-        const float tau = A.seg[seg].spec_thr;
-        return tau > 0.0f ? tau : -1.0f;
+        return seg - R.seg_lo < kSegCache ? sm_tau[seg - R.seg_lo] : -1.0f;     // (candidates carry a cache index)
+    };
+    // A slot (8 elements of one lane) that may hold a survivor: only its place is noted here, inside the sweep;
+    // its values are fetched into shared memory in one asynchronous wave when the CTA's sweep is over.
+    auto list_slot = [&](int e, int seg_i) {
+        const int q = atomicAdd(&sm_nslot, 1);
+        if (q < kSlotCap) { sm_slot_e[q] = e; sm_slot_seg[q] = (unsigned char)seg_i; }
+    };
+    // Start the copies of the slots listed since the last call (all threads; after the sweep's stores are
+    // fenced and the CTA has met).  They complete in the background, behind the fits.
+    auto fetch_slots = [&]() {
+        const int from = sm_nfetched, to = min(sm_nslot, kSlotCap);
+        for (int q = from + (int)threadIdx.x; q < to; q += kThreads) {
+            const float* src = A.residual + sm_slot_e[q];
+            cp_async_16(sm_slot_val + q * kComp, src);
+            cp_async_16(sm_slot_val + q * kComp + 4, src + 4);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) sm_nfetched = to;
+    };
+    // A chunk whose survivors no candidate list will hold: the final selection reads it.
+    auto list_chunk = [&](int c) {
+        if (lane == 0) {
+            const int q = atomicAdd(&sm_nrest, 1);
+            if (q < kThreads) sm_rest[q] = c - c0;
+        }
     };
 
     // ------------------------------------------------------------------ P1
     {
-        int tau_seg = -1;
-        float tau = -1.0f;
+        int tau_seg = -1, seg_m = 1;
+        float tau = 3.4e38f;       // candidate threshold of the chunk's segment (huge: none)
         const bool keep = true;    // ask for L2 residency of the acc lines
         Desc cur = first_desc;
         while (cur.c >= 0) {
@@ -1091,10 +1109,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             const int e0 = wb + lane * kComp;
             if (cur.seg != tau_seg) {
                 tau_seg = cur.seg;
-                const int m = stages_of(cur.seg);
-                tau = m == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments flag in P3
+                seg_m = stages_of(cur.seg);
+                const float t = seg_m == 1 ? spec_tau(cur.seg) : -1.0f;    // two-stage segments record in P3
+                tau = t > 0.0f ? t : 3.4e38f;
             }
-            unsigned flags = 0;
 
             double s1 = 0.0, s2 = 0.0, prod = 1.0;
             int esum = 0, nnz = 0;
@@ -1135,11 +1153,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             big = fmaxf(big, fabsf(a));
                         }
                         st8_res(A.residual + e0 + (b + j) * 256, r8[j], keep);
-                        flags |= (unsigned)(big >= tau) << (b + j);
+                        if (big >= tau) list_slot(e0 + (b + j) * 256, cur.seg - R.seg_lo);
                     }
                 }
-                if (tau > 0.0f) A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
+                if (seg_m == 1 && !(tau < 3.0e38f)) list_chunk(c);        // single stage, no candidates recorded
             } else {
+                if (seg_m == 1) list_chunk(c);
                 #pragma unroll 1
                 for (int j = 0; j < kSlots; ++j) {
                     const int e = e0 + j * 256;
@@ -1190,7 +1209,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             cur = nxt;
         }
     }
-    arrive_and_fit(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6);
+    arrive_and_fit(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6, fetch_slots);
     if (threadIdx.x == 0) sm_next = 0;
     __syncthreads();
     const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
@@ -1217,7 +1236,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     const bool flag_chunk = tau2 > 0.0f && vec_ok && lo == wb && hi == wb + kChunk;
                     // (elements outside the chunk read as zero and the threshold is never negative, so they
                     // pass no strict compare)
-                    unsigned mask = 0, flags = 0;
+                    unsigned mask = 0;
                     double sy = 0.0, sy2 = 0.0;
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j) {
@@ -1233,11 +1252,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                                 mask |= 1u << (8 * j + cc);
                             }
                         }
-                        flags |= (unsigned)(big >= tau2) << j;
+                        if (flag_chunk && big >= tau2) list_slot(wb + lane * kComp + j * 256, cur.seg - R.seg_lo);
                     }
-                    if (flag_chunk) {
-                        A.cand[(size_t)c * 32 + lane] = (unsigned char)flags;
-                    } else {
+                    if (!flag_chunk) {
+                        list_chunk(c);
                         // The side region also takes the entries equal to eta_1: they are no exceedances (the
                         // statistics above leave them out), but if no later stage raises the threshold
                         // (eta_M = eta_1, e.g. a segment of equal magnitudes) the final rule |x| >= eta_M selects them.
@@ -1251,22 +1269,30 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                                     if (fabsf(v[j][cc]) == sv.thr_gt) keep_mask |= 1u << (8 * j + cc);
                             keep_mask &= valid;
                         }
-                        // The kept values go to the chunk's side region dense and in index order: every lane puts its
-                        // own at their positions in the warp's shared-memory staging area, and the warp copies the
-                        // area out with 16-byte stores.
-                        int pos[kSlots];
-                        const int kept = side_positions(keep_mask, pos);
-                        float* stage = sm_stage + warp * kChunk;
+                        // The kept values go to the chunk's side region dense and in index order, one slot row at a
+                        // time: every lane puts its own at their positions in the warp's shared-memory staging area,
+                        // and the warp copies the area out with 16-byte stores.  A row rarely ends on a 16-byte
+                        // boundary: its last few values are carried to the front of the next row's staging.
+                        int pos[kSlots], base[kSlots];
+                        const int kept = side_positions(keep_mask, pos, base);
+                        float* stage = sm_stage + warp * kStageRow;
+                        float4* side = reinterpret_cast<float4*>(A.side_val + (size_t)c * kChunk);
                         #pragma unroll
                         for (int j = 0; j < kSlots; ++j) {
-                            int q = pos[j];
+                            const int a0 = base[j] & ~3;                   // first position this round writes
+                            const int end = j + 1 < kSlots ? base[j + 1] : kept;
+                            int q = pos[j] - a0;
                             #pragma unroll
                             for (int cc = 0; cc < kComp; ++cc)
                                 if ((keep_mask >> (8 * j + cc)) & 1u) stage[q++] = v[j][cc];
+                            __syncwarp();
+                            const int n4 = (end - a0 + 3) >> 2;
+                            for (int q4 = lane; q4 < n4; q4 += 32) side[(a0 >> 2) + q4] = reinterpret_cast<const float4*>(stage)[q4];
+                            const int tail = end & 3;
+                            const float carry = lane < tail ? stage[(end & ~3) - a0 + lane] : 0.0f;
+                            __syncwarp();
+                            if (lane < tail) stage[lane] = carry;
                         }
-                        __syncwarp();
-                        float4* side = reinterpret_cast<float4*>(A.side_val + (size_t)c * kChunk);
-                        for (int q = lane; 4 * q < kept; q += 32) side[q] = reinterpret_cast<const float4*>(stage)[q];
                         __syncwarp();
                         if (lane == 0) A.side_cnt[c] = kept;
                         A.side_mask[(size_t)c * 32 + lane] = keep_mask;
@@ -1281,7 +1307,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 cur = nxt;
             }
         }
-        arrive_and_fit(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8);
+        arrive_and_fit(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8, fetch_slots);
         if (threadIdx.x == 0) sm_next = 0;
         __syncthreads();
         SIDCO_STAMP(if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns());
@@ -1331,349 +1357,210 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     cur = nxt;
                 }
             }
-            arrive_and_fit(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10);
+            arrive_and_fit(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10, [] {});
             if (threadIdx.x == 0) sm_next = 0;
             __syncthreads();
             SIDCO_STAMP(if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns());
         }
     }
 
-    // ------------------------------------------------------------------ P5a: stage survivors per chunk
-    int warp_total = 0;
+    // ------------------------------------------------------------------ P5: the final selection
+    // Two ways.  (A) The usual one keeps everything in shared memory: the candidates recorded by the sweeps
+    // are compared with the final thresholds, the few chunks without candidates (ragged chunks, segments with
+    // three or more stages, segments whose candidate threshold turned out too high) are read by the warps, and
+    // all survivors of the run end up in one unordered shared-memory list that is then put in index order
+    // (grouped by 1024-element window with a counting pass, ranked inside a window by comparison), written to
+    // its final place and zeroed in the residual.  Nothing is modified before the list is known to fit.
+    // (B) Otherwise (many survivors per run, e.g. delta = 0.1) the warps go through all chunks of the run,
+    // stage each chunk's survivors in order in the chunk's staging region, and the placement goes through a
+    // block scan over the chunk counts.
+    publish_params(A, R, 0, -1, 100);          // one thread per segment waits (bounded) for its last threshold
+    cp_async_wait_all();                       // this thread's share of the candidate slots has arrived
+    __syncthreads();
+    const bool cand_overflow = sm_nslot > kSlotCap;
+    // the recorded candidates of cached segment i contain all its survivors among the chunks that recorded some
+    auto seg_cand_ok = [&](int i) -> bool { return !cand_overflow && sm_tau[i] > 0.0f && R.thr[i] >= sm_tau[i]; };
+    const int run_e0 = sm_run_e[0], run_e1 = sm_run_e[1];
+    const int win0 = run_e0 >> 10;
+    const int n_win = c1 > c0 ? ((run_e1 - 1) >> 10) - win0 + 1 : 0;
+    bool path_a = run_n_seg <= kSegCache && n_win <= kWinCap;
+    int cta_count = 0;
 
-    // Block-wide pass over the full chunks that carry candidate flags (the common case for one- and two-stage
-    // segments).  The flagged slots of up to kCoopPass chunks are listed in shared memory in chunk order
-    // (chunk, slot, lane) and fetched two per thread in one wave, so the whole run costs a few memory round
-    // trips instead of one per chunk and warp.  Listing and fetching need no threshold: they are issued before
-    // the CTA waits for the fits of its segments, and overlap that wait.  Once a segment's threshold is known
-    // its flags either proved valid (eta >= tau: survivors are taken from the fetched slots, a block scan over
-    // the per-slot counts giving each its place in the chunk's staging region, and the chunk is marked in
-    // sm_done) or not (the fetched slots are dropped).  The warp loop below takes every chunk not marked
-    // (ragged chunks, invalid flags, side regions).
-    // Survivors found by this pass are also kept in shared memory at their rank within the run (the passes
-    // and their scans go through the run in order).  If the pass ends up covering every chunk of the run and
-    // the survivors fit, the final placement copies them from there instead of reading the staging regions.
-    bool published = false;
-    int coop_n = 0;                       // leading chunks of the run this pass covers
-    int coop_done = 0;                    // chunks it took
-    int before_pass = 0;                  // survivors found by the passes before the current one
-    // (A run of at most one chunk per warp goes straight to the warp loop: its two round trips beat the pass.)
-    if (vec_ok && sm_any_tau && c1 - c0 > kWarps) {
-        coop_n = min(c1 - c0, kCoopChunks);
-        // Threshold of a chunk's segment once its last stage is fitted; true if the chunk's listed slots
-        // hold all its survivors.  `tag` is the segment's cache index, plus kAllSlots if all of the chunk's
-        // slots were listed (then no flags are involved).
-        constexpr int kAllSlots = 1 << 16;
-        auto seg_thr = [&](int tag, float& thr) -> bool {
-            const int i = tag & (kAllSlots - 1);
-            long long spins = 0;
-            while (R.ok[i] != 100) {                       // published by a thread of this CTA
-                if (++spins > A.spin_limit) { atomicExch(&A.ctl->timeout, 1); break; }
-                __nanosleep(20);
-            }
-            __threadfence_block();
-            thr = R.thr[i];
-            return (tag & kAllSlots) || thr >= sm_tau[i];
-        };
-        for (int base = 0; base < coop_n; base += kCoopPass) {
-            // two threads per chunk: this one lists slots jj and jj + 1 of all 32 lanes
-            const int cl = threadIdx.x >> 1;
-            const int k = base + cl;
-            const int c = c0 + k;
-            const int jj = (threadIdx.x & 1) * 2;
-            // Chunks taken here: full chunks that carry flags, and ragged chunks made of whole slots, all of
-            // which are listed (a run has few of them).  Both need acc as the source of the final selection,
-            // i.e. a segment with at most two stages.
-            int seg_i = -1;                       // see seg_thr
-            unsigned long long bits = 0ull;       // bit 32 (j - jj) + lane: slot j of that lane is listed
-            uint4 fa = make_uint4(0u, 0u, 0u, 0u), fb = fa;      // the chunk's 32 flag bytes
-            if (k < coop_n) {
-                // (loaded whether or not the chunk turns out to carry flags, so that this costs one round
-                // trip, not two)
-                const uint4* fp = reinterpret_cast<const uint4*>(A.cand + (size_t)c * 32);
-                fa = __ldcg(fp);
-                fb = __ldcg(fp + 1);
-                const int seg = __ldg(A.chunk_seg + c);
-                const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
-                const int i = seg - R.seg_lo;
-                if (i < kSegCache && sm_meff[i] <= 2) {
-                    const int wb = lo & ~(kChunk - 1);
-                    if (lo == wb && hi == wb + kChunk) {
-                        if (sm_tau[i] > 0.0f) seg_i = i;
-                    } else if (((lo | hi) & (kComp - 1)) == 0) {
-                        seg_i = i | kAllSlots;
-                        #pragma unroll
-                        for (int dj = 0; dj < 2; ++dj) {
-                            const int row = wb + (jj + dj) * 256;                     // slot row: 32 lanes x 8 elements
-                            const int a = max(lo, row), b = min(hi, row + 256);
-                            if (b > a) {
-                                const int l0 = (a - row) / kComp, nl = (b - a) / kComp;  // lanes l0 .. l0 + nl - 1
-                                const unsigned m = (nl >= 32 ? kFull : ((1u << nl) - 1u)) << l0;
-                                bits |= (unsigned long long)m << (32 * dj);
-                            }
-                        }
-                    }
-                }
-            }
-            if (seg_i >= 0 && !(seg_i & kAllSlots)) {
-                // bit j of each of a word's four bytes, gathered into four adjacent bits
-                auto pick = [](unsigned w, int j) -> unsigned { return ((((w >> j) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu; };
-                auto lanes = [&](int j) -> unsigned {
-                    return pick(fa.x, j) | (pick(fa.y, j) << 4) | (pick(fa.z, j) << 8) | (pick(fa.w, j) << 12) |
-                           (pick(fb.x, j) << 16) | (pick(fb.y, j) << 20) | (pick(fb.z, j) << 24) | (pick(fb.w, j) << 28);
-                };
-                bits = (unsigned long long)lanes(jj) | ((unsigned long long)lanes(jj + 1) << 32);
-            }
-            int total = 0;
-            int off = block_exscan(__popcll(bits), sm_warp, total);
-            const bool listed = total <= kCoopItems;       // same for every thread; otherwise the warp loop takes these chunks
-            if (listed) {
-                #pragma unroll
-                for (int dj = 0; dj < 2; ++dj) {
-                    unsigned m = (unsigned)(bits >> (32 * dj));
-                    const int head = (cl << 7) | ((jj + dj) << 5);
-                    if (seg_i >= 0 && (seg_i & kAllSlots)) {        // a ragged chunk's row: one run of lanes
-                        const int l0 = __ffs(m) - 1, nl = __popc(m);
-                        for (int q = 0; q < nl; ++q) sm_items[off + q] = (unsigned short)(head | (l0 + q));
-                        off += nl;
-                    } else {
-                        while (m) {
-                            const int q = __ffs(m) - 1;
-                            m &= m - 1u;
-                            sm_items[off++] = (unsigned short)(head | q);
-                        }
-                    }
-                }
-                if ((threadIdx.x & 1) == 0) { sm_cseg[cl] = seg_i; sm_ccnt[cl] = 0; }
-            }
-            __syncthreads();
-            if (!listed) continue;
-            int carry = 0;                    // survivors of the rounds before this one
-            for (int r0 = 0; r0 < total; r0 += 2 * kThreads) {
-                F8 x[2];
-                int e[2], icl[2], clo[2];
-                unsigned m8[2];
-                #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int r = r0 + 2 * (int)threadIdx.x + u;
-                    e[u] = -1; icl[u] = 0; clo[u] = 0; m8[u] = 0u;
-                    if (r < total) {
-                        const int it = sm_items[r];
-                        icl[u] = it >> 7;
-                        clo[u] = __ldg(A.chunk_start + c0 + base + icl[u]);       // staging region of the chunk starts here
-                        e[u] = (clo[u] & ~(kChunk - 1)) + ((it >> 5) & 3) * 256 + (it & 31) * kComp;
-                        x[u] = ld8_evict_last(A.residual + e[u]);
-                    }
-                }
-                // the fits are waited for only now, with the slot loads in flight
-                if (!published) { publish_params(A, R, 0, -1, 100); published = true; }
-                #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    float t;
-                    if (e[u] >= 0 && seg_thr(sm_cseg[icl[u]], t)) {
-                        #pragma unroll
-                        for (int cc = 0; cc < kComp; ++cc)
-                            if (fabsf(x[u].v[cc]) >= t) m8[u] |= 1u << cc;
-                    }
-                }
-                const int n0 = __popc(m8[0]), n1 = __popc(m8[1]);
-                int round_total = 0;
-                const int ex = carry + block_exscan(n0 + n1, sm_warp, round_total);
-                #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int r = r0 + 2 * (int)threadIdx.x + u;
-                    // the first listed slot of a chunk records how many survivors precede the chunk
-                    if (e[u] >= 0 && (r == 0 || (sm_items[r - 1] >> 7) != icl[u])) sm_cbase[icl[u]] = ex + (u ? n0 : 0);
-                }
-                __syncthreads();
-                #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    if (m8[u]) {
-                        int pos = clo[u] + ex + (u ? n0 : 0) - sm_cbase[icl[u]];
-                        int rank = before_pass + ex + (u ? n0 : 0);
-                        #pragma unroll
-                        for (int cc = 0; cc < kComp; ++cc) {
-                            if (m8[u] & (1u << cc)) {
-                                A.stage_idx[pos] = e[u] + cc;
-                                A.stage_val[pos] = x[u].v[cc];
-                                A.residual[e[u] + cc] = 0.0f;
-                                if (rank < kOutCache) { sm_oidx[rank] = e[u] + cc; sm_oval[rank] = x[u].v[cc]; }
-                                ++pos;
-                                ++rank;
-                            }
-                        }
-                        atomicAdd(&sm_ccnt[icl[u]], u ? n1 : n0);
-                    }
-                }
-                carry += round_total;
-            }
-            if (!published) { publish_params(A, R, 0, -1, 100); published = true; }
-            __syncthreads();
-            bool took = false;
-            if (threadIdx.x < kCoopPass) {            // whole warps: one thread per chunk of the pass
-                const int k2 = base + (int)threadIdx.x;
-                int key = -1, cnt = 0;
-                float t;
-                if (k2 < coop_n && sm_cseg[threadIdx.x] >= 0 && seg_thr(sm_cseg[threadIdx.x], t)) {
-                    took = true;
-                    atomicOr(&sm_done[k2 >> 5], 1u << (k2 & 31));
-                    cnt = sm_ccnt[threadIdx.x];
-                    A.chunk_cnt[c0 + k2] = cnt;
-                    if (cnt) key = sm_cseg[threadIdx.x] & (kAllSlots - 1);
-                }
-                // one counter update per segment and warp (the pass takes cached segments only)
-                const unsigned peers = __match_any_sync(kFull, key);
-                const int sum = __reduce_add_sync(peers, cnt);
-                if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&sm_segk[key], sum);
-            }
-            if (threadIdx.x == 0) sm_coop_total += carry;
-            before_pass += carry;
-            coop_done += __syncthreads_count(took);
-        }
-        if (threadIdx.x == 0) warp_total += sm_coop_total;
-    }
-    if (!published) publish_params(A, R, 0, -1, 100);
-    // The chunks left for the warp loop, if the pass above covered the whole run: listed, so that the warps
-    // do not take turns at the queue for every chunk already done (few are left).
-    int n_rest = -1;                      // < 0: no list, the loop goes through the queue and skips the chunks done
-    if (coop_n == c1 - c0 && coop_done == coop_n) {
-        n_rest = 0;                       // nothing left (the usual case)
-    } else if (coop_n == c1 - c0 && coop_n > 0) {
-        for (int k = threadIdx.x; k < coop_n; k += kThreads)
-            if (!((sm_done[k >> 5] >> (k & 31)) & 1u)) {
-                const int p = atomicAdd(&sm_count[0], 1);
-                if (p < kThreads) sm_list[p] = k;
-            }
-        __syncthreads();
-        n_rest = sm_count[0];
-        __syncthreads();
-        if (threadIdx.x == 0) sm_count[0] = 0;
-        if (n_rest > kThreads) n_rest = -1;          // more than the list holds
-    }
-    const bool place_from_smem = n_rest == 0 && before_pass <= kOutCache;
-    // survivors of a segment found by the warp loop: into the run's shared-memory count if the segment has one
-    auto add_seg_count = [&](int seg, int n) {
-        const int i = seg - R.seg_lo;
-        if (i < kSegCache) atomicAdd(&sm_segk[i], n);
-        else atomicAdd(&A.seg[seg].k_acc, n);
-    };
-    auto next_chunk = [&]() -> int {
-        return n_rest >= 0 ? queue.next_listed(sm_list, n_rest) : queue.next_undone(!p1_desc, sm_done, coop_n);
+    // Survivor into the run's unordered list (path A).
+    auto append = [&](int e, float val, int seg_i) {
+        const int sp = atomicAdd(&sm_nsurv, 1);
+        if (sp < kOutCache) { sm_oidx[sp] = e; sm_oval[sp] = val; }
+        atomicAdd(&sm_wcnt[(e >> 10) - win0], 1);
+        atomicAdd(&sm_segk[seg_i], 1);
     };
 
-    {
+    // The warps' pass over chunks.  list_n >= 0: the chunks sm_rest[0 .. list_n); < 0: all chunks of the run,
+    // skipping (if skip_covered) those whose survivors the candidates already gave.  to_list: survivors go to the
+    // shared-memory list and nothing is modified; otherwise they are staged per chunk and zeroed in the residual.
+    auto warp_pass = [&](int list_n, bool skip_covered, bool to_list) -> int {
+        int total = 0;
         SegView sv;
-        bool seg_from_side = false, seg_flagged = false, seg_two_flagged = false;
-        int seg_count = 0;       // survivors of sv.seg not yet added to its counter
+        bool seg_from_side = false, seg_cand = false, seg_covered = false;
+        int seg_count = 0;       // survivors of sv.seg not yet added to its counter (staging mode)
         const bool any_side = M_max_eff >= 2;      // some chunk of this run may have a side region
-        Desc cur = fetch_desc(A, n_rest == 0 ? -1 : next_chunk(), any_side, true);
+        auto next_chunk = [&]() -> int { return list_n >= 0 ? queue.next_listed(sm_rest, list_n) : queue.next(!p1_desc); };
+        auto add_seg_count = [&](int seg, int n) {
+            const int i = seg - R.seg_lo;
+            if (i < kSegCache) atomicAdd(&sm_segk[i], n);
+            else atomicAdd(&A.seg[seg].k_acc, n);
+        };
+        Desc cur = fetch_desc(A, list_n == 0 ? -1 : next_chunk(), any_side);
         while (cur.c >= 0) {
-            const Desc nxt = fetch_desc(A, next_chunk(), any_side, true);
+            const Desc nxt = fetch_desc(A, next_chunk(), any_side);
             if (cur.seg != sv.seg) {
                 if (seg_count && lane == 0) add_seg_count(sv.seg, seg_count);
                 seg_count = 0;
                 view_load(A, R, sv, cur.seg, 0, -1, 100, cap);
-                // multi-stage segments keep their exceedances in the side region; single-stage ones
-                // have valid candidate flags if the candidate threshold proved low enough
-                const float tau = spec_tau(cur.seg);
-                seg_two_flagged = sv.M_eff == 2 && tau > 0.0f;      // P3 wrote flags for its full chunks
+                const int i = cur.seg - R.seg_lo;
+                seg_cand = spec_tau(cur.seg) > 0.0f;               // its full chunks recorded candidates
                 seg_from_side = sv.M_eff >= 2;
-                seg_flagged = tau > 0.0f && sv.thr_ge >= tau;
+                seg_covered = i < kSegCache && seg_cand && seg_cand_ok(i);
             }
-            const int c = cur.c, lo = cur.lo;
+            const int c = cur.c, lo = cur.lo, hi = cur.hi;
             const int wb = lo & ~(kChunk - 1);
-            // a full chunk of a flag-carrying two-stage segment has no side region: it is read from acc,
-            // through its flags if they proved valid, in full otherwise
-            const bool from_side = seg_from_side && !(seg_two_flagged && vec_ok && lo == wb && cur.hi == wb + kChunk);
+            const bool cand_chunk = seg_cand && vec_ok && lo == wb && hi == wb + kChunk;
             int cnt = 0;
-            if (from_side) {
-                // The side region is a dense list in index order.  Lanes read it 16 bytes at a time; a survivor is
-                // known by its position in the list, and the lane that holds the element at that position (found
-                // through the per-lane masks, only for chunks that have a survivor at all) marks it in a mask of
-                // the chunk's own layout, which gives the survivors their indices and their order.
-                const int n = cur.side_n;
-                const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
+            if (!(skip_covered && cand_chunk && seg_covered)) {
                 unsigned surv = 0;
-                int pos[kSlots];
-                unsigned smask = 0;
-                bool have_pos = false;
-                auto take = [&](const float4& x, int first) {
-                    const float a[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
-                    unsigned hit = 0;
-                    #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (first + u < n && a[u] >= sv.thr_ge) hit |= 1u << u;
-                    unsigned any = __ballot_sync(kFull, hit != 0);
-                    if (any == 0) return;
-                    if (!have_pos) {
-                        smask = __ldcg(A.side_mask + (size_t)c * 32 + lane);
-                        side_positions(smask, pos);
-                        have_pos = true;
-                    }
-                    while (any) {
-                        const int src = __ffs(any) - 1;
-                        any &= any - 1u;
-                        unsigned h = __shfl_sync(kFull, hit, src);
-                        const int base = __shfl_sync(kFull, first, src);
-                        while (h) {
-                            const int p = base + __ffs(h) - 1;         // position in the list
-                            h &= h - 1u;
-                            // the lane whose elements of some slot cover position p
-                            #pragma unroll
-                            for (int j = 0; j < kSlots; ++j) {
-                                const unsigned byte = (smask >> (8 * j)) & 0xFFu;
-                                const int r = p - pos[j];
-                                if (r >= 0 && r < __popc(byte)) surv |= (1u << (8 * j)) << (__fns(byte, 0, r + 1));
+                float v[kSlots][kComp];
+                // a full chunk of a candidate-recording two-stage segment has no side region: it is read from acc
+                const bool from_side = seg_from_side && !cand_chunk;
+                if (from_side) {
+                    // The side region is a dense list in index order.  Lanes read it 16 bytes at a time; a survivor
+                    // is known by its position in the list, and the lane that holds the element at that position
+                    // (found through the per-lane masks, only for chunks that have a survivor at all) marks it
+                    // in a mask of the chunk's own layout, which gives the survivors their indices and order.
+                    const int n = cur.side_n;
+                    const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
+                    int pos[kSlots], base[kSlots];
+                    unsigned smask = 0;
+                    bool have_pos = false;
+                    auto take = [&](const float4& x, int first) {
+                        const float a[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
+                        unsigned hit = 0;
+                        #pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (first + u < n && a[u] >= sv.thr_ge) hit |= 1u << u;
+                        unsigned any = __ballot_sync(kFull, hit != 0);
+                        if (any == 0) return;
+                        if (!have_pos) {
+                            smask = __ldcg(A.side_mask + (size_t)c * 32 + lane);
+                            side_positions(smask, pos, base);
+                            have_pos = true;
+                        }
+                        while (any) {
+                            const int src = __ffs(any) - 1;
+                            any &= any - 1u;
+                            unsigned h = __shfl_sync(kFull, hit, src);
+                            const int base = __shfl_sync(kFull, first, src);
+                            while (h) {
+                                const int p = base + __ffs(h) - 1;         // position in the list
+                                h &= h - 1u;
+                                // the lane whose elements of some slot cover position p
+                                #pragma unroll
+                                for (int j = 0; j < kSlots; ++j) {
+                                    const unsigned byte = (smask >> (8 * j)) & 0xFFu;
+                                    const int r = p - pos[j];
+                                    if (r >= 0 && r < __popc(byte)) surv |= (1u << (8 * j)) << (__fns(byte, 0, r + 1));
+                                }
                             }
                         }
-                    }
-                };
-                #pragma unroll
-                for (int u = 0; u < kSidePre; ++u) take(cur.pre[u], 128 * u + 4 * lane);
-                for (int t = kSidePre; 128 * t < n; ++t) take(__ldcg(side + 32 * t), 128 * t + 4 * lane);
-                if (__ballot_sync(kFull, surv != 0)) {
-                    const int e0 = wb + lane * kComp;
-                    cnt = ordered_emit(surv, lo, [&](int p, int j, int cc) {
-                        const int e = e0 + j * 256 + cc;
-                        A.stage_idx[p] = e;
-                        A.stage_val[p] = __ldcg(A.residual + e);
-                        A.residual[e] = 0.0f;
-                    });
-                }
-            } else {
-                const int hi = cur.hi;
-                const bool flagged = seg_flagged && vec_ok && lo == wb && hi == wb + kChunk;
-                if (!flagged) ++resweep;
-                if (!(flagged && __ballot_sync(kFull, cur.flags != 0) == 0)) {
-                    float v[kSlots][kComp];
-                    const unsigned valid = flagged ? load_flagged(A.residual, wb, cur.flags, v)
-                                                   : load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
-                    unsigned mask = 0;
+                    };
+                    #pragma unroll
+                    for (int u = 0; u < kSidePre; ++u) take(cur.pre[u], 128 * u + 4 * lane);
+                    for (int t = kSidePre; 128 * t < n; ++t) take(__ldcg(side + 32 * t), 128 * t + 4 * lane);
+                } else {
+                    ++resweep;
+                    const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j)
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc)
-                            if (fabsf(v[j][cc]) >= sv.thr_ge) mask |= 1u << (8 * j + cc);
-                    mask &= valid;
-                    if (__ballot_sync(kFull, mask != 0)) {
-                        const int e0 = wb + lane * kComp;
-                        cnt = ordered_emit(mask, lo, [&](int p, int j, int cc) {
+                            if (fabsf(v[j][cc]) >= sv.thr_ge) surv |= 1u << (8 * j + cc);
+                    surv &= valid;
+                }
+                if (__ballot_sync(kFull, surv != 0)) {
+                    const int e0 = wb + lane * kComp;
+                    if (to_list) {
+                        const int seg_i = cur.seg - R.seg_lo;
+                        unsigned m = surv;
+                        while (m) {
+                            const int bit = __ffs(m) - 1;
+                            m &= m - 1u;
+                            const int e = e0 + (bit >> 3) * 256 + (bit & 7);
+                            append(e, __ldcg(A.residual + e), seg_i);
+                        }
+                    } else {
+                        cnt = ordered_emit(surv, lo, [&](int p, int j, int cc) {
                             const int e = e0 + j * 256 + cc;
                             A.stage_idx[p] = e;
-                            A.stage_val[p] = v[j][cc];
+                            A.stage_val[p] = from_side ? __ldcg(A.residual + e) : v[j][cc];
                             A.residual[e] = 0.0f;
                         });
                     }
                 }
             }
-            if (lane == 0) A.chunk_cnt[c] = cnt;
-            seg_count += cnt;
-            warp_total += cnt;
+            if (!to_list) {
+                if (lane == 0) A.chunk_cnt[c] = cnt;
+                seg_count += cnt;
+                total += cnt;
+            }
             cur = nxt;
         }
         if (seg_count && lane == 0) add_seg_count(sv.seg, seg_count);
+        return total;
+    };
+
+    if (path_a) {
+        for (int w = threadIdx.x; w < n_win; w += kThreads) { sm_wcnt[w] = 0; sm_wfill[w] = 0; }
+        // a segment that recorded candidates which turned out unusable: its chunks are in no list
+        for (int i = threadIdx.x; i < R.n_seg; i += kThreads)
+            if (sm_q1[i] > sm_q0[i] && sm_tau[i] > 0.0f && !seg_cand_ok(i)) sm_scan_all = 1;
+        __syncthreads();
+        const int n_slot = min(sm_nslot, kSlotCap);
+        for (int q = threadIdx.x; q < n_slot; q += kThreads) {
+            const int i = sm_slot_seg[q];
+            if (seg_cand_ok(i)) {
+                const float thr = R.thr[i];
+                const int e = sm_slot_e[q];
+                #pragma unroll
+                for (int cc = 0; cc < kComp; ++cc) {
+                    const float val = sm_slot_val[q * kComp + cc];
+                    if (fabsf(val) >= thr) append(e + cc, val, i);
+                }
+            }
+        }
+        const bool scan_all = sm_scan_all != 0 || sm_nrest > kThreads;
+        warp_pass(scan_all ? -1 : sm_nrest, true, true);
+        __syncthreads();
+        cta_count = sm_nsurv;
+        if (cta_count > kOutCache) {
+            // too many for the list: start over the other way (nothing has been modified yet)
+            path_a = false;
+            for (int i = threadIdx.x; i < kSegCache; i += kThreads) sm_segk[i] = 0;
+            if (threadIdx.x == 0) sm_next = 0;
+            __syncthreads();
+        }
     }
-    if (lane == 0) { sm_warp[warp] = warp_total; if (resweep) atomicAdd(&sm_resweep, resweep); }
+    if (!path_a) {
+        const int warp_total = warp_pass(-1, false, false);
+        if (lane == 0) sm_warp[warp] = warp_total;
+        __syncthreads();
+        if (warp == 0) {
+            int x = sm_warp[lane];
+            #pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(kFull, x, o);
+            if (lane == 0) sm_base = x;
+        }
+        __syncthreads();
+        cta_count = sm_base;
+    }
+    if (lane == 0 && resweep) atomicAdd(&sm_resweep, resweep);
     __syncthreads();
     SIDCO_STAMP(if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns());
     SIDCO_STAMP(if (stamper) A.ctl->t_ns[12] = global_ns());
@@ -1684,18 +1571,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // above it poll for their output base; a segment's total count comes out of the atomic by which the last of
     // its runs reports (SegDev::k_arr).  Neither needs a fence: the words carry everything their readers use,
     // and what this CTA stored for its own placement it reads back itself.
-    int cta_count = 0;
-    if (warp == 0) {
-        int x = sm_warp[lane];
-        #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(kFull, x, o);
-        if (lane == 0) {
-            st_relaxed_u64(&A.cta_pub[cta], ((unsigned long long)call_id << 32) | (unsigned)x);
-            sm_base = x;
-        }
-    }
-    __syncthreads();
-    cta_count = sm_base;
+    if (threadIdx.x == 0) st_relaxed_u64(&A.cta_pub[cta], ((unsigned long long)call_id << 32) | (unsigned)cta_count);
 
     // Per-segment end of call: counts, last stage count, adaptation (Algorithm 1, Adapt_Stages), next call's
     // candidate threshold.  Done by the thread whose report completes the segment; reads nothing that another
@@ -1770,8 +1646,28 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             seg_finish(s, f.M_eff, 0, f.thr);
         }
 
-    // ------------------------------------------------------------------ P5b: final positions
+    // ------------------------------------------------------------------ placement
     {
+        // In path A the list is put in index order while the counts of the runs below are on their way: a
+        // counting pass groups the survivors by window, then every survivor is ranked inside its window.
+        if (path_a && cta_count > 0) {
+            // window bases: exclusive prefix sums of the window counts, two windows per thread
+            const int w2 = 2 * (int)threadIdx.x;
+            const int a0 = w2 < n_win ? sm_wcnt[w2] : 0, a1 = w2 + 1 < n_win ? sm_wcnt[w2 + 1] : 0;
+            int total = 0;
+            const int ex = block_exscan(a0 + a1, sm_warp, total);
+            __syncthreads();
+            if (w2 < n_win) sm_wcnt[w2] = ex;
+            if (w2 + 1 < n_win) sm_wcnt[w2 + 1] = ex + a0;
+            __syncthreads();
+            for (int q = threadIdx.x; q < cta_count; q += kThreads) {
+                const int e = sm_oidx[q], w = (e >> 10) - win0;
+                const int slot = sm_wcnt[w] + atomicAdd(&sm_wfill[w], 1);
+                sm_cidx[slot] = e;                       // (the candidate arrays are free by now)
+                sm_cval[slot] = sm_oval[q];
+            }
+            __syncthreads();
+        }
         // survivors of the runs below this one: each run's word is polled (bounded) until it carries this
         // call's number; summed by one warp (a grid has a few hundred CTAs at most)
         if (warp == 0) {
@@ -1794,15 +1690,19 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         SIDCO_STAMP(if (stamper) A.ctl->t_ns[4] = global_ns());
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
-        if (place_from_smem) {
-            // every survivor of the run sits in shared memory at its rank
-            for (int r = threadIdx.x; r < cta_count; r += kThreads) {
-                A.out_idx[run_base + r] = sm_oidx[r];
-                A.out_val[run_base + r] = sm_oval[r];
+        if (path_a) {
+            for (int q = threadIdx.x; q < cta_count; q += kThreads) {
+                const int e = sm_cidx[q], w = (e >> 10) - win0;
+                const int g0 = sm_wcnt[w], g1 = g0 + sm_wfill[w];
+                int rank = 0;
+                for (int t = g0; t < g1; ++t) rank += sm_cidx[t] < e;
+                A.out_idx[run_base + g0 + rank] = e;
+                A.out_val[run_base + g0 + rank] = sm_cval[q];
+                A.residual[e] = 0.0f;
             }
         }
-        // otherwise: chunk bases by a block-wide exclusive scan, kThreads chunks at a time
-        for (int pass = c0; pass < c1 && cta_count > 0 && !place_from_smem; pass += kThreads) {
+        // path B: chunk bases by a block-wide exclusive scan, kThreads chunks at a time
+        for (int pass = c0; pass < c1 && cta_count > 0 && !path_a; pass += kThreads) {
             const int c = pass + (int)threadIdx.x;
             const int cnt = c < c1 ? ld_cg(A.chunk_cnt + c) : 0;
             int incl = cnt;
