@@ -60,6 +60,8 @@ extern "C" {
 #define SIDCO_ST_DEGENERATE 2   /* a fit took one of its degenerate-case rules */
 #define SIDCO_ST_ALL_ZERO   4   /* every magnitude is zero: nothing is selected */
 #define SIDCO_ST_TIMEOUT    8   /* a bounded wait inside the kernel ran out; results are invalid */
+#define SIDCO_ST_BOUNDS     16  /* -DSIDCO_BOUNDS_CHECK builds only: an index fell outside its buffer and the access
+                                   was skipped; results are invalid */
 
 typedef struct sidco_seg_debug {
     int32_t M_used;                       /* stages used by the last call (after the cap for delta) */
@@ -250,6 +252,12 @@ int sidco_get_phase_times(const float* residual, double* us_out);
  * 1 stage-2 sweep, 2 last refit sweep, 3 survivor staging).  Writes at most max_ctas rows and returns
  * the number of rows written (>= 0) or an error code (< 0).  Synchronises the device. */
 int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_ctas);
+
+/* (Profile builds only.)  How the final selection of the last call went, per CTA: out[8*i + 0] 1 if the run's
+ * survivors went through the shared-memory list, [1] candidate slots recorded, [2] chunks read by the warps,
+ * [3] survivors of the run, [4] chunks of acc read a second time in full, [5] chunks of the run.  Returns the
+ * number of rows written or an error code (< 0).  Synchronises the device. */
+int sidco_get_cta_selection_info(const float* residual, int32_t* out, int max_ctas);
 
 /* Checkpointing of the adaptation state (Algorithm 1 keeps M and the running k_hat sum across
  * iterations): host blobs of 3 int64 per segment (M, calls, k_sum).  Both synchronise the device. */

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libsidco%s.so" % ("_" + _VARIANT if _VARIANT els
 SID_EXP, SID_GAMMA, SID_GPD = 0, 1, 2
 MAX_STAGES = 8
 
-ST_NONFINITE, ST_DEGENERATE, ST_ALL_ZERO, ST_TIMEOUT = 1, 2, 4, 8
+ST_NONFINITE, ST_DEGENERATE, ST_ALL_ZERO, ST_TIMEOUT, ST_BOUNDS = 1, 2, 4, 8, 16
 BUILD_PROFILE, BUILD_BOUNDS_CHECK = 1, 2
 
 
@@ -43,7 +43,7 @@ EXPORTS = [
     "sidco_set_params", "sidco_reset_state", "sidco_get_debug", "sidco_state_save", "sidco_state_load",
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
-    "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate", "sidco_compress_bf16",
+    "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate", "sidco_compress_bf16", "sidco_get_cta_selection_info",
 ]
 
 _lib = None
@@ -110,6 +110,8 @@ def lib() -> C.CDLL:
     L.sidco_set_test_hooks.restype = i32
     L.sidco_build_flags.argtypes = []
     L.sidco_build_flags.restype = i32
+    L.sidco_get_cta_selection_info.argtypes = [vp, C.POINTER(C.c_int32), i32]
+    L.sidco_get_cta_selection_info.restype = i32
     L.sidco_aggregate.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp]
     L.sidco_aggregate.restype = i32
     _lib = L
@@ -282,6 +284,15 @@ def sidco_get_cta_sweep_times(residual, max_ctas: int = 1024) -> np.ndarray:
     if rc < 0:
         raise SidcoError(rc, "sidco_get_cta_sweep_times")
     return np.ctypeslib.as_array(buf)[: 4 * rc].reshape(rc, 4).copy()
+
+
+def sidco_get_cta_selection_info(residual, max_ctas: int = 1024) -> np.ndarray:
+    """(n_ctas, 8) int array, profile builds only: see sidco.h."""
+    buf = (C.c_int32 * (8 * max_ctas))()
+    rc = lib().sidco_get_cta_selection_info(_ptr(residual), buf, max_ctas)
+    if rc < 0:
+        raise SidcoError(rc, "sidco_get_cta_selection_info")
+    return np.ctypeslib.as_array(buf)[: 8 * rc].reshape(rc, 8).copy()
 
 
 STATIC_MAX_ELEMS = 1048576

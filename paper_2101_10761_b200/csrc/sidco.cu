@@ -39,7 +39,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_desc;
-    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, cta_dbg, seg, ctl;
     size_t total;
 };
 
@@ -64,6 +64,7 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.cta_total = take(sizeof(unsigned long long) * (size_t)(G + 1));
     L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
     L.cta_ns = take(sizeof(unsigned long long) * 4 * (size_t)(G + 1));
+    L.cta_dbg = take(sizeof(int) * 8 * (size_t)(G + 1));
     L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
     L.ctl = take(sizeof(Control));
     L.total = o;
@@ -348,7 +349,7 @@ cudaError_t launch_persistent(const void* fn, int grid, void** kargs, cudaStream
 
 // Fill the kernel's argument block for a workspace at `base` laid out as `L` and enqueue the persistent kernel.
 // Used by every entry point, so that they cannot drift apart.
-int launch_compress(char* base, const Layout& L, int T, int S, int G, const float* grad, float* residual, float delta,
+int launch_compress(char* base, const Layout& L, int64_t d, int T, int S, int G, const float* grad, float* residual, float delta,
                     int sid, int max_stages, int32_t* out_idx, float* out_val, int32_t* out_k, cudaStream_t stream,
                     const Params& prm, bool grad_bf16 = false) {
     Args a{};
@@ -374,6 +375,7 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
     a.cta_pub = (unsigned long long*)(base + L.cta_total);
     a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.cta_ns = (unsigned long long*)(base + L.cta_ns);
+    a.cta_dbg = (int*)(base + L.cta_dbg);
     a.seg = (SegDev*)(base + L.seg);
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;
@@ -387,6 +389,7 @@ int launch_compress(char* base, const Layout& L, int T, int S, int G, const floa
     a.C = T;
     a.S = S;
     a.G = G;
+    a.d = (int)d;
     // 256-bit accesses to the residual and an fp32 gradient, 128-bit ones to a bf16 gradient
     a.vec_ok = (((uintptr_t)residual & 31u) | ((uintptr_t)grad & (grad_bf16 ? 15u : 31u))) == 0;
     a.grad_bf16 = grad_bf16 ? 1 : 0;
@@ -418,7 +421,7 @@ int compress_impl(Context* c, const float* grad, float* residual, const int64_t*
         if (cap != cudaStreamCaptureStatusNone) return SIDCO_E_CAPTURE;
         if ((e = build_tables(c, off, S, stream)) != cudaSuccess) return (int)e;
     }
-    return launch_compress((char*)c->ws, c->L, c->T, c->S, c->G, grad, residual, delta, sid, max_stages, out_idx,
+    return launch_compress((char*)c->ws, c->L, c->d, c->T, c->S, c->G, grad, residual, delta, sid, max_stages, out_idx,
                            out_val, out_k, stream, prm, grad_bf16);
 }
 
@@ -581,7 +584,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         c.key = residual;
         c.tables_valid = true;
     }
-    return launch_compress((char*)c.base, c.L, c.T, c.S, c.G, grad, residual, delta, sid_type, max_stages, out_idx,
+    return launch_compress((char*)c.base, c.L, d, c.T, c.S, c.G, grad, residual, delta, sid_type, max_stages, out_idx,
                            out_val, out_k, stream, g_params);
 }
 
@@ -720,7 +723,7 @@ int sidco_get_debug(const float* residual, sidco_seg_debug* out, int n_segs) {
     for (int s = 0; s < c->S; ++s) {
         out[s].M_used = seg[s].M_eff;
         out[s].M_next = seg[s].M;
-        out[s].status = seg[s].status | (ctl.timeout ? SIDCO_ST_TIMEOUT : 0);
+        out[s].status = seg[s].status | (ctl.timeout ? SIDCO_ST_TIMEOUT : 0) | (ctl.bounds ? SIDCO_ST_BOUNDS : 0);
         out[s].calls = seg[s].calls;
         out[s].k_sum = seg[s].k_sum;
         for (int m = 0; m < SIDCO_MAX_STAGES; ++m) {
@@ -779,6 +782,25 @@ int sidco_get_cta_sweep_times(const float* residual, double* us_out, int max_cta
         return (int)e;
     const int n = c->G < max_ctas ? c->G : max_ctas;
     for (int i = 0; i < 4 * n; ++i) us_out[i] = (double)(long long)(ns[i] - ctl.t_ns[0]) * 1e-3;
+    return n;
+#endif
+}
+
+int sidco_get_cta_selection_info(const float* residual, int32_t* out, int max_ctas) {
+#ifndef SIDCO_PROFILE
+    (void)residual; (void)out; (void)max_ctas;
+    return SIDCO_E_UNSUPPORTED;
+#else
+    if (!out) return SIDCO_E_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    auto it = g_ctx.find(residual);
+    if (it == g_ctx.end() || !it->second->tables_valid) return SIDCO_E_UNKNOWN_KEY;
+    Context* c = it->second;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return (int)e;
+    const int n = c->G < max_ctas ? c->G : max_ctas;
+    if ((e = cudaMemcpy(out, (char*)c->ws + c->L.cta_dbg, sizeof(int32_t) * 8 * n, cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return (int)e;
     return n;
 #endif
 }

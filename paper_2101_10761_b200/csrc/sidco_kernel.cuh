@@ -69,9 +69,10 @@ constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
 constexpr int kSegCache = 256;                    // segments of a CTA run whose table entries sit in shared memory
 constexpr int kOutCache = 2048;                   // survivors of a run the shared-memory selection can hold
-constexpr int kSlotCap = 1536;                    // candidate slots (8 elements) of a run held in shared memory
+constexpr int kSlotCap = 4096;                    // candidate slots (8 elements of one lane) a run can note
+constexpr int kSlotPre = 1280;                    // the first of them have their values copied to shared memory ahead
 constexpr int kWinCap = 2048;                     // 1024-element windows of a run the shared-memory selection covers
-static_assert(kSlotCap * kComp >= 2 * kOutCache, "the ordered survivors reuse the candidate values' space");
+static_assert(kSlotPre * kComp >= 2 * kOutCache, "the ordered survivors reuse the candidate values' space");
 constexpr float kSpecRatio = 0.85f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
 constexpr unsigned kFull = 0xffffffffu;
@@ -116,6 +117,8 @@ struct Control {
     int timeout;         // set when a bounded wait ran out
     int residual_is_zero;  // the next call takes the residual's contents as zeros and does not read them
                          // (set by a state reset, cleared by the call)
+    int bounds;          // -DSIDCO_BOUNDS_CHECK builds: an index fell outside its buffer (the access was skipped)
+    int pad;
     unsigned long long t_ns[16];  // globaltimer at phase boundaries, written by CTA 0 (diagnostics)
 };
 
@@ -144,6 +147,7 @@ struct Args {
     unsigned long long* cta_pub; // [G] {call number, survivors of the run}: published once the run's selection is done
     int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
     unsigned long long* cta_ns;  // [G][4] globaltimer when the CTA finished its P1, P3, last P4, P5a sweep
+    int* cta_dbg;                // [G][8] profile builds: how the final selection of the run went
     SegDev* seg;                 // [S]
     Control* ctl;
     // scalars
@@ -153,6 +157,7 @@ struct Args {
     double ln_ratio[kMaxStages + 1], ln_inv_ratio[kMaxStages + 1];
     int Q, sid, max_stages;
     int C, S, G;
+    int d;                       // elements of the vector
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
     int grad_bf16;               // grad points to bf16 values, widened exactly to fp32 before the add
@@ -164,6 +169,17 @@ struct Args {
 // ----------------------------------------------------------------------------
 // small helpers
 // ----------------------------------------------------------------------------
+
+// Range check of an index into a caller or workspace buffer.  Only a build with -DSIDCO_BOUNDS_CHECK checks
+// anything (the stand-in for an external memory checker): a bad index is recorded in the control block and the
+// access is skipped.  In the product build this is the constant true.
+#ifdef SIDCO_BOUNDS_CHECK
+#define SIDCO_IN_RANGE(A, i, n) sidco::in_range_checked((A), (long long)(i), (long long)(n))
+#else
+#define SIDCO_IN_RANGE(A, i, n) true
+#endif
+
+__device__ __forceinline__ bool in_range_checked(const Args& A, long long i, long long n);
 
 __device__ __forceinline__ int ld_cg(const int* p) { return __ldcg(p); }
 __device__ __forceinline__ float ld_cg(const float* p) { return __ldcg(p); }
@@ -212,6 +228,12 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
+}
+
+__device__ __forceinline__ bool in_range_checked(const Args& A, long long i, long long n) {
+    if (i >= 0 && i < n) return true;
+    atomicOr(&A.ctl->bounds, 1);
+    return false;
 }
 
 // Single-thread wait until segment `sg` has `need` stages fitted in call `call_id` (bounded).  Returns the
@@ -702,7 +724,7 @@ constexpr int kSidePre4 = 2;                      // the same in the sweeps that
 // small on purpose: what shared memory takes, the L1 loses, and the first sweep's bandwidth suffers.)
 constexpr int kStageRow = kChunk / kSlots + 8;    // floats of staging per warp: one slot row plus the carried tail
 constexpr int kStageBytes = kWarps * kStageRow * (int)sizeof(float);
-constexpr int kDynSmemBytes = kStageBytes + kSlotCap * (kComp * (int)sizeof(float) + (int)sizeof(int) + 1);
+constexpr int kDynSmemBytes = kStageBytes + kSlotPre * kComp * (int)sizeof(float) + kSlotCap * ((int)sizeof(int) + 1);
 static_assert(kStageBytes >= kOutCache * 8 + kWinCap * 8, "survivor list and window counters fit over the staging area");
 
 // Positions of a lane's kept elements in the chunk's dense, index-ordered side region.  `mask` has bit
@@ -988,7 +1010,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     __shared__ int sm_ok[kSegCache];
     __shared__ int sm_segk[kSegCache];      // survivors of the run per cached segment
     __shared__ int sm_rest[kThreads];       // chunks (relative to c0) whose survivors the candidates do not cover
-    __shared__ int sm_nrest, sm_nslot, sm_nfetched, sm_nsurv, sm_scan_all;
+    __shared__ int sm_nrest, sm_nslot, sm_nfetched, sm_nsurv;
     __shared__ int sm_run_e[2];             // first element of the run and one past its last
     // over the staging area (used after the last sweep that stages): the run's unordered survivor list and the
     // per-window counters that put it in order
@@ -999,7 +1021,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // behind it: the candidate slots (their 8 values, first element, segment of the run); once the survivors are
     // known, the space of the values takes the ordered list
     float* const sm_slot_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sm_stage) + kStageBytes);
-    int* const sm_slot_e = reinterpret_cast<int*>(sm_slot_val + kSlotCap * kComp);
+    int* const sm_slot_e = reinterpret_cast<int*>(sm_slot_val + kSlotPre * kComp);
     unsigned char* const sm_slot_seg = reinterpret_cast<unsigned char*>(sm_slot_e + kSlotCap);
     int* const sm_cidx = reinterpret_cast<int*>(sm_slot_val);
     float* const sm_cval = sm_slot_val + kOutCache;
@@ -1024,7 +1046,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     [[maybe_unused]] const bool stamper = (cta == 0 && threadIdx.x == 0);
     SIDCO_STAMP(if (stamper) A.ctl->t_ns[0] = global_ns());
     if (threadIdx.x == 0) sm_mloc = 1;
-    if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_nrest = 0; sm_nslot = 0; sm_nfetched = 0; sm_nsurv = 0; sm_scan_all = 0; }
+    if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_nrest = 0; sm_nslot = 0; sm_nfetched = 0; sm_nsurv = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
     if (threadIdx.x < 2) sm_run_e[threadIdx.x] = __ldg(A.chunk_start + (threadIdx.x ? c1 : c0));
     // What changes from call to call lives in the workspace (and is advanced by the CTA that finishes the call
@@ -1071,16 +1093,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         return seg - R.seg_lo < kSegCache ? sm_tau[seg - R.seg_lo] : -1.0f;     // (candidates carry a cache index)
     };
     // A slot (8 elements of one lane) that may hold a survivor: only its place is noted here, inside the sweep;
-    // its values are fetched into shared memory in one asynchronous wave when the CTA's sweep is over.
+    // its values are fetched into shared memory in one asynchronous wave when the CTA's sweep is over (for the
+    // first kSlotPre slots; a run with more reads the others from acc when it compares them).
     auto list_slot = [&](int e, int seg_i) {
         const int q = atomicAdd(&sm_nslot, 1);
-        if (q < kSlotCap) { sm_slot_e[q] = e; sm_slot_seg[q] = (unsigned char)seg_i; }
+        if (q < kSlotCap && SIDCO_IN_RANGE(A, e + kComp - 1, A.d) && SIDCO_IN_RANGE(A, seg_i, kSegCache)) {
+            sm_slot_e[q] = e;
+            sm_slot_seg[q] = (unsigned char)seg_i;
+        }
     };
     // Start the copies of the slots listed since the last call (all threads; after the sweep's stores are
     // fenced and the CTA has met).  They complete in the background, behind the fits.
     auto fetch_slots = [&]() {
-        const int from = sm_nfetched, to = min(sm_nslot, kSlotCap);
+        const int from = sm_nfetched, to = min(sm_nslot, kSlotPre);
         for (int q = from + (int)threadIdx.x; q < to; q += kThreads) {
+            if (!SIDCO_IN_RANGE(A, sm_slot_e[q] + kComp - 1, A.d)) continue;
             const float* src = A.residual + sm_slot_e[q];
             cp_async_16(sm_slot_val + q * kComp, src);
             cp_async_16(sm_slot_val + q * kComp + 4, src + 4);
@@ -1133,7 +1160,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
             };
 
-            if (vec_ok && lo == wb && hi == wb + kChunk) {
+            if (vec_ok && lo == wb && hi == wb + kChunk && SIDCO_IN_RANGE(A, wb + kChunk - 1, A.d) && SIDCO_IN_RANGE(A, c, A.C)) {
                 #pragma unroll
                 for (int b = 0; b < kSlots; b += 2) {
                     F8 g8[2], r8[2];
@@ -1158,21 +1185,27 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
                 if (seg_m == 1 && !(tau < 3.0e38f)) list_chunk(c);        // single stage, no candidates recorded
             } else {
-                if (seg_m == 1) list_chunk(c);
+                // a ragged chunk made of whole slots records candidates like a full one
+                const bool whole_slots = vec_ok && ((lo | hi) & (kComp - 1)) == 0;
+                if (seg_m == 1 && !(whole_slots && tau < 3.0e38f)) list_chunk(c);
                 #pragma unroll 1
                 for (int j = 0; j < kSlots; ++j) {
                     const int e = e0 + j * 256;
                     if (e + kComp <= lo || e >= hi) continue;
+                    if (!SIDCO_IN_RANGE(A, hi - 1, A.d) || !SIDCO_IN_RANGE(A, lo, A.d)) continue;
                     if (vec_ok && e >= lo && e + kComp <= hi) {
                         const F8 g = ld8_grad(A.grad, e, g_bf16);
                         F8 r;
                         if (!res_zero) r = ld8_res(A.residual + e, keep);
+                        float big = 0.0f;
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc) {
                             r.v[cc] = res_zero ? g.v[cc] : g.v[cc] + r.v[cc];
                             accumulate(r.v[cc]);
+                            big = fmaxf(big, fabsf(r.v[cc]));
                         }
                         st8_res(A.residual + e, r, keep);
+                        if (whole_slots && big >= tau) list_slot(e, cur.seg - R.seg_lo);
                     } else {
                         for (int cc = 0; cc < kComp; ++cc) {
                             if (e + cc >= lo && e + cc < hi) {
@@ -1201,7 +1234,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 second = (double)esum * 0.693147180559945309417232121458 + log(m);   // used from lane 0 only
             }
             Sums r = warp_tree(s1, SID == kSidGamma ? 0.0 : second, nnz);
-            if (lane == 0) {
+            if (lane == 0 && SIDCO_IN_RANGE(A, c, A.C)) {
                 A.part[3 * (size_t)c + 0] = r.a;
                 A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
                 A.part_n[c] = r.n;
@@ -1229,11 +1262,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     const int c = cur.c, lo = cur.lo, hi = cur.hi;
                     const int wb = lo & ~(kChunk - 1);
                     float v[kSlots][kComp];
+                    if (!SIDCO_IN_RANGE(A, hi - 1, A.d) || !SIDCO_IN_RANGE(A, lo, A.d) || !SIDCO_IN_RANGE(A, c, A.C)) { cur = nxt; continue; }
                     const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
                     // Stage 2 is the last stage of a two-stage segment: nothing reads its exceedances again except
                     // the final selection, which can work from slot flags (as after P1 for one stage).
                     const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
-                    const bool flag_chunk = tau2 > 0.0f && vec_ok && lo == wb && hi == wb + kChunk;
+                    const bool flag_chunk = tau2 > 0.0f && vec_ok && ((lo | hi) & (kComp - 1)) == 0;
                     // (elements outside the chunk read as zero and the threshold is never negative, so they
                     // pass no strict compare)
                     unsigned mask = 0;
@@ -1284,10 +1318,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             int q = pos[j] - a0;
                             #pragma unroll
                             for (int cc = 0; cc < kComp; ++cc)
-                                if ((keep_mask >> (8 * j + cc)) & 1u) stage[q++] = v[j][cc];
+                                if ((keep_mask >> (8 * j + cc)) & 1u) { if (SIDCO_IN_RANGE(A, q, kStageRow)) stage[q] = v[j][cc]; ++q; }
                             __syncwarp();
                             const int n4 = (end - a0 + 3) >> 2;
-                            for (int q4 = lane; q4 < n4; q4 += 32) side[(a0 >> 2) + q4] = reinterpret_cast<const float4*>(stage)[q4];
+                            for (int q4 = lane; q4 < n4; q4 += 32)
+                                if (SIDCO_IN_RANGE(A, (a0 >> 2) + q4, kChunk / 4))
+                                    side[(a0 >> 2) + q4] = reinterpret_cast<const float4*>(stage)[q4];
                             const int tail = end & 3;
                             const float carry = lane < tail ? stage[(end & ~3) - a0 + lane] : 0.0f;
                             __syncwarp();
@@ -1324,7 +1360,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     if (sw.M_eff > m) {
                         // the side region is a dense list: 16 bytes per lane and step, the first steps fetched
                         // with the descriptor
-                        const int c = cur.c, n = cur.side_n;
+                        const int c = cur.c, n = SIDCO_IN_RANGE(A, cur.side_n, kChunk + 1) && SIDCO_IN_RANGE(A, cur.c, A.C) ? cur.side_n : 0;
                         const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
                         double sy = 0.0, sy2 = 0.0;
                         int cnt = 0;
@@ -1390,8 +1426,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     auto append = [&](int e, float val, int seg_i) {
         const int sp = atomicAdd(&sm_nsurv, 1);
         if (sp < kOutCache) { sm_oidx[sp] = e; sm_oval[sp] = val; }
-        atomicAdd(&sm_wcnt[(e >> 10) - win0], 1);
-        atomicAdd(&sm_segk[seg_i], 1);
+        if (SIDCO_IN_RANGE(A, (e >> 10) - win0, n_win)) atomicAdd(&sm_wcnt[(e >> 10) - win0], 1);
+        if (SIDCO_IN_RANGE(A, seg_i, kSegCache)) atomicAdd(&sm_segk[seg_i], 1);
     };
 
     // The warps' pass over chunks.  list_n >= 0: the chunks sm_rest[0 .. list_n); < 0: all chunks of the run,
@@ -1423,19 +1459,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             }
             const int c = cur.c, lo = cur.lo, hi = cur.hi;
             const int wb = lo & ~(kChunk - 1);
-            const bool cand_chunk = seg_cand && vec_ok && lo == wb && hi == wb + kChunk;
+            const bool cand_chunk = seg_cand && vec_ok && ((lo | hi) & (kComp - 1)) == 0;
             int cnt = 0;
-            if (!(skip_covered && cand_chunk && seg_covered)) {
+            const bool chunk_ok = SIDCO_IN_RANGE(A, c, A.C) && SIDCO_IN_RANGE(A, lo, A.d) && SIDCO_IN_RANGE(A, hi - 1, A.d);
+            if (chunk_ok && !(skip_covered && cand_chunk && seg_covered)) {
                 unsigned surv = 0;
                 float v[kSlots][kComp];
-                // a full chunk of a candidate-recording two-stage segment has no side region: it is read from acc
+                // a whole-slot chunk of a candidate-recording two-stage segment has no side region: it is read from acc
                 const bool from_side = seg_from_side && !cand_chunk;
                 if (from_side) {
                     // The side region is a dense list in index order.  Lanes read it 16 bytes at a time; a survivor
                     // is known by its position in the list, and the lane that holds the element at that position
                     // (found through the per-lane masks, only for chunks that have a survivor at all) marks it
                     // in a mask of the chunk's own layout, which gives the survivors their indices and order.
-                    const int n = cur.side_n;
+                    const int n = SIDCO_IN_RANGE(A, cur.side_n, kChunk + 1) ? cur.side_n : 0;
                     const float4* side = reinterpret_cast<const float4*>(A.side_val + (size_t)c * kChunk) + lane;
                     int pos[kSlots], base[kSlots];
                     unsigned smask = 0;
@@ -1493,11 +1530,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             const int bit = __ffs(m) - 1;
                             m &= m - 1u;
                             const int e = e0 + (bit >> 3) * 256 + (bit & 7);
-                            append(e, __ldcg(A.residual + e), seg_i);
+                            if (SIDCO_IN_RANGE(A, e, A.d)) append(e, __ldcg(A.residual + e), seg_i);
                         }
                     } else {
                         cnt = ordered_emit(surv, lo, [&](int p, int j, int cc) {
                             const int e = e0 + j * 256 + cc;
+                            if (!SIDCO_IN_RANGE(A, p, A.d) || !SIDCO_IN_RANGE(A, e, A.d)) return;
                             A.stage_idx[p] = e;
                             A.stage_val[p] = from_side ? __ldcg(A.residual + e) : v[j][cc];
                             A.residual[e] = 0.0f;
@@ -1518,9 +1556,32 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
 
     if (path_a) {
         for (int w = threadIdx.x; w < n_win; w += kThreads) { sm_wcnt[w] = 0; sm_wfill[w] = 0; }
-        // a segment that recorded candidates which turned out unusable: its chunks are in no list
-        for (int i = threadIdx.x; i < R.n_seg; i += kThreads)
-            if (sm_q1[i] > sm_q0[i] && sm_tau[i] > 0.0f && !seg_cand_ok(i)) sm_scan_all = 1;
+        // A segment that recorded candidates which turned out unusable (its threshold fell below the candidate
+        // threshold): its chunks made of whole slots are in no list yet.  (A first or last chunk that is not
+        // recorded no candidates and was listed by the sweep.)  If the candidate slots overflowed, every chunk is
+        // read instead.
+        if (cand_overflow) {
+            if (threadIdx.x == 0) sm_nrest = kThreads + 1;
+        } else if (vec_ok) {
+            // (such segments are rare: they are collected first, then all threads list their chunks)
+            for (int i = threadIdx.x; i < R.n_seg; i += kThreads)
+                if (sm_q1[i] > sm_q0[i] && sm_tau[i] > 0.0f && !seg_cand_ok(i)) sm_list[atomicAdd(&sm_count[0], 1)] = i;
+            __syncthreads();
+            const int n_bad = sm_count[0];
+            for (int k = 0; k < n_bad; ++k) {
+                const int i = sm_list[k];
+                const int qa = max(sm_q0[i], c0), qb = min(sm_q1[i], c1);
+                for (int c = qa + (int)threadIdx.x; c < qb; c += kThreads) {
+                    const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
+                    if (((lo | hi) & (kComp - 1)) == 0) {
+                        const int q = atomicAdd(&sm_nrest, 1);
+                        if (q < kThreads) sm_rest[q] = c - c0;
+                    }
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) sm_count[0] = 0;
+        }
         __syncthreads();
         const int n_slot = min(sm_nslot, kSlotCap);
         for (int q = threadIdx.x; q < n_slot; q += kThreads) {
@@ -1528,14 +1589,21 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             if (seg_cand_ok(i)) {
                 const float thr = R.thr[i];
                 const int e = sm_slot_e[q];
-                #pragma unroll
-                for (int cc = 0; cc < kComp; ++cc) {
-                    const float val = sm_slot_val[q * kComp + cc];
-                    if (fabsf(val) >= thr) append(e + cc, val, i);
+                float x[kComp];
+                if (q < kSlotPre) {
+                    #pragma unroll
+                    for (int cc = 0; cc < kComp; ++cc) x[cc] = sm_slot_val[q * kComp + cc];
+                } else {
+                    const float4 a = __ldcg(reinterpret_cast<const float4*>(A.residual + e));
+                    const float4 b = __ldcg(reinterpret_cast<const float4*>(A.residual + e) + 1);
+                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
                 }
+                #pragma unroll
+                for (int cc = 0; cc < kComp; ++cc)
+                    if (fabsf(x[cc]) >= thr) append(e + cc, x[cc], i);
             }
         }
-        const bool scan_all = sm_scan_all != 0 || sm_nrest > kThreads;
+        const bool scan_all = sm_nrest > kThreads;
         warp_pass(scan_all ? -1 : sm_nrest, true, true);
         __syncthreads();
         cta_count = sm_nsurv;
@@ -1562,6 +1630,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     }
     if (lane == 0 && resweep) atomicAdd(&sm_resweep, resweep);
     __syncthreads();
+    SIDCO_STAMP(if (threadIdx.x == 0) {
+        int* dbg = A.cta_dbg + 8 * cta;
+        dbg[0] = path_a; dbg[1] = sm_nslot; dbg[2] = sm_nrest; dbg[3] = cta_count; dbg[4] = sm_resweep + resweep; dbg[5] = c1 - c0;
+    });
     SIDCO_STAMP(if (threadIdx.x == 0) A.cta_ns[4 * cta + 3] = global_ns());
     SIDCO_STAMP(if (stamper) A.ctl->t_ns[12] = global_ns());
     // next call: start the first sweep where this call's last full sweep over acc ended
@@ -1663,6 +1735,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             for (int q = threadIdx.x; q < cta_count; q += kThreads) {
                 const int e = sm_oidx[q], w = (e >> 10) - win0;
                 const int slot = sm_wcnt[w] + atomicAdd(&sm_wfill[w], 1);
+                if (!SIDCO_IN_RANGE(A, slot, kOutCache)) continue;
                 sm_cidx[slot] = e;                       // (the candidate arrays are free by now)
                 sm_cval[slot] = sm_oval[q];
             }
@@ -1696,6 +1769,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 const int g0 = sm_wcnt[w], g1 = g0 + sm_wfill[w];
                 int rank = 0;
                 for (int t = g0; t < g1; ++t) rank += sm_cidx[t] < e;
+                if (!SIDCO_IN_RANGE(A, run_base + g0 + rank, A.d) || !SIDCO_IN_RANGE(A, e, A.d)) continue;
                 A.out_idx[run_base + g0 + rank] = e;
                 A.out_val[run_base + g0 + rank] = sm_cval[q];
                 A.residual[e] = 0.0f;
@@ -1739,6 +1813,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
                 const int i = a - 1;
                 const int src = __ldg(A.chunk_start + pass + i) + (pos - sm_scan[i]);
+                if (!SIDCO_IN_RANGE(A, pos, A.d) || !SIDCO_IN_RANGE(A, src, A.d)) continue;
                 A.out_idx[pos] = ld_cg(A.stage_idx + src);
                 A.out_val[pos] = ld_cg(A.stage_val + src);
             }
