@@ -625,6 +625,10 @@ def run_gpu(args):
     if rank == 0 and not args.no_aggregate and hasattr(B, "sidco_aggregate"):
         aggregate = bench_aggregate(torch, B, wl, head, dev, peak)
 
+    reference_points = None
+    if rank == 0 and not args.no_variants and hasattr(B, "sidco_topk"):
+        reference_points = bench_reference_points(torch, B, wl, grads, dev, statistics.median(region_ms) / args.steps, by_sid)
+
     sweep = None
     if rank == 0 and args.sweep:
         sweep = bench_sweep(torch, B, dev, peak, args)
@@ -697,6 +701,7 @@ def run_gpu(args):
             },
             "variants": variants,
             "aggregate": aggregate,
+            "reference_points": reference_points,
             "sweep": sweep,
             "gpu_launches": int(launches),
             "clocks": sampler.summary(),
@@ -756,6 +761,53 @@ def bench_aggregate(torch, B, wl, head, dev, peak, n_workers=8):
                          "bytes_note": "8 bytes per gathered (index, value) pair read + 4 d bytes written",
                          "traffic": None},
             "l2": "three output buffers (3 x 4 d bytes) in rotation"}
+
+
+def bench_reference_points(torch, B, wl, grads, dev, sidco_ms_per_step, by_sid):
+    """Context, never the target: the paper's two comparison compressors (exact Top-k, sampled threshold) on the
+    same inputs and protocol-free steady calls (residual carried over ten gradient buffers), with the achieved
+    ratio k_hat / k of each next to SIDCo's."""
+    from paper_2101_10761_b200 import workloads as W
+    d = wl.d
+    k = int(np.ceil(np.float64(DELTA) * d))
+    pos_h = W.sample_positions(d, 0.01, 9000)
+    pos = torch.from_numpy(pos_h).to(dev)
+    ws_bytes = B.sidco_reference_workspace_bytes(d, pos_h.size)
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device=dev)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    res = torch.zeros(d, dtype=torch.float32, device=dev)
+    out_idx = torch.empty(d, dtype=torch.int32, device=dev)
+    out_val = torch.empty(d, dtype=torch.float32, device=dev)
+    out_k = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = {}
+    for name in ("topk", "dgc"):
+        res.zero_()
+
+        def call(i):
+            if name == "topk":
+                B.sidco_topk(grads[i % RUN_LEN], res, d, k, out_idx, out_val, out_k, ws_ptr, ws_bytes)
+            else:
+                B.sidco_dgc(grads[i % RUN_LEN], res, d, DELTA, pos, pos_h.size, out_idx, out_val, out_k, ws_ptr, ws_bytes)
+        for i in range(RUN_LEN):
+            call(i)
+        ts, ks = [], []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(2 * RUN_LEN):
+                call(i)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / (2 * RUN_LEN))
+            ks.append(int(out_k.item()))
+        ms = statistics.median(ts)
+        out[name] = {"us_per_step": round(ms * 1e3, 2), "k_hat_over_k": round(statistics.mean(ks) / (DELTA * d), 4),
+                     "sidco_speedup": round(ms / sidco_ms_per_step, 2)}
+    out["sidco_k_hat_over_k"] = {sid: round(v["k_hat_mean"] / (DELTA * d), 4) for sid, v in by_sid.items()}
+    out["note"] = ("whole-vector Top-k (k = ceil(delta d), radix select) and sampled threshold (1 % sample, seed 9000); "
+                   "sidco_speedup = their time per call over the headline's ms_per_step; sidco_k_hat_over_k is per "
+                   "SID under the headline protocol (adaptive stages, per segment)")
+    return out
 
 
 SWEEP_SIZES = [

@@ -209,6 +209,34 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
 int sidco_aggregate(const int32_t* idx_all, const float* val_all, const int32_t* counts, int n_workers,
                     int64_t stride, int64_t d, float* out_dense, int32_t* status, void* stream);
 
+/*
+ * Reference points: the two compressors the paper compares its method with (Section 1 and Fig. 1), on the same
+ * inputs and with the same error-compensation wrapper, so that speed and achieved ratio can be compared on one
+ * machine.  Whole-vector selection, as in the paper's micro-benchmark.  Both compute acc = grad + residual
+ * (stored over residual), write the selected (index, value) pairs in ascending index order, set the selected
+ * residual entries to +0.0f, and write the number selected to out_k[0].  Magnitudes are compared as the bit
+ * patterns of |acc| (finite < infinite < NaN).
+ *
+ * sidco_topk - exact Top-k: the k largest magnitudes; among equal magnitudes the lower index wins.
+ * sidco_dgc  - sampled threshold (Deep Gradient Compression style): the threshold is the ceil(delta * n_sample)-th
+ *              largest magnitude (at least the largest) among acc[sample_idx[0 .. n_sample)]; every element of the
+ *              vector whose magnitude reaches it is selected.  The sample positions are the caller's (any
+ *              generator; a position outside [0, d) counts as a zero).
+ *
+ * grad, residual, out_idx, out_val   device, as in sidco_compress (capacity d).
+ * out_k       device, int32[1].
+ * sample_idx  device, int32[n_sample].
+ * workspace   device, 256-byte aligned, at least sidco_reference_workspace_bytes(d, n_sample) bytes (n_sample = 0
+ *             for sidco_topk); caller-owned, no state is kept in it between calls.
+ * stream      everything is enqueued here (about ten kernels); no synchronisation, no allocation.
+ */
+size_t sidco_reference_workspace_bytes(int64_t d, int64_t n_sample);
+int sidco_topk(const float* grad, float* residual, int64_t d, int64_t k, int32_t* out_idx, float* out_val,
+               int32_t* out_k, void* workspace, size_t workspace_bytes, void* stream);
+int sidco_dgc(const float* grad, float* residual, int64_t d, float delta, const int32_t* sample_idx,
+              int64_t n_sample, int32_t* out_idx, float* out_val, int32_t* out_k, void* workspace,
+              size_t workspace_bytes, void* stream);
+
 /* Bytes of device scratch one residual key needs for a vector of d elements in n_segs segments. */
 size_t sidco_workspace_bytes(int64_t d, int n_segs);
 

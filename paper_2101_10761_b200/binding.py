@@ -44,6 +44,7 @@ EXPORTS = [
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
     "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate", "sidco_compress_bf16", "sidco_get_cta_selection_info",
+    "sidco_reference_workspace_bytes", "sidco_topk", "sidco_dgc",
 ]
 
 _lib = None
@@ -112,6 +113,12 @@ def lib() -> C.CDLL:
     L.sidco_build_flags.restype = i32
     L.sidco_get_cta_selection_info.argtypes = [vp, C.POINTER(C.c_int32), i32]
     L.sidco_get_cta_selection_info.restype = i32
+    L.sidco_reference_workspace_bytes.argtypes = [i64, i64]
+    L.sidco_reference_workspace_bytes.restype = C.c_size_t
+    L.sidco_topk.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, C.c_size_t, vp]
+    L.sidco_topk.restype = i32
+    L.sidco_dgc.argtypes = [vp, vp, i64, f32, vp, i64, vp, vp, vp, vp, C.c_size_t, vp]
+    L.sidco_dgc.restype = i32
     L.sidco_aggregate.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp]
     L.sidco_aggregate.restype = i32
     _lib = L
@@ -249,6 +256,28 @@ def sidco_aggregate(idx_all, val_all, counts, n_workers: int, stride: int, d: in
                                _ptr(out_dense), _ptr(status), _stream(stream))
     if rc:
         raise SidcoError(rc, "sidco_aggregate")
+
+
+def sidco_reference_workspace_bytes(d: int, n_sample: int = 0) -> int:
+    return int(lib().sidco_reference_workspace_bytes(d, n_sample))
+
+
+def sidco_topk(grad, residual, d: int, k: int, out_idx, out_val, out_k, workspace, workspace_bytes: int,
+               stream=None) -> None:
+    """Exact Top-k reference point (device buffers; see sidco.h)."""
+    rc = lib().sidco_topk(_ptr(grad), _ptr(residual), d, k, _ptr(out_idx), _ptr(out_val), _ptr(out_k),
+                          _ptr(workspace), workspace_bytes, _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_topk")
+
+
+def sidco_dgc(grad, residual, d: int, delta: float, sample_idx, n_sample: int, out_idx, out_val, out_k,
+              workspace, workspace_bytes: int, stream=None) -> None:
+    """Sampled-threshold reference point (device buffers; see sidco.h)."""
+    rc = lib().sidco_dgc(_ptr(grad), _ptr(residual), d, delta, _ptr(sample_idx), n_sample, _ptr(out_idx),
+                         _ptr(out_val), _ptr(out_k), _ptr(workspace), workspace_bytes, _stream(stream))
+    if rc:
+        raise SidcoError(rc, "sidco_dgc")
 
 
 def sidco_set_test_hooks(grid: int = 0, spec_enable: int = 1, spin_limit: int = 0,
