@@ -54,6 +54,24 @@ class Params:
 
 
 @dataclass
+class Policy:
+    """Variants the paper describes and then replaces or leaves open.  All off: the method as evaluated.
+
+    gamma_exact        Corollary 1.2 without its two shortcuts: the shape is the maximum-likelihood estimate
+                       (root of the digamma equation the proof states) and the threshold is
+                       beta * P^{-1}(alpha, 1 - delta), the exact quantile, instead of the closed-form bound.
+    ratio_from_counts  the last stage aims at the target count directly: its ratio is k / k_hat_{M-1}
+                       (target count over the exceedances the stage before it left) instead of the nominal
+                       delta / delta_1^(M-1).  [reading: the paper only states delta = prod delta_m]
+    adapt_reversed     Adapt_Stages with the opposite sign (too many selected -> one stage more), the
+                       direction the prose of the experiments suggests; Algorithm 1 prints the other one.
+    """
+    gamma_exact: bool = False
+    ratio_from_counts: bool = False
+    adapt_reversed: bool = False
+
+
+@dataclass
 class SegState:
     """Adaptation state of one segment, carried across calls."""
     M: int = 1
@@ -135,6 +153,121 @@ def gamma_shape(s: float) -> float:
     return (3.0 - s + math.sqrt((s - 3.0) ** 2 + 24.0 * s)) / (12.0 * s)
 
 
+# -- special functions for the exact forms of Corollary 1.2 (plain series; pinned against a library in the tests)
+
+def digamma(x: float) -> float:
+    """psi(x) for x > 0: recurrence up to x >= 8, then the asymptotic series."""
+    acc = 0.0
+    while x < 8.0:
+        acc -= 1.0 / x
+        x += 1.0
+    f = 1.0 / (x * x)
+    return acc + math.log(x) - 0.5 / x - f * (1.0 / 12 - f * (1.0 / 120 - f * (1.0 / 252 - f * (1.0 / 240 - f / 132))))
+
+
+def trigamma(x: float) -> float:
+    """psi'(x) for x > 0."""
+    acc = 0.0
+    while x < 8.0:
+        acc += 1.0 / (x * x)
+        x += 1.0
+    f = 1.0 / (x * x)
+    return acc + 1.0 / x + 0.5 * f + (1.0 / x) * f * (1.0 / 6 - f * (1.0 / 30 - f * (1.0 / 42 - f / 30)))
+
+
+def gamma_shape_mle(s: float) -> float:
+    """Maximum-likelihood shape: the root of log(alpha) - psi(alpha) = s (the equation in the proof of
+    Corollary 1.2), by Newton's method from the closed-form estimate."""
+    alpha = gamma_shape(s)
+    for _ in range(100):
+        f = math.log(alpha) - digamma(alpha) - s
+        step = f / (1.0 / alpha - trigamma(alpha))
+        new = alpha - step
+        if new <= 0.0:
+            new = 0.5 * alpha
+        if abs(new - alpha) <= 1e-15 * alpha:
+            return new
+        alpha = new
+    return alpha
+
+
+def gamma_upper_q(a: float, x: float) -> float:
+    """Q(a, x) = 1 - P(a, x), the regularised upper incomplete gamma function: the power series of P for
+    x < a + 1, the continued fraction of Q otherwise."""
+    if x <= 0.0:
+        return 1.0
+    log_front = a * math.log(x) - x - math.lgamma(a)
+    if x < a + 1.0:
+        term = 1.0 / a
+        total = term
+        n = 0
+        while abs(term) > 1e-17 * abs(total) and n < 10000:
+            n += 1
+            term *= x / (a + n)
+            total += term
+        return 1.0 - total * math.exp(log_front)
+    tiny = 1e-300
+    b = x + 1.0 - a
+    c = 1.0 / tiny
+    d = 1.0 / b
+    h = d
+    for i in range(1, 10000):
+        an = -i * (i - a)
+        b += 2.0
+        d = an * d + b
+        d = tiny if abs(d) < tiny else d
+        c = b + an / c
+        c = tiny if abs(c) < tiny else c
+        d = 1.0 / d
+        delta = d * c
+        h *= delta
+        if abs(delta - 1.0) < 1e-16:
+            break
+    return h * math.exp(log_front)
+
+
+def gamma_upper_quantile(a: float, q: float) -> float:
+    """x with Q(a, x) = q, i.e. P^{-1}(a, 1 - q): bracketing by doubling, then bisection on log Q refined by
+    Newton steps that stay inside the bracket."""
+    if q >= 1.0:
+        return 0.0
+    lo, hi = 0.0, max(1.0, a)
+    while gamma_upper_q(a, hi) > q:
+        lo, hi = hi, 2.0 * hi
+    x = 0.5 * (lo + hi)
+    for _ in range(200):
+        qx = gamma_upper_q(a, x)
+        if qx > q:
+            lo = x
+        else:
+            hi = x
+        # Newton on log Q: d/dx log Q = -x^(a-1) e^(-x) / (Gamma(a) Q)
+        dens = math.exp((a - 1.0) * math.log(x) - x - math.lgamma(a))
+        new = x + (math.log(qx) - math.log(q)) * qx / dens if qx > 0.0 and dens > 0.0 else 0.5 * (lo + hi)
+        if not (lo < new < hi):
+            new = 0.5 * (lo + hi)
+        if abs(new - x) <= 1e-15 * x:
+            return new
+        x = new
+    return x
+
+
+def gamma_first_stage_exact(a: np.ndarray, ratio: float):
+    """Corollary 1.2 without the shortcuts: maximum-likelihood shape and the exact quantile.  Same reading of
+    zeros and of constant magnitudes as gamma_first_stage.  Returns (eta, degenerate)."""
+    n = a.size
+    nz = a[a > 0.0]
+    n_nz = nz.size
+    mu = float(np.sum(nz)) / n_nz
+    s = math.log(mu) - float(np.sum(np.log(nz))) / n_nz
+    ratio_nz = min(1.0, ratio * n / n_nz)
+    if s <= 1e-12:
+        return max(exp_quantile_step(mu, ratio_nz), 0.0), True
+    alpha = gamma_shape_mle(s)
+    beta = mu / alpha
+    return beta * gamma_upper_quantile(alpha, ratio_nz), False
+
+
 def gamma_first_stage(a: np.ndarray, ratio: float):
     """Corollary 1.2 on the magnitudes ``a`` (fp64).  Returns (eta, degenerate).
 
@@ -161,7 +294,8 @@ def gamma_first_stage(a: np.ndarray, ratio: float):
     return eta, False
 
 
-def thresholds(a: np.ndarray, delta: float, sid: int, M: int, delta1: float) -> SegReport:
+def thresholds(a: np.ndarray, delta: float, sid: int, M: int, delta1: float,
+               policy: Policy = Policy()) -> SegReport:
     """Multi-stage threshold estimation for one segment (Section 2.4).
 
     ``a`` holds the fp64 magnitudes |acc|.  Stage 1 fits all of them; stage
@@ -201,7 +335,7 @@ def thresholds(a: np.ndarray, delta: float, sid: int, M: int, delta1: float) -> 
         eta, deg = gpd_quantile_step(mu, var, ratios[0])
         rep.status |= ST_DEGENERATE if deg else 0
     elif sid == SID_GAMMA:
-        eta, deg = gamma_first_stage(a, ratios[0])
+        eta, deg = (gamma_first_stage_exact if policy.gamma_exact else gamma_first_stage)(a, ratios[0])
         rep.status |= ST_DEGENERATE if deg else 0
     else:
         raise ValueError("unknown SID")
@@ -216,6 +350,9 @@ def thresholds(a: np.ndarray, delta: float, sid: int, M: int, delta1: float) -> 
             continue
         y = exceed - eta
         ybar = float(np.sum(y)) / y.size
+        if policy.ratio_from_counts and m == M_eff - 1:
+            # the last stage keeps the target count out of what the stage before it left
+            ratios[m] = min(1.0, delta * n / exceed.size)
         if sid == SID_EXP:
             inc = exp_quantile_step(ybar, ratios[m])
         else:
@@ -234,22 +371,25 @@ def thresholds(a: np.ndarray, delta: float, sid: int, M: int, delta1: float) -> 
 # Stage adaptation (Algorithm 1, Adapt_Stages)
 # ---------------------------------------------------------------------------
 
-def adapt_stages(M: int, k_avg: float, k: float, eps_H: float, eps_L: float, M_max: int) -> int:
-    """Too many selected -> one stage fewer; too few -> one more; clamp."""
+def adapt_stages(M: int, k_avg: float, k: float, eps_H: float, eps_L: float, M_max: int,
+                 reversed_direction: bool = False) -> int:
+    """Too many selected -> one stage fewer; too few -> one more; clamp.  (reversed_direction: the opposite.)"""
+    step = -1 if reversed_direction else 1
     if k_avg > k * (1.0 + eps_H):
-        M = M - 1
+        M = M - step
     if k_avg < k * (1.0 - eps_L):
-        M = M + 1
+        M = M + step
     return min(max(M, 1), M_max)
 
 
-def adapt_update(st: SegState, k_hat: int, k: float, params: Params, M_max: int) -> None:
+def adapt_update(st: SegState, k_hat: int, k: float, params: Params, M_max: int,
+                 policy: Policy = Policy()) -> None:
     """[reading] calls are counted from one, every k_hat is added, and the mean
     of exactly Q values is compared at every Q-th call."""
     st.calls += 1
     st.k_sum += int(k_hat)
     if st.calls % params.Q == 0:
-        st.M = adapt_stages(st.M, st.k_sum / params.Q, k, params.eps_H, params.eps_L, M_max)
+        st.M = adapt_stages(st.M, st.k_sum / params.Q, k, params.eps_H, params.eps_L, M_max, policy.adapt_reversed)
         st.k_sum = 0
 
 
@@ -259,7 +399,7 @@ def adapt_update(st: SegState, k_hat: int, k: float, params: Params, M_max: int)
 
 def sidco_compress(grad: np.ndarray, residual: np.ndarray, seg_offsets, delta: float,
                    sid: int, max_stages: int, state: Optional[List[SegState]] = None,
-                   params: Params = Params()) -> Result:
+                   params: Params = Params(), policy: Policy = Policy()) -> Result:
     """max_stages > 0: adaptive, M starts at 1 and moves inside [1, max_stages]
     (``state`` is updated in place); max_stages < 0: fixed M = -max_stages."""
     grad = np.asarray(grad, dtype=np.float32)
@@ -280,14 +420,14 @@ def sidco_compress(grad: np.ndarray, residual: np.ndarray, seg_offsets, delta: f
             M = min(max(state[s].M, 1), max_stages)
         else:
             M = -max_stages
-        rep = thresholds(a, delta, sid, M, params.delta1)
+        rep = thresholds(a, delta, sid, M, params.delta1, policy)
         eta = rep.eta[-1]
         keep = np.nonzero(a >= eta)[0]              # final selection: |x| >= eta_M
         out_k[s] = keep.size
         idx_parts.append(keep + lo)
         reports.append(rep)
         if adaptive:
-            adapt_update(state[s], keep.size, delta * (hi - lo), params, max_stages)
+            adapt_update(state[s], keep.size, delta * (hi - lo), params, max_stages, policy)
     idx = (np.concatenate(idx_parts) if idx_parts else np.zeros(0, np.int64)).astype(np.int32)
     out_k[n_segs] = idx.size
     val = acc[idx]

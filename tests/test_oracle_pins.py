@@ -195,30 +195,47 @@ def gamma_sample(n, alpha, theta, seed):
     return (np.where(r.random(n) < 0.5, -1.0, 1.0) * r.gamma(alpha, theta, n)).astype(np.float32)
 
 
-def test_gamma_first_stage_matches_formula_with_library_pieces():
-    n, alpha, theta, delta = 500000, 0.6, 2e-3, 0.01
+@pytest.mark.parametrize("delta,expected", [(0.1, 0.66), (0.01, 0.50), (0.001, 0.42)])
+def test_gamma_closed_form_underselects_gamma_data_by_the_known_factor(delta, expected):
+    """On Gamma(0.6) magnitudes the closed-form threshold of Corollary 1.2 is an upper bound of the true
+    quantile, so the single-stage gamma fit keeps fewer than k elements: the population values of
+    k_hat / k are 0.66, 0.50 and 0.42 at delta = 0.1, 0.01, 0.001 (computed from the gamma survival function
+    at the closed form evaluated with the biased shape estimate; independent of this oracle)."""
+    n, alpha, theta = 2_000_000, 0.6, 2e-3
     x = gamma_sample(n, alpha, theta, 9)
+    out = O.sidco_compress(x, np.zeros_like(x), [0, n], delta, O.SID_GAMMA, -1)
+    ratio = out.idx.size / (delta * n)
+    # population value recomputed here from library functions only
+    s_pop = math.log(alpha) - sps.digamma(alpha)
+    a_hat = (3 - s_pop + math.sqrt((s_pop - 3) ** 2 + 24 * s_pop)) / (12 * s_pop)
+    eta_over_theta = -(alpha / a_hat) * (math.log(delta) + sps.gammaln(a_hat))
+    pop = sst.gamma.sf(eta_over_theta, alpha) / delta
+    assert pop == pytest.approx(expected, abs=0.01)
+    k = delta * n
+    assert ratio == pytest.approx(pop, abs=6 * math.sqrt(pop / k) + 0.02)
+
+
+@pytest.mark.parametrize("alpha", [0.3, 0.6, 0.9])
+@pytest.mark.parametrize("delta", [0.01, 0.001])
+def test_gamma_threshold_of_the_oracle_upper_bounds_the_exact_quantile(alpha, delta):
+    """Corollary 1.2: for a fitted shape <= 1 (and an exact quantile >= 1 in units of the scale) the closed form
+    lies above beta * P^-1(alpha, 1 - delta).  Checked on the oracle's own output with a library inverse."""
+    n = 300000
+    x = gamma_sample(n, alpha, 1e-3, 31)
     a = np.abs(x).astype(np.float64)
     eta, deg = O.gamma_first_stage(a, delta)
     assert not deg
-    # fitted shape near the population bias for alpha = 0.6 and scale consistent with it
-    s = math.log(a.mean()) - np.log(a).mean()
-    al = O.gamma_shape(s)
-    assert al / alpha - 1 == pytest.approx(-0.013, abs=0.01)
-    assert eta == pytest.approx(-(a.mean() / al) * (math.log(delta) + sps.gammaln(al)), rel=1e-12)
-
-
-@pytest.mark.parametrize("alpha", [0.3, 0.6, 0.9, 1.0])
-@pytest.mark.parametrize("delta", [0.01, 0.001])
-def test_gamma_closed_form_upper_bounds_exact_quantile(alpha, delta):
-    # Corollary 1.2: -[log delta + log Gamma(alpha)] >= P^-1(alpha, 1-delta) for alpha <= 1
-    # whenever the exact quantile is >= 1, with equality at alpha = 1.
-    exact = sps.gammaincinv(alpha, 1.0 - delta)
-    assert exact >= 1.0
-    closed = -(math.log(delta) + math.lgamma(alpha))
-    assert closed >= exact * (1 - 1e-12)
-    if alpha == 1.0:
-        assert closed == pytest.approx(exact, rel=1e-10)
+    s_hat = math.log(a.mean()) - np.log(a).mean()
+    a_hat = O.gamma_shape(s_hat)
+    b_hat = a.mean() / a_hat
+    exact = sps.gammaincinv(a_hat, 1.0 - delta)
+    assert a_hat <= 1.0 and exact >= 1.0
+    assert eta / b_hat >= exact * (1 - 1e-12)
+    # and the bound is tight at shape one (exponential data)
+    e = np.abs(laplace_acc(n, 1e-3, 32)).astype(np.float64)
+    eta1, _ = O.gamma_first_stage(e, delta)
+    a1 = O.gamma_shape(math.log(e.mean()) - np.log(e).mean())
+    assert eta1 / (e.mean() / a1) == pytest.approx(sps.gammaincinv(a1, 1.0 - delta), rel=0.02)
 
 
 def test_gamma_on_exponential_data_close_to_exp_threshold():
@@ -465,3 +482,85 @@ def test_bf16_widening_matches_an_independent_conversion():
     x = r.standard_normal(1000).astype(np.float32)
     xb = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.all(np.abs(O.bf16_bits_to_f32(xb) - x) <= np.abs(x) * 2.0 ** -8)
+
+
+# ------------------------------------------------------------------ variants the paper describes and replaces
+
+@pytest.mark.parametrize("x", [0.03, 0.2, 0.6, 1.0, 2.5, 7.9, 8.0, 33.0, 400.0])
+def test_digamma_and_trigamma_against_the_library(x):
+    assert O.digamma(x) == pytest.approx(sps.digamma(x), rel=1e-12, abs=1e-12)
+    assert O.trigamma(x) == pytest.approx(float(sps.polygamma(1, x)), rel=1e-10)
+
+
+@pytest.mark.parametrize("a", [0.05, 0.3, 0.6, 1.0, 2.0, 9.0])
+@pytest.mark.parametrize("q", [1.0, 0.9, 0.25, 0.04, 1e-3, 1e-7])
+def test_gamma_upper_quantile_against_the_library_inverse(a, q):
+    x = O.gamma_upper_quantile(a, q)
+    if q >= 1.0:
+        assert x == 0.0
+        return
+    assert x == pytest.approx(sps.gammainccinv(a, q), rel=1e-10)
+    assert O.gamma_upper_q(a, x) == pytest.approx(q, rel=1e-10)
+    assert O.gamma_upper_q(a, x) == pytest.approx(sps.gammaincc(a, x), rel=1e-11)
+
+
+@pytest.mark.parametrize("s", [1e-3, 0.05, 0.5772156649, 1.5, 6.0])
+def test_mle_shape_solves_the_digamma_equation(s):
+    al = O.gamma_shape_mle(s)
+    assert math.log(al) - sps.digamma(al) == pytest.approx(s, rel=1e-10, abs=1e-12)
+    # Minka's closed form is within about 1.5 % of it
+    assert O.gamma_shape(s) == pytest.approx(al, rel=0.02)
+
+
+@pytest.mark.parametrize("alpha", [0.3, 0.6, 1.0, 2.0])
+@pytest.mark.parametrize("delta", [0.1, 0.01, 0.001])
+def test_exact_gamma_policy_reaches_the_target_ratio_on_gamma_data(alpha, delta):
+    """With the maximum-likelihood shape and the exact quantile the single-stage gamma fit keeps k elements up
+    to sampling error (binomial count plus the estimator's own error), where the closed form keeps 0.4-0.7 k."""
+    n = 1_000_000
+    x = gamma_sample(n, alpha, 2e-3, 40)
+    pol = O.Policy(gamma_exact=True)
+    out = O.sidco_compress(x, np.zeros_like(x), [0, n], delta, O.SID_GAMMA, -1, policy=pol)
+    k = delta * n
+    assert out.idx.size == pytest.approx(k, abs=6 * math.sqrt(k) + 0.03 * k)
+    # the threshold is the library's quantile of the fitted law
+    a = np.abs(x).astype(np.float64)
+    s_hat = math.log(a.mean()) - np.log(a).mean()
+    al = O.gamma_shape_mle(s_hat)
+    assert out.report[0].eta[0] == pytest.approx(sst.gamma.isf(delta, al, scale=a.mean() / al), rel=1e-9)
+
+
+def test_ratio_from_counts_policy_uses_the_achieved_count_of_the_previous_stage():
+    n, delta = 400000, 0.001
+    x = laplace_acc(n, 1e-3, 50)
+    a = np.abs(x).astype(np.float64)
+    pol = O.Policy(ratio_from_counts=True)
+    for M in (2, 3, 4):
+        rep_n = O.thresholds(a, delta, O.SID_EXP, M, 0.25)
+        rep_c = O.thresholds(a, delta, O.SID_EXP, M, 0.25, pol)
+        assert rep_c.eta[:-1] == rep_n.eta[:-1]                      # only the last stage changes
+        exceed = a[a > rep_c.eta[-2]]
+        want = rep_c.eta[-2] + (exceed - rep_c.eta[-2]).mean() * math.log(exceed.size / (delta * n))
+        assert rep_c.eta[-1] == pytest.approx(want, rel=1e-12)
+    # exponential magnitudes: the stages before the last keep a quarter each up to sampling error, so the two
+    # rules nearly coincide, and both land on k
+    k = delta * n
+    for rep in (O.thresholds(a, delta, O.SID_EXP, 3, 0.25), O.thresholds(a, delta, O.SID_EXP, 3, 0.25, pol)):
+        assert rep.k_stage[-1] == pytest.approx(k, abs=6 * math.sqrt(k) + 0.05 * k)
+
+
+def test_reversed_adaptation_policy_flips_the_transition_table():
+    for k_avg in (50.0, 100.0, 150.0):         # away from the clamps the two directions mirror each other
+        fwd = O.adapt_stages(3, k_avg, 100.0, 0.2, 0.2, 5)
+        rev = O.adapt_stages(3, k_avg, 100.0, 0.2, 0.2, 5, True)
+        assert fwd - 3 == -(rev - 3)
+    assert O.adapt_stages(2, 150.0, 100.0, 0.2, 0.2, 4, True) == 3        # too many -> one more stage
+    assert O.adapt_stages(2, 50.0, 100.0, 0.2, 0.2, 4, True) == 1         # too few  -> one fewer
+    assert O.adapt_stages(2, 110.0, 100.0, 0.2, 0.2, 4, True) == 2
+    assert O.adapt_stages(1, 50.0, 100.0, 0.2, 0.2, 4, True) == 1 and O.adapt_stages(4, 150.0, 100.0, 0.2, 0.2, 4, True) == 4
+    # scripted counts through the bookkeeping: five calls that select twice the target
+    st_a, st_b = O.SegState(M=2), O.SegState(M=2)
+    for _ in range(5):
+        O.adapt_update(st_a, 200, 100.0, O.Params(), 4)
+        O.adapt_update(st_b, 200, 100.0, O.Params(), 4, O.Policy(adapt_reversed=True))
+    assert (st_a.M, st_a.calls, st_a.k_sum) == (1, 5, 0) and (st_b.M, st_b.calls, st_b.k_sum) == (3, 5, 0)
