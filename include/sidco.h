@@ -249,6 +249,19 @@ int sidco_set_workspace(const float* residual, void* device_ptr, size_t bytes);
  * delta_1 = 0.25, eps_H = eps_L = 0.2, Q = 5).  0 < delta1 < 1, 0 <= eps < 1, Q >= 1. */
 int sidco_set_params(double delta1, double eps_H, double eps_L, int Q);
 
+/* Variants the paper describes and then replaces or leaves open, for subsequent calls (all 0 by default: the
+ * method as the paper evaluates it).  They exist to quantify what the shortcuts cost in achieved ratio.
+ *   gamma_exact        Corollary 1.2 without its two shortcuts: the shape is the maximum-likelihood estimate (the
+ *                      root of the digamma equation in the corollary's proof, Newton's method on the device) and
+ *                      the first-stage threshold is beta * P^{-1}(alpha, 1 - delta), the exact gamma quantile,
+ *                      instead of the closed-form bound.  Costs tens of microseconds of serial fp64 per call.
+ *   ratio_from_counts  the last stage of a multi-stage fit aims at the target count itself: its ratio is
+ *                      k / k_hat_{M-1} (delta * n over the exceedances the stage before it left, at most 1) instead
+ *                      of the nominal delta / delta_1^(M-1) (Section 2.4 only fixes the product of the ratios).
+ *   adapt_reversed     Adapt_Stages (Algorithm 1) with the opposite sign: too many selected -> one stage more.
+ */
+int sidco_set_policy(int gamma_exact, int ratio_from_counts, int adapt_reversed);
+
 /* Start over for `residual`: the adaptation state is forgotten (M back to 1, counters to 0) and the error
  * compensation memory is declared empty - the next sidco_compress on it takes the residual as all zeros
  * without reading it (and overwrites it), so the caller need not clear the buffer.  Synchronises the device. */

@@ -44,7 +44,7 @@ EXPORTS = [
     "sidco_release", "sidco_release_all", "sidco_launch_count", "sidco_error_string", "sidco_version",
     "sidco_get_phase_times", "sidco_get_cta_sweep_times", "sidco_compress_static",
     "sidco_reset_state_async", "sidco_set_test_hooks", "sidco_build_flags", "sidco_aggregate", "sidco_compress_bf16", "sidco_get_cta_selection_info",
-    "sidco_reference_workspace_bytes", "sidco_topk", "sidco_dgc",
+    "sidco_reference_workspace_bytes", "sidco_topk", "sidco_dgc", "sidco_set_policy",
 ]
 
 _lib = None
@@ -119,6 +119,8 @@ def lib() -> C.CDLL:
     L.sidco_topk.restype = i32
     L.sidco_dgc.argtypes = [vp, vp, i64, f32, vp, i64, vp, vp, vp, vp, C.c_size_t, vp]
     L.sidco_dgc.restype = i32
+    L.sidco_set_policy.argtypes = [i32, i32, i32]
+    L.sidco_set_policy.restype = i32
     L.sidco_aggregate.argtypes = [vp, vp, vp, i32, i64, i64, vp, vp, vp]
     L.sidco_aggregate.restype = i32
     _lib = L
@@ -196,6 +198,13 @@ def sidco_set_params(delta1: float = 0.25, eps_H: float = 0.2, eps_L: float = 0.
     rc = lib().sidco_set_params(delta1, eps_H, eps_L, Q)
     if rc:
         raise SidcoError(rc, "sidco_set_params")
+
+
+def sidco_set_policy(gamma_exact: bool = False, ratio_from_counts: bool = False, adapt_reversed: bool = False) -> None:
+    """Variants the paper describes and replaces (see sidco.h); the defaults restore the method as evaluated."""
+    rc = lib().sidco_set_policy(int(gamma_exact), int(ratio_from_counts), int(adapt_reversed))
+    if rc:
+        raise SidcoError(rc, "sidco_set_policy")
 
 
 def sidco_reset_state(residual) -> None:

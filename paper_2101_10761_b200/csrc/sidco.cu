@@ -24,6 +24,7 @@ using sidco::kChunk;
 struct Params {
     double delta1 = 0.25, eps_H = 0.2, eps_L = 0.2;
     int Q = 5;
+    int gamma_exact = 0, ratio_counts = 0, adapt_rev = 0;      // sidco_set_policy
 };
 
 struct DeviceInfo {
@@ -393,6 +394,9 @@ int launch_compress(char* base, const Layout& L, int64_t d, int T, int S, int G,
     // 256-bit accesses to the residual and an fp32 gradient, 128-bit ones to a bf16 gradient
     a.vec_ok = (((uintptr_t)residual & 31u) | ((uintptr_t)grad & (grad_bf16 ? 15u : 31u))) == 0;
     a.grad_bf16 = grad_bf16 ? 1 : 0;
+    a.pol_gamma_exact = prm.gamma_exact;
+    a.pol_ratio_counts = prm.ratio_counts;
+    a.pol_adapt_rev = prm.adapt_rev;
     const Hooks& h = hooks();
     a.spec_enable = h.spec_enable;           // (the result is the same with or without the pre-selection)
     a.spin_limit = h.spin_limit;
@@ -661,6 +665,14 @@ int sidco_set_params(double delta1, double eps_H, double eps_L, int Q) {
     g_params.eps_H = eps_H;
     g_params.eps_L = eps_L;
     g_params.Q = Q;
+    return 0;
+}
+
+int sidco_set_policy(int gamma_exact, int ratio_from_counts, int adapt_reversed) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_params.gamma_exact = gamma_exact ? 1 : 0;
+    g_params.ratio_counts = ratio_from_counts ? 1 : 0;
+    g_params.adapt_rev = adapt_reversed ? 1 : 0;
     return 0;
 }
 

@@ -161,6 +161,10 @@ struct Args {
     int vec_ok;                  // grad and residual are 32-byte aligned (256-bit accesses)
     int spec_enable;             // candidate pre-selection in the first sweep (see P1)
     int grad_bf16;               // grad points to bf16 values, widened exactly to fp32 before the add
+    // variants the paper describes and replaces (sidco_set_policy; all zero: the method as evaluated)
+    int pol_gamma_exact;         // Corollary 1.2 with the maximum-likelihood shape and the exact quantile
+    int pol_ratio_counts;        // last stage's ratio = target count / exceedances the stage before it left
+    int pol_adapt_rev;           // Adapt_Stages with the opposite sign
     long long spin_limit;        // polls after which a bounded wait gives up (kSpinLimit unless a test shortens it)
     int drop_pub_seg;            // test hook: the published words of this segment are withheld (-1: none), so that
                                  // the runs waiting for them run into the bound
@@ -407,6 +411,88 @@ __device__ inline double gpd_step(double mean, double var, double ln_ratio, doub
 // Corollary 1.1 / 2.1.
 __device__ inline double exp_step(double mean, double ln_inv_ratio) { return mean * ln_inv_ratio; }
 
+// ---- special functions for the exact forms of Corollary 1.2 (policy pol_gamma_exact; one thread, fp64)
+
+// psi(x) and psi'(x), x > 0: recurrence up to x >= 8, then the asymptotic series.
+__device__ inline void digamma_trigamma(double x, double& psi, double& psi1) {
+    double a0 = 0.0, a1 = 0.0;
+    while (x < 8.0) {
+        const double r = 1.0 / x;
+        a0 -= r;
+        a1 += r * r;
+        x += 1.0;
+    }
+    const double r = 1.0 / x, f = r * r;
+    psi = a0 + log(x) - 0.5 * r - f * (1.0 / 12 - f * (1.0 / 120 - f * (1.0 / 252 - f * (1.0 / 240 - f / 132))));
+    psi1 = a1 + r + 0.5 * f + r * f * (1.0 / 6 - f * (1.0 / 30 - f * (1.0 / 42 - f / 30)));
+}
+
+// Maximum-likelihood gamma shape: the root of log(alpha) - psi(alpha) = s, Newton from the closed form.
+__device__ inline double gamma_shape_mle(double s, double alpha) {
+    for (int it = 0; it < 100; ++it) {
+        double psi, psi1;
+        digamma_trigamma(alpha, psi, psi1);
+        const double f = log(alpha) - psi - s;
+        double nw = alpha - f / (1.0 / alpha - psi1);
+        if (!(nw > 0.0)) nw = 0.5 * alpha;
+        const bool done = fabs(nw - alpha) <= 1e-15 * alpha;
+        alpha = nw;
+        if (done) break;
+    }
+    return alpha;
+}
+
+// Q(a, x), the regularised upper incomplete gamma function: power series of P below a + 1, continued fraction
+// of Q above.
+__device__ inline double gamma_upper_q(double a, double x) {
+    if (!(x > 0.0)) return 1.0;
+    const double log_front = a * log(x) - x - lgamma(a);
+    if (x < a + 1.0) {
+        double term = 1.0 / a, total = term;
+        for (int n = 1; n < 10000; ++n) {
+            term *= x / (a + n);
+            total += term;
+            if (fabs(term) <= 1e-17 * fabs(total)) break;
+        }
+        return 1.0 - total * exp(log_front);
+    }
+    const double tiny = 1e-300;
+    double b = x + 1.0 - a, c = 1.0 / tiny, d = 1.0 / b, h = d;
+    for (int i = 1; i < 10000; ++i) {
+        const double an = -(double)i * ((double)i - a);
+        b += 2.0;
+        d = an * d + b;
+        if (fabs(d) < tiny) d = tiny;
+        c = b + an / c;
+        if (fabs(c) < tiny) c = tiny;
+        d = 1.0 / d;
+        const double del = d * c;
+        h *= del;
+        if (fabs(del - 1.0) < 1e-16) break;
+    }
+    return h * exp(log_front);
+}
+
+// x with Q(a, x) = q: bracket by doubling, then Newton on log Q kept inside the bracket (bisection otherwise).
+__device__ inline double gamma_upper_quantile(double a, double q) {
+    if (q >= 1.0) return 0.0;
+    double lo = 0.0, hi = a > 1.0 ? a : 1.0;
+    for (int it = 0; it < 2000 && gamma_upper_q(a, hi) > q; ++it) { lo = hi; hi = 2.0 * hi; }
+    double x = 0.5 * (lo + hi);
+    const double lq = log(q);
+    for (int it = 0; it < 200; ++it) {
+        const double qx = gamma_upper_q(a, x);
+        if (qx > q) lo = x; else hi = x;
+        const double dens = exp((a - 1.0) * log(x) - x - lgamma(a));
+        double nw = (qx > 0.0 && dens > 0.0) ? x + (log(qx) - lq) * qx / dens : 0.5 * (lo + hi);
+        if (!(lo < nw && nw < hi)) nw = 0.5 * (lo + hi);
+        const bool done = fabs(nw - x) <= 1e-15 * x;
+        x = nw;
+        if (done) break;
+    }
+    return x;
+}
+
 // What the fitting thread hands to its own CTA (the other runs of the segment read SegDev::pub).
 struct Fit {
     double eta;
@@ -517,10 +603,15 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
             eta = mu * log(1.0 / rz);
             if (!(eta > 0.0)) eta = 0.0;
         } else {
-            const double alpha = (3.0 - s + sqrt((s - 3.0) * (s - 3.0) + 24.0 * s)) / (12.0 * s);
-            const double beta = mu / alpha;
-            eta = -beta * (log(rz) + lgamma(alpha));
-            if (eta <= 0.0) { status |= kStDegenerate; eta = 0.0; }
+            double alpha = (3.0 - s + sqrt((s - 3.0) * (s - 3.0) + 24.0 * s)) / (12.0 * s);
+            if (A.pol_gamma_exact) {
+                alpha = gamma_shape_mle(s, alpha);
+                eta = (mu / alpha) * gamma_upper_quantile(alpha, rz);
+            } else {
+                const double beta = mu / alpha;
+                eta = -beta * (log(rz) + lgamma(alpha));
+                if (eta <= 0.0) { status |= kStDegenerate; eta = 0.0; }
+            }
         }
     }
     // an empty segment takes part in no later phase: all its stages count as fitted here
@@ -534,15 +625,23 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
 // Stage index m >= 1 (eta_{m+1} in the paper's numbering) of an M_eff-stage segment from the shifted peaks
 // over prev = eta_m: n_e = #{|x| > eta_m}, Sy = sum(|x| - eta_m), Sy2 = sum(|x| - eta_m)^2.
 __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, double prev, int n_e, double Sy,
-                                  double Sy2, const LnTab& T) {
+                                  double Sy2, const LnTab& T, int n_seg) {
     double eta = prev;
     int status = 0;
     if (n_e > 0) {
         const int slot = ratio_slot(M_eff, m);
+        double ln = T.ln[slot], ln_inv = T.ln_inv[slot];
+        if (A.pol_ratio_counts && m + 1 == M_eff) {
+            // the last stage keeps the target count out of what the stage before it left
+            double ratio = A.delta * (double)n_seg / (double)n_e;
+            if (ratio > 1.0) ratio = 1.0;
+            ln = log(ratio);
+            ln_inv = log(1.0 / ratio);
+        }
         const double ybar = Sy / n_e;
         double inc;
-        if (A.sid == kSidExp) inc = exp_step(ybar, T.ln_inv[slot]);
-        else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, T.ln[slot], T.ln_inv[slot], status);
+        if (A.sid == kSidExp) inc = exp_step(ybar, ln_inv);
+        else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, ln, ln_inv, status);
         eta = prev + inc;
     }
     Fit f = publish_stage(A, T.call_id, sg, m + 1, m + 1 == M_eff, eta);
@@ -919,7 +1018,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                 // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
                 const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
                 const double prev = cached ? R.eta_prev[i2] : ld_cg(&sg->eta[stage - 1]);
-                f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T);
+                f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2]);
             }
             if (cached) {
                 R.thr[i2] = f.thr;
@@ -1661,8 +1760,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 const double k_avg = (double)k_sum / (double)A.Q;
                 const double k_target = A.delta * (double)A.seg_n[s];
                 int M = sg->M;
-                if (k_avg > k_target * (1.0 + A.eps_H)) M = M - 1;
-                if (k_avg < k_target * (1.0 - A.eps_L)) M = M + 1;
+                const int step = A.pol_adapt_rev ? -1 : 1;
+                if (k_avg > k_target * (1.0 + A.eps_H)) M = M - step;
+                if (k_avg < k_target * (1.0 - A.eps_L)) M = M + step;
                 if (M < 1) M = 1;
                 if (M > A.max_stages) M = A.max_stages;
                 sg->M = M;
