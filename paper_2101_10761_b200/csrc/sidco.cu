@@ -39,7 +39,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
-    size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, cta_desc;
+    size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, seg_tile0, tile_arr, tile_part, cta_desc;
     size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, cta_dbg, seg, ctl;
     size_t total;
 };
@@ -53,6 +53,10 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.seg_chunk0 = take(sizeof(int32_t) * (size_t)(S + 1));
     L.seg_n = take(sizeof(int32_t) * (size_t)(S + 1));
     L.seg_runs = take(sizeof(int32_t) * (size_t)(S + 1));
+    L.seg_tile0 = take(sizeof(int32_t) * (size_t)(S + 2));
+    const size_t tiles = (size_t)(T / sidco::kTile + S + 2);          // upper bound on the tiles of giant segments
+    L.tile_arr = take(sizeof(int32_t) * tiles);
+    L.tile_part = take(sizeof(double) * 3 * tiles);
     L.cta_desc = take(sizeof(int4) * (size_t)(G + 1));
     L.part = take(sizeof(double) * 3 * (size_t)(T + 1));
     L.part_n = take(sizeof(int32_t) * (size_t)(T + 1));
@@ -194,6 +198,7 @@ int launch_grid(const DeviceInfo& di) {
 struct HostTables {
     int32_t* chunk_start; int32_t* chunk_seg;                  // [T + 1]
     int32_t* seg_chunk0; int32_t* seg_n; int32_t* seg_runs;    // [S + 1]
+    int32_t* seg_tile0;                                         // [S + 1]
     int32_t* cta_chunk0;                                        // [G + 1]
     int4* cta_desc;                                             // [G + 1]
 };
@@ -220,6 +225,14 @@ int compute_tables(const int64_t* off, int S, int G, const HostTables& t) {
     t.seg_chunk0[S] = T;
     t.seg_n[S] = 0;
     t.seg_runs[S] = 0;
+    // tiles of the giant segments (summed in two levels)
+    int tiles = 0;
+    for (int s = 0; s < S; ++s) {
+        t.seg_tile0[s] = tiles;
+        const int chunks = t.seg_chunk0[s + 1] - t.seg_chunk0[s];
+        if (chunks > sidco::kGiantSeg) tiles += (chunks + sidco::kTile - 1) / sidco::kTile;
+    }
+    t.seg_tile0[S] = tiles;
     t.chunk_start[T] = (int32_t)off[S];
     t.chunk_seg[T] = 0;
     const double per_chunk = 128.0;
@@ -261,11 +274,11 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
 
     const size_t cap = (size_t)max_chunks(d, S) + 1;
     std::vector<int32_t> chunk_start(cap), chunk_seg(cap), seg_chunk0(S + 1), seg_n(S + 1), seg_runs(S + 1),
-        cta_chunk0(G + 1);
+        seg_tile0(S + 1), cta_chunk0(G + 1);
     std::vector<int4> cta_desc(G + 1);
     const int T = compute_tables(off, S, G, HostTables{chunk_start.data(), chunk_seg.data(), seg_chunk0.data(),
-                                                       seg_n.data(), seg_runs.data(), cta_chunk0.data(),
-                                                       cta_desc.data()});
+                                                       seg_n.data(), seg_runs.data(), seg_tile0.data(),
+                                                       cta_chunk0.data(), cta_desc.data()});
 
     const Layout L = make_layout(d, S, T, G);
     if (c->ws && c->ws_bytes < L.total) {
@@ -316,6 +329,8 @@ cudaError_t build_tables(Context* c, const int64_t* off, int S, cudaStream_t str
     if ((e = up(L.seg_chunk0, seg_chunk0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg_n, seg_n.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg_runs, seg_runs.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = up(L.seg_tile0, seg_tile0.data(), sizeof(int32_t) * (S + 1))) != cudaSuccess) return e;
+    if ((e = cudaMemset(base + L.tile_arr, 0, sizeof(int32_t) * (size_t)(T / sidco::kTile + S + 2))) != cudaSuccess) return e;
     if ((e = up(L.cta_desc, cta_desc.data(), sizeof(int4) * (G + 1))) != cudaSuccess) return e;
     if ((e = up(L.seg, seg_host.data(), sizeof(SegDev) * (S + 1))) != cudaSuccess) return e;
     if ((e = up(L.ctl, &ctl_host, sizeof(Control))) != cudaSuccess) return e;
@@ -364,6 +379,9 @@ int launch_compress(char* base, const Layout& L, int64_t d, int T, int S, int G,
     a.seg_chunk0 = (const int32_t*)(base + L.seg_chunk0);
     a.seg_n = (const int32_t*)(base + L.seg_n);
     a.seg_runs = (const int32_t*)(base + L.seg_runs);
+    a.seg_tile0 = (const int32_t*)(base + L.seg_tile0);
+    a.tile_arr = (int32_t*)(base + L.tile_arr);
+    a.tile_part = (double*)(base + L.tile_part);
     a.cta_desc = (const int4*)(base + L.cta_desc);
     a.part = (double*)(base + L.part);
     a.part_n = (int32_t*)(base + L.part_n);
@@ -504,6 +522,7 @@ struct StaticContext {
     int64_t offsets[kStaticMaxSegs + 1];
     int32_t chunk_start[kStaticMaxChunks + 1], chunk_seg[kStaticMaxChunks + 1];
     int32_t seg_chunk0[kStaticMaxSegs + 1], seg_n[kStaticMaxSegs + 1], seg_runs[kStaticMaxSegs + 1];
+    int32_t seg_tile0[kStaticMaxSegs + 1];
     int32_t cta_chunk0[kMaxGrid + 1];
     int4 cta_desc[kMaxGrid + 1];
     SegDev seg_init[kStaticMaxSegs + 1];
@@ -554,7 +573,7 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         const int G = launch_grid(*di);
         if (G > kMaxGrid) return SIDCO_E_SIZE;
         c.T = compute_tables(seg_offsets, n_segs, G, HostTables{c.chunk_start, c.chunk_seg, c.seg_chunk0, c.seg_n,
-                                                                c.seg_runs, c.cta_chunk0, c.cta_desc});
+                                                                c.seg_runs, c.seg_tile0, c.cta_chunk0, c.cta_desc});
         c.S = n_segs;
         c.G = G;
         for (int s = 0; s <= n_segs; ++s) c.offsets[s] = seg_offsets[s];
@@ -573,6 +592,8 @@ int sidco_compress_static(const float* grad, float* residual, const int64_t* seg
         if ((e = up(L.seg_chunk0, c.seg_chunk0, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg_n, c.seg_n, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg_runs, c.seg_runs, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = up(L.seg_tile0, c.seg_tile0, sizeof(int32_t) * (n_segs + 1))) != cudaSuccess) return (int)e;
+        if ((e = cudaMemsetAsync(c.base + L.tile_arr, 0, sizeof(int32_t) * (size_t)(c.T / sidco::kTile + n_segs + 2), stream)) != cudaSuccess) return (int)e;
         if ((e = up(L.cta_desc, c.cta_desc, sizeof(int4) * (c.G + 1))) != cudaSuccess) return (int)e;
         if ((e = up(L.seg, c.seg_init, sizeof(SegDev) * (n_segs + 1))) != cudaSuccess) return (int)e;
         // The array keeps whatever the last call left.  What must start at zero (the control block: finished-CTA
@@ -701,6 +722,7 @@ int sidco_reset_state(const float* residual) {
     std::memset(&ctl, 0, sizeof(Control));
     ctl.residual_is_zero = 1;
     if ((e = cudaMemset(base + c->L.cta_total, 0, sizeof(unsigned long long) * (c->G + 1))) != cudaSuccess) return (int)e;
+    if ((e = cudaMemset(base + c->L.tile_arr, 0, sizeof(int32_t) * (size_t)(c->T / sidco::kTile + c->S + 2))) != cudaSuccess) return (int)e;
     if ((e = cudaMemcpy(base + c->L.ctl, &ctl, sizeof(Control), cudaMemcpyHostToDevice)) != cudaSuccess) return (int)e;
     return 0;
 }

@@ -67,6 +67,8 @@ constexpr int kChunk = 1024;                      // window: elements per full c
 constexpr int kComp = 8;                          // elements per slot: one 32-byte access per lane
 constexpr int kSlots = kChunk / (32 * kComp);     // slots per lane per chunk (4)
 constexpr int kSmallSeg = 256;                    // segments of <= 256 chunks are summed by one warp
+constexpr int kGiantSeg = 4096;                   // segments of more chunks are summed in two levels:
+constexpr int kTile = 1024;                       // tiles of this many chunks first (by the run that completes a tile)
 constexpr int kSegCache = 256;                    // segments of a CTA run whose table entries sit in shared memory
 constexpr int kOutCache = 2048;                   // survivors of a run the shared-memory selection can hold
 constexpr int kSlotCap = 4096;                    // candidate slots (8 elements of one lane) a run can note
@@ -134,6 +136,9 @@ struct Args {
     const int32_t* seg_chunk0;   // [S + 1]
     const int32_t* seg_n;        // [S]
     const int32_t* seg_runs;     // [S] number of CTA runs that hold chunks of the segment
+    const int32_t* seg_tile0;    // [S + 1] first tile of the segment (segments of more than kGiantSeg chunks have tiles)
+    int32_t* tile_arr;           // [tiles] chunks of the tile whose partials are in (self-resetting)
+    double* tile_part;           // [tiles][3] sums over the tile's chunk partials
     const int4* cta_desc;        // [G] {first chunk, one past last chunk, first segment, segments} of the run
     // scratch
     double* part;                // [C][3] per-chunk partial sums
@@ -931,6 +936,7 @@ struct RunSegs {
     float* thr;                 // [kSegCache] thr_gt of the stage the phase shifts by; thr_ge of the last stage in P5a
     double* eta_prev;           // [kSegCache]
     volatile int* ok;           // [kSegCache] == phase tag once the two values above are valid
+    int c0, c1;                 // chunks of the run
     __device__ __forceinline__ void get(const Args& A, int i, int& a, int& b, int& r) const {
         if (i < kSegCache) { a = q0[i]; b = q1[i]; r = runs[i]; }
         else { a = A.seg_chunk0[seg_lo + i]; b = A.seg_chunk0[seg_lo + i + 1]; r = A.seg_runs[seg_lo + i]; }
@@ -1037,8 +1043,9 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
             if (q1 > q0) {
                 SegDev* sg = &A.seg[R.seg_lo + i];
                 const bool takes_part = stage == 0 || (i < kSegCache ? R.m_eff[i] : seg_stages(A, R.seg_lo + i, cap)) > stage;
-                bool complete = takes_part && runs == 1;
-                if (takes_part && runs > 1) {
+                const bool giant = q1 - q0 > kGiantSeg;
+                bool complete = takes_part && runs == 1 && !giant;
+                if (takes_part && runs > 1 && !giant) {
                     complete = atom_add_acquire(&sg->arrived, 1) == runs - 1;
                     if (complete) sg->arrived = 0;     // (the other runs' partials, read next, came with the acquire)
                 }
@@ -1046,10 +1053,28 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
                     if (q1 - q0 <= kSmallSeg) sm_small[atomicAdd(&sm_count[0], 1)] = i;
                     else sm_large[atomicAdd(&sm_count[1], 1)] = i;
                 }
+                if (takes_part && giant) {
+                    // A giant segment is summed in two levels, so that no single CTA has to read all its chunk
+                    // partials: tiles of kTile chunks (counted from the segment's first chunk, whatever the grid)
+                    // are summed by the run whose arrival completes the tile; the run that completes the last
+                    // tile adds the tile sums up and fits.
+                    const int ca = max(q0, R.c0), cb = min(q1, R.c1);
+                    const int t0 = A.seg_tile0[R.seg_lo + i];
+                    for (int t = (ca - q0) / kTile; t * kTile + q0 < cb; ++t) {
+                        const int ta = q0 + t * kTile, tb = min(ta + kTile, q1);
+                        const int mine = min(cb, tb) - max(ca, ta);
+                        const int old = atom_add_acquire(&A.tile_arr[t0 + t], mine);
+                        if (old + mine == tb - ta) {
+                            A.tile_arr[t0 + t] = 0;
+                            const int slot = atomicAdd(&sm_count[1], 1);
+                            if (slot < kThreads) sm_large[slot] = i | ((t + 1) << 20);      // (tile number + 1 above the segment)
+                        }
+                    }
+                }
             }
         }
         __syncthreads();
-        const int n_small = sm_count[0], n_large = sm_count[1];
+        const int n_small = sm_count[0], n_large = min(sm_count[1], kThreads);
         // Large segments (other runs wait for them) are fitted by two groups of twelve warps, two segments at
         // a time: threads stride over the chunk partials, fixed tree over the group.  The other eight warps
         // take the small segments meanwhile (all warps do if there is no large one).
@@ -1057,14 +1082,46 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         if (g < kFitGroups) {
             const int tg = threadIdx.x - g * 32 * kFitGroupWarps;
             for (int k = g; k < n_large; k += kFitGroups) {
-                const int i2 = sm_large[k];
+                const int i2 = sm_large[k] & 0xFFFFF, tile = (sm_large[k] >> 20) - 1;
                 int q0, q1, runs;
                 R.get(A, i2, q0, q1, runs);
                 SegDev* sg = &A.seg[R.seg_lo + i2];
                 const int M_state = (stage == 0 && tg == 0) ? (i2 < kSegCache ? R.m_eff[i2] : sg->M) : 0;
-                const Sums t = strided_partials(A, q0 + tg, q1, 32 * kFitGroupWarps);
-                Sums r = group_tree(t.a, t.b, t.n, sm_red + kFitGroupWarps * g, g);
-                if (tg < 32) fit_and_cache(sg, i2, M_state, r);
+                if (tile < 0) {
+                    const Sums t = strided_partials(A, q0 + tg, q1, 32 * kFitGroupWarps);
+                    Sums r = group_tree(t.a, t.b, t.n, sm_red + kFitGroupWarps * g, g);
+                    if (tg < 32) fit_and_cache(sg, i2, M_state, r);
+                } else {
+                    // one tile of a giant segment; if it is the segment's last, the tile sums and the fit
+                    const int t0 = A.seg_tile0[R.seg_lo + i2], n_tiles = (q1 - q0 + kTile - 1) / kTile;
+                    const int ta = q0 + tile * kTile, tb = min(ta + kTile, q1);
+                    const Sums t = strided_partials(A, ta + tg, tb, 32 * kFitGroupWarps);
+                    Sums r = group_tree(t.a, t.b, t.n, sm_red + kFitGroupWarps * g, g);
+                    if (tg < 32) {
+                        int last = 0;
+                        if (lane == 0) {
+                            double* tp = A.tile_part + 3 * (size_t)(t0 + tile);
+                            tp[0] = r.a; tp[1] = r.b; tp[2] = (double)r.n;
+                            __threadfence();
+                            last = atom_add_acquire(&sg->arrived, 1) == n_tiles - 1;
+                            if (last) sg->arrived = 0;
+                        }
+                        if (__shfl_sync(kFull, last, 0)) {
+                            double a = 0.0, b = 0.0, c = 0.0;
+                            for (int u = lane; u < n_tiles; u += 32) {             // lanes stride over the tiles
+                                const double* tp = A.tile_part + 3 * (size_t)(t0 + u);
+                                a += ld_cg(tp); b += ld_cg(tp + 1); c += ld_cg(tp + 2);
+                            }
+                            #pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) {
+                                a += __shfl_down_sync(kFull, a, o);
+                                b += __shfl_down_sync(kFull, b, o);
+                                c += __shfl_down_sync(kFull, c, o);
+                            }
+                            fit_and_cache(sg, i2, M_state, Sums{a, b, (int)c});
+                        }
+                    }
+                }
             }
         }
         // small segments: one warp each, lanes stride over the chunk partials, fixed shuffle tree
@@ -1182,7 +1239,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     __syncthreads();
     const unsigned call_id = sm_call;
     const bool res_zero = sm_reszero != 0;
-    RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok};
+    RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok, c0, c1};
     const LnTab T{A.ln_ratio, A.ln_inv_ratio, call_id};
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep

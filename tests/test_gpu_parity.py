@@ -207,6 +207,40 @@ print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [o
     assert outs[0] == outs[1] == outs[2]
 
 
+def test_giant_segments_are_summed_in_tiles_whatever_the_grid():
+    """A segment of more than 4096 chunks is summed in two levels (tiles counted from the segment's first
+    chunk).  Thresholds must match the oracle and be bit-identical for every grid."""
+    import json
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import json, sys, numpy as np
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+from oracle import sidco_oracle as O
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, check_parity, f32
+sizes = [777, 6_000_123, 4_300_000, 50]
+off = W.offsets_from_sizes(sizes)
+run = GpuRun(off)
+res_o = np.zeros(int(off[-1]), np.float32)
+for call in range(2):
+    g = W.ragged_case(300 + call, sizes, 1e-3)
+    ora = O.sidco_compress(g, res_o, off, f32(0.001), 2, -3)
+    out = run.step(g, f32(0.001), 2, -3)
+    check_parity(out, ora, off)
+    res_o = ora.residual
+print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [int(out["out_k"][-1])]))
+''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for grid in ("100000", "37", "5"):
+        env = dict(os.environ, SIDCO_GRID=grid)
+        r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
+        assert r.returncode == 0, r.stderr[-3000:]
+        outs.append(json.loads(r.stdout.strip().splitlines()[-1]))
+    assert outs[0] == outs[1] == outs[2]
+
+
 @pytest.mark.parametrize("sid", SIDS)
 @pytest.mark.parametrize("M", [2, 3])
 def test_ties_with_the_first_threshold(sid, M):
