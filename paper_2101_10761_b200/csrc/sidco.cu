@@ -132,12 +132,12 @@ void sidco_internal::note_launch() { g_launches.fetch_add(1); }
 
 namespace {
 
-template <int SID>
+template <int SID, bool EXACT = false>
 cudaError_t occupancy(int* out) {
-    cudaError_t e = cudaFuncSetAttribute(sidco::sidco_persistent_kernel<SID>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         sidco::kDynSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(sidco::sidco_persistent_kernel<SID, EXACT>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, sidco::kDynSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sidco::sidco_persistent_kernel<SID>, kThreads,
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sidco::sidco_persistent_kernel<SID, EXACT>, kThreads,
                                                          sidco::kDynSmemBytes);
 }
 
@@ -148,12 +148,14 @@ cudaError_t device_info(int dev, DeviceInfo** out) {
         cudaError_t e = cudaGetDeviceProperties(&prop, dev);
         if (e != cudaSuccess) return e;
         if (!prop.cooperativeLaunch) return cudaErrorNotSupported;
-        int a = 0, b = 0, c = 0;
+        int a = 0, b = 0, c = 0, x = 0;
         if ((e = occupancy<0>(&a)) != cudaSuccess) return e;
         if ((e = occupancy<1>(&b)) != cudaSuccess) return e;
         if ((e = occupancy<2>(&c)) != cudaSuccess) return e;
+        if ((e = occupancy<1, true>(&x)) != cudaSuccess) return e;
         int occ = a < b ? a : b;
         occ = occ < c ? occ : c;
+        occ = occ < x ? occ : x;
         if (occ < 1) return cudaErrorLaunchOutOfResources;
         di.sm_count = prop.multiProcessorCount;
         di.ctas_per_sm = occ;
@@ -422,7 +424,8 @@ int launch_compress(char* base, const Layout& L, int64_t d, int T, int S, int G,
 
     void* kargs[] = {(void*)&a};
     const void* fn = sid == 0   ? (const void*)sidco::sidco_persistent_kernel<0>
-                     : sid == 1 ? (const void*)sidco::sidco_persistent_kernel<1>
+                     : sid == 1 ? (prm.gamma_exact ? (const void*)sidco::sidco_persistent_kernel<1, true>
+                                                   : (const void*)sidco::sidco_persistent_kernel<1>)
                                 : (const void*)sidco::sidco_persistent_kernel<2>;
     const cudaError_t e = launch_persistent(fn, G, kargs, stream);
     if (e != cudaSuccess) return (int)e;

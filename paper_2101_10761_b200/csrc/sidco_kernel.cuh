@@ -283,6 +283,18 @@ __device__ __forceinline__ Sums warp_tree(double a, double b, int n) {
     return Sums{a, b, n};
 }
 
+// The same tree over the sums a sweep of family SID needs: `b` only where a second moment (GPD) is kept, the
+// count by a warp reduction (integer addition has no order to fix).  Result valid in lane 0.
+template <bool WithB>
+__device__ __forceinline__ Sums chunk_tree(double a, double b, int n) {
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_down_sync(kFull, a, o);
+        if (WithB) b += __shfl_down_sync(kFull, b, o);
+    }
+    return Sums{a, WithB ? b : 0.0, (int)__reduce_add_sync(kFull, n)};
+}
+
 // Block-wide sums with a fixed tree (warp trees, then one warp over the 32 warp results);
 // result valid in thread 0.
 __device__ __forceinline__ Sums block_tree(double a, double b, int n, double (*sm)[3]) {
@@ -571,6 +583,9 @@ __device__ inline Fit publish_stage(const Args& A, unsigned call_id, SegDev* sg,
 
 // Stage 1 from the segment sums: S1 = sum|x|, and S2 = sum x^2 (GPD) or SL = sum log|x| over the
 // n_nz nonzero magnitudes (gamma).
+// EXACT: the exact forms of Corollary 1.2 are compiled in (a kernel instantiation of its own, so that the default
+// one does not carry their code and registers).
+template <bool EXACT>
 __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, double S1, double S2_or_SL,
                                  int n_nz, int cap, const LnTab& T) {
     int M;
@@ -609,7 +624,7 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
             if (!(eta > 0.0)) eta = 0.0;
         } else {
             double alpha = (3.0 - s + sqrt((s - 3.0) * (s - 3.0) + 24.0 * s)) / (12.0 * s);
-            if (A.pol_gamma_exact) {
+            if (EXACT && A.pol_gamma_exact) {
                 alpha = gamma_shape_mle(s, alpha);
                 eta = (mu / alpha) * gamma_upper_quantile(alpha, rz);
             } else {
@@ -999,7 +1014,7 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
 // fitted at once; one shared with other runs is fitted by the run that arrives last.
 // The fitting thread also puts the result into this CTA's own parameter cache, tagged for the phase that
 // uses it next, so that the CTA does not wait for its own publication to come back through L2.
-template <class AfterSweep>
+template <bool EXACT, class AfterSweep>
 __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
                                                int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3],
                                                int stamp_slot, const AfterSweep& after_sweep) {
@@ -1019,7 +1034,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
         Fit f{};
         if (lane == 0) {
             if (stage == 0) {
-                f = fit_stage1(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
+                f = fit_stage1<EXACT>(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
             } else {
                 // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
                 const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
@@ -1148,7 +1163,7 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
 // the kernel
 // ----------------------------------------------------------------------------
 
-template <int SID>
+template <int SID, bool EXACT = false>
 __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __grid_constant__ Args A) {
     extern __shared__ __align__(16) float sm_stage[];        // [kWarps][kChunk] (kDynSmemBytes)
     __shared__ double sm_red[kWarps][3];
@@ -1389,7 +1404,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
                 second = (double)esum * 0.693147180559945309417232121458 + log(m);   // used from lane 0 only
             }
-            Sums r = warp_tree(s1, SID == kSidGamma ? 0.0 : second, nnz);
+            Sums r = chunk_tree<SID == kSidGpd>(s1, second, nnz);
             if (lane == 0 && SIDCO_IN_RANGE(A, c, A.C)) {
                 A.part[3 * (size_t)c + 0] = r.a;
                 A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
@@ -1398,7 +1413,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             cur = nxt;
         }
     }
-    arrive_and_fit(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6, fetch_slots);
+    arrive_and_fit<EXACT>(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6, fetch_slots);
     if (threadIdx.x == 0) sm_next = 0;
     __syncthreads();
     const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
@@ -1431,17 +1446,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     #pragma unroll
                     for (int j = 0; j < kSlots; ++j) {
                         float big = 0.0f;
+                        double sj = 0.0, sj2 = 0.0;        // (one short chain per slot, added up in slot order)
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc) {
                             const float a = fabsf(v[j][cc]);
                             big = fmaxf(big, a);
                             if (a > sv.thr_gt) {
                                 const double y = (double)a - sv.eta_prev;
-                                sy += y;
-                                if (SID != kSidExp) sy2 = fma(y, y, sy2);
+                                sj += y;
+                                if (SID != kSidExp) sj2 = fma(y, y, sj2);
                                 mask |= 1u << (8 * j + cc);
                             }
                         }
+                        sy += sj;
+                        if (SID != kSidExp) sy2 += sj2;
                         if (flag_chunk && big >= tau2) list_slot(wb + lane * kComp + j * 256, cur.seg - R.seg_lo);
                     }
                     if (!flag_chunk) {
@@ -1489,7 +1507,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         if (lane == 0) A.side_cnt[c] = kept;
                         A.side_mask[(size_t)c * 32 + lane] = keep_mask;
                     }
-                    Sums r = warp_tree(sy, sy2, __popc(mask));
+                    Sums r = chunk_tree<SID != kSidExp>(sy, sy2, __popc(mask));
                     if (lane == 0) {
                         A.part[3 * (size_t)c + 0] = r.a;
                         A.part[3 * (size_t)c + 1] = r.b;
@@ -1499,7 +1517,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 cur = nxt;
             }
         }
-        arrive_and_fit(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8, fetch_slots);
+        arrive_and_fit<EXACT>(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8, fetch_slots);
         if (threadIdx.x == 0) sm_next = 0;
         __syncthreads();
         SIDCO_STAMP(if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns());
@@ -1539,7 +1557,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             take(x0, 128 * t + 4 * lane);
                             take(x1, 128 * (t + 1) + 4 * lane);
                         }
-                        Sums r = warp_tree(sy, sy2, cnt);
+                        Sums r = chunk_tree<SID != kSidExp>(sy, sy2, cnt);
                         if (lane == 0) {
                             A.part[3 * (size_t)c + 0] = r.a;
                             A.part[3 * (size_t)c + 1] = r.b;
@@ -1549,7 +1567,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     cur = nxt;
                 }
             }
-            arrive_and_fit(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10, [] {});
+            arrive_and_fit<EXACT>(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10, [] {});
             if (threadIdx.x == 0) sm_next = 0;
             __syncthreads();
             SIDCO_STAMP(if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns());
@@ -1870,7 +1888,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // are done here, spread over the grid.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
         if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) {
-            const Fit f = fit_stage1(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
+            const Fit f = fit_stage1<EXACT>(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
             record_stage(&A.seg[s], 0, f, 0, 1);
             seg_finish(s, f.M_eff, 0, f.thr);
         }
