@@ -40,7 +40,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // Offsets of the workspace parts for d elements, S segments, T chunks and G CTAs.
 struct Layout {
     size_t chunk_start, chunk_seg, seg_chunk0, seg_n, seg_runs, seg_tile0, tile_arr, tile_part, cta_desc;
-    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, cta_dbg, seg, ctl;
+    size_t part, part_n, side_cnt, chunk_cnt, side_val, side_mask, stage_idx, stage_val, cta_total, cta_dir, cta_ns, cta_dbg, slot_spill_e, slot_spill_seg, seg, ctl;
     size_t total;
 };
 
@@ -70,6 +70,8 @@ Layout make_layout(int64_t d, int S, int64_t T, int G) {
     L.cta_dir = take(sizeof(int32_t) * (size_t)(G + 1));
     L.cta_ns = take(sizeof(unsigned long long) * 4 * (size_t)(G + 1));
     L.cta_dbg = take(sizeof(int) * 8 * (size_t)(G + 1));
+    L.slot_spill_e = take(sizeof(int32_t) * (size_t)(d / 8 + G + 8));
+    L.slot_spill_seg = take((size_t)(d / 8 + G + 8));
     L.seg = take(sizeof(SegDev) * (size_t)(S + 1));
     L.ctl = take(sizeof(Control));
     L.total = o;
@@ -397,6 +399,8 @@ int launch_compress(char* base, const Layout& L, int64_t d, int T, int S, int G,
     a.cta_dir = (int32_t*)(base + L.cta_dir);
     a.cta_ns = (unsigned long long*)(base + L.cta_ns);
     a.cta_dbg = (int*)(base + L.cta_dbg);
+    a.slot_spill_e = (int32_t*)(base + L.slot_spill_e);
+    a.slot_spill_seg = (unsigned char*)(base + L.slot_spill_seg);
     a.seg = (SegDev*)(base + L.seg);
     a.ctl = (Control*)(base + L.ctl);
     a.delta = (double)delta;

@@ -153,6 +153,8 @@ struct Args {
     int32_t* cta_dir;            // [G] 1: this CTA's next first sweep runs over descending chunks
     unsigned long long* cta_ns;  // [G][4] globaltimer when the CTA finished its P1, P3, last P4, P5a sweep
     int* cta_dbg;                // [G][8] profile builds: how the final selection of the run went
+    int32_t* slot_spill_e;       // [d / 8 + G] candidate slots beyond what shared memory holds: first element ...
+    unsigned char* slot_spill_seg;   // ... and segment of the run (a run's entries start at its first element / 8)
     SegDev* seg;                 // [S]
     Control* ctl;
     // scalars
@@ -1268,9 +1270,15 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // first kSlotPre slots; a run with more reads the others from acc when it compares them).
     auto list_slot = [&](int e, int seg_i) {
         const int q = atomicAdd(&sm_nslot, 1);
-        if (q < kSlotCap && SIDCO_IN_RANGE(A, e + kComp - 1, A.d) && SIDCO_IN_RANGE(A, seg_i, kSegCache)) {
+        if (!SIDCO_IN_RANGE(A, e + kComp - 1, A.d) || !SIDCO_IN_RANGE(A, seg_i, kSegCache)) return;
+        if (q < kSlotCap) {
             sm_slot_e[q] = e;
             sm_slot_seg[q] = (unsigned char)seg_i;
+        } else {
+            // beyond what shared memory holds: to the run's part of the spill arrays (a run has at most one slot
+            // per 8 elements, and its part starts at its first element / 8, so it cannot run out)
+            const size_t at = (size_t)(sm_run_e[0] >> 3) + blockIdx.x + (size_t)(q - kSlotCap);
+            if (SIDCO_IN_RANGE(A, at, (size_t)(A.d >> 3) + A.G)) { A.slot_spill_e[at] = e; A.slot_spill_seg[at] = (unsigned char)seg_i; }
         }
     };
     // Start the copies of the slots listed since the last call (all threads; after the sweep's stores are
@@ -1587,21 +1595,33 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     publish_params(A, R, 0, -1, 100);          // one thread per segment waits (bounded) for its last threshold
     cp_async_wait_all();                       // this thread's share of the candidate slots has arrived
     __syncthreads();
-    const bool cand_overflow = sm_nslot > kSlotCap;
     // the recorded candidates of cached segment i contain all its survivors among the chunks that recorded some
-    auto seg_cand_ok = [&](int i) -> bool { return !cand_overflow && sm_tau[i] > 0.0f && R.thr[i] >= sm_tau[i]; };
+    auto seg_cand_ok = [&](int i) -> bool { return sm_tau[i] > 0.0f && R.thr[i] >= sm_tau[i]; };
     const int run_e0 = sm_run_e[0], run_e1 = sm_run_e[1];
     const int win0 = run_e0 >> 10;
     const int n_win = c1 > c0 ? ((run_e1 - 1) >> 10) - win0 + 1 : 0;
     bool path_a = run_n_seg <= kSegCache && n_win <= kWinCap;
     int cta_count = 0;
+    // Lists longer than shared memory holds continue in the run's own part of the staging buffers (one entry per
+    // element of the run at most; the first half takes the unordered list, the second the ordered one).
+    const int run_n = run_e1 - run_e0;
+    int* const g_uidx = A.stage_idx + run_e0;
+    float* const g_uval = A.stage_val + run_e0;
+    int* const g_oidx = A.stage_idx + run_e0 + run_n / 2;
+    float* const g_oval = A.stage_val + run_e0 + run_n / 2;
+    const int list_cap = max(kOutCache, run_n / 2 - 8);           // denser selections go the other way
 
-    // Survivor into the run's unordered list (path A).
-    auto append = [&](int e, float val, int seg_i) {
-        const int sp = atomicAdd(&sm_nsurv, 1);
+    // Survivors into the run's unordered list (path A).  reserve(): room for n survivors that lie in one
+    // 1024-element window and one segment (one atomic each on the list, the window and the segment counter,
+    // whatever n); put(): one of them at its reserved place.
+    auto reserve = [&](int n, int e_any, int seg_i) -> int {
+        if (SIDCO_IN_RANGE(A, (e_any >> 10) - win0, n_win)) atomicAdd(&sm_wcnt[(e_any >> 10) - win0], n);
+        if (SIDCO_IN_RANGE(A, seg_i, kSegCache)) atomicAdd(&sm_segk[seg_i], n);
+        return atomicAdd(&sm_nsurv, n);
+    };
+    auto put = [&](int sp, int e, float val) {
         if (sp < kOutCache) { sm_oidx[sp] = e; sm_oval[sp] = val; }
-        if (SIDCO_IN_RANGE(A, (e >> 10) - win0, n_win)) atomicAdd(&sm_wcnt[(e >> 10) - win0], 1);
-        if (SIDCO_IN_RANGE(A, seg_i, kSegCache)) atomicAdd(&sm_segk[seg_i], 1);
+        else if (sp < list_cap) { g_uidx[sp - kOutCache] = e; g_uval[sp - kOutCache] = val; }
     };
 
     // The warps' pass over chunks.  list_n >= 0: the chunks sm_rest[0 .. list_n); < 0: all chunks of the run,
@@ -1700,11 +1720,13 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     if (to_list) {
                         const int seg_i = cur.seg - R.seg_lo;
                         unsigned m = surv;
+                        int sp = m ? reserve(__popc(m), wb, seg_i) : 0;       // (a chunk lies in one window)
                         while (m) {
                             const int bit = __ffs(m) - 1;
                             m &= m - 1u;
                             const int e = e0 + (bit >> 3) * 256 + (bit & 7);
-                            if (SIDCO_IN_RANGE(A, e, A.d)) append(e, __ldcg(A.residual + e), seg_i);
+                            if (SIDCO_IN_RANGE(A, e, A.d)) put(sp, e, __ldcg(A.residual + e));
+                            ++sp;
                         }
                     } else {
                         cnt = ordered_emit(surv, lo, [&](int p, int j, int cc) {
@@ -1732,11 +1754,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         for (int w = threadIdx.x; w < n_win; w += kThreads) { sm_wcnt[w] = 0; sm_wfill[w] = 0; }
         // A segment that recorded candidates which turned out unusable (its threshold fell below the candidate
         // threshold): its chunks made of whole slots are in no list yet.  (A first or last chunk that is not
-        // recorded no candidates and was listed by the sweep.)  If the candidate slots overflowed, every chunk is
-        // read instead.
-        if (cand_overflow) {
-            if (threadIdx.x == 0) sm_nrest = kThreads + 1;
-        } else if (vec_ok) {
+        // recorded no candidates and was listed by the sweep.)
+        if (vec_ok) {
             // (such segments are rare: they are collected first, then all threads list their chunks)
             for (int i = threadIdx.x; i < R.n_seg; i += kThreads)
                 if (sm_q1[i] > sm_q0[i] && sm_tau[i] > 0.0f && !seg_cand_ok(i)) sm_list[atomicAdd(&sm_count[0], 1)] = i;
@@ -1757,12 +1776,13 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             if (threadIdx.x == 0) sm_count[0] = 0;
         }
         __syncthreads();
-        const int n_slot = min(sm_nslot, kSlotCap);
+        const int n_slot = sm_nslot;
+        const size_t spill0 = (size_t)(run_e0 >> 3) + blockIdx.x;
         for (int q = threadIdx.x; q < n_slot; q += kThreads) {
-            const int i = sm_slot_seg[q];
+            const int i = q < kSlotCap ? sm_slot_seg[q] : A.slot_spill_seg[spill0 + (q - kSlotCap)];
             if (seg_cand_ok(i)) {
                 const float thr = R.thr[i];
-                const int e = sm_slot_e[q];
+                const int e = q < kSlotCap ? sm_slot_e[q] : __ldcg(A.slot_spill_e + spill0 + (q - kSlotCap));
                 float x[kComp];
                 if (q < kSlotPre) {
                     #pragma unroll
@@ -1772,16 +1792,23 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     const float4 b = __ldcg(reinterpret_cast<const float4*>(A.residual + e) + 1);
                     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
                 }
+                unsigned m = 0;
                 #pragma unroll
                 for (int cc = 0; cc < kComp; ++cc)
-                    if (fabsf(x[cc]) >= thr) append(e + cc, x[cc], i);
+                    if (fabsf(x[cc]) >= thr) m |= 1u << cc;
+                if (m) {
+                    int sp = reserve(__popc(m), e, i);                       // (a slot lies in one window)
+                    #pragma unroll
+                    for (int cc = 0; cc < kComp; ++cc)
+                        if ((m >> cc) & 1u) put(sp++, e + cc, x[cc]);
+                }
             }
         }
         const bool scan_all = sm_nrest > kThreads;
         warp_pass(scan_all ? -1 : sm_nrest, true, true);
         __syncthreads();
         cta_count = sm_nsurv;
-        if (cta_count > kOutCache) {
+        if (cta_count > list_cap) {
             // too many for the list: start over the other way (nothing has been modified yet)
             path_a = false;
             for (int i = threadIdx.x; i < kSegCache; i += kThreads) sm_segk[i] = 0;
@@ -1907,12 +1934,24 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             if (w2 < n_win) sm_wcnt[w2] = ex;
             if (w2 + 1 < n_win) sm_wcnt[w2 + 1] = ex + a0;
             __syncthreads();
-            for (int q = threadIdx.x; q < cta_count; q += kThreads) {
-                const int e = sm_oidx[q], w = (e >> 10) - win0;
-                const int slot = sm_wcnt[w] + atomicAdd(&sm_wfill[w], 1);
-                if (!SIDCO_IN_RANGE(A, slot, kOutCache)) continue;
-                sm_cidx[slot] = e;                       // (the candidate arrays are free by now)
-                sm_cval[slot] = sm_oval[q];
+            const bool in_smem = cta_count <= kOutCache;
+            for (int q0 = 0; q0 < cta_count; q0 += kThreads) {
+                const int q = q0 + (int)threadIdx.x;
+                const bool on = q < cta_count;
+                const int e = on ? (q < kOutCache ? sm_oidx[q] : g_uidx[q - kOutCache]) : 0;
+                const int w = on ? (e >> 10) - win0 : -1;
+                const float val = on ? (q < kOutCache ? sm_oval[q] : g_uval[q - kOutCache]) : 0.0f;
+                // (neighbours in the list mostly share a window: one atomic per window and warp)
+                const unsigned peers = __match_any_sync(kFull, w);
+                const int leader = __ffs(peers) - 1;
+                int first = 0;
+                if (on && lane == leader) first = atomicAdd(&sm_wfill[w], __popc(peers));
+                first = __shfl_sync(kFull, first, leader);
+                if (!on) continue;
+                const int slot = sm_wcnt[w] + first + __popc(peers & ((1u << lane) - 1u));
+                if (!SIDCO_IN_RANGE(A, slot, in_smem ? kOutCache : run_n - run_n / 2)) continue;
+                if (in_smem) { sm_cidx[slot] = e; sm_cval[slot] = val; }      // (the candidate values' space is free by now)
+                else { g_oidx[slot] = e; g_oval[slot] = val; }
             }
             __syncthreads();
         }
@@ -1939,15 +1978,56 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         int run_base = sm_base;
         if (cta == A.G - 1 && threadIdx.x == 0) A.out_k[A.S] = run_base + cta_count;
         if (path_a) {
+            const bool in_smem = cta_count <= kOutCache;
+            const int* oidx = in_smem ? sm_cidx : g_oidx;
+            const float* oval = in_smem ? sm_cval : g_oval;
+            constexpr int kDenseWin = 32;       // windows with more survivors are ranked through a bitmap, by one warp
             for (int q = threadIdx.x; q < cta_count; q += kThreads) {
-                const int e = sm_cidx[q], w = (e >> 10) - win0;
-                const int g0 = sm_wcnt[w], g1 = g0 + sm_wfill[w];
+                const int e = oidx[q], w = (e >> 10) - win0;
+                const int g0 = sm_wcnt[w], n_w = sm_wfill[w];
+                if (n_w > kDenseWin) continue;
                 int rank = 0;
-                for (int t = g0; t < g1; ++t) rank += sm_cidx[t] < e;
+                for (int t = g0; t < g0 + n_w; ++t) rank += oidx[t] < e;
                 if (!SIDCO_IN_RANGE(A, run_base + g0 + rank, A.d) || !SIDCO_IN_RANGE(A, e, A.d)) continue;
                 A.out_idx[run_base + g0 + rank] = e;
-                A.out_val[run_base + g0 + rank] = sm_cval[q];
+                A.out_val[run_base + g0 + rank] = oval[q];
                 A.residual[e] = 0.0f;
+            }
+            // A window with many survivors: its 1024 positions as a bitmap (one word per lane), prefix counts over
+            // the words, and every survivor's rank is the number of set bits below its own.
+            {
+                unsigned* bm = reinterpret_cast<unsigned*>(sm_scan) + warp * 32;
+                int* pf = sm_list + warp * 32;
+                for (int w = warp; w < n_win; w += kWarps) {
+                    const int n_w = sm_wfill[w];
+                    if (n_w <= kDenseWin) continue;
+                    const int g0 = sm_wcnt[w];
+                    bm[lane] = 0u;
+                    __syncwarp();
+                    for (int t = lane; t < n_w; t += 32) {
+                        const int o = oidx[g0 + t] & (kChunk - 1);
+                        atomicOr(&bm[o >> 5], 1u << (o & 31));
+                    }
+                    __syncwarp();
+                    const int mine = __popc(bm[lane]);
+                    int incl = mine;
+                    #pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int t = __shfl_up_sync(kFull, incl, o);
+                        if (lane >= o) incl += t;
+                    }
+                    pf[lane] = incl - mine;
+                    __syncwarp();
+                    for (int t = lane; t < n_w; t += 32) {
+                        const int e = oidx[g0 + t], o = e & (kChunk - 1);
+                        const int rank = pf[o >> 5] + __popc(bm[o >> 5] & ((1u << (o & 31)) - 1u));
+                        if (!SIDCO_IN_RANGE(A, run_base + g0 + rank, A.d) || !SIDCO_IN_RANGE(A, e, A.d)) continue;
+                        A.out_idx[run_base + g0 + rank] = e;
+                        A.out_val[run_base + g0 + rank] = oval[g0 + t];
+                        A.residual[e] = 0.0f;
+                    }
+                    __syncwarp();
+                }
             }
         }
         // path B: chunk bases by a block-wide exclusive scan, kThreads chunks at a time
