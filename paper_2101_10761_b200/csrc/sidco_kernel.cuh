@@ -71,9 +71,11 @@ constexpr int kGiantSeg = 4096;                   // segments of more chunks are
 constexpr int kTile = 1024;                       // tiles of this many chunks first (by the run that completes a tile)
 constexpr int kSegCache = 256;                    // segments of a CTA run whose table entries sit in shared memory
 constexpr int kOutCache = 2048;                   // survivors of a run the shared-memory selection can hold
-constexpr int kSlotCap = 4096;                    // candidate slots (8 elements of one lane) a run can note
+constexpr int kSlotCap = 3072;                    // candidate slots (8 elements of one lane) a run can note
 constexpr int kSlotPre = 1280;                    // the first of them have their values copied to shared memory ahead
 constexpr int kWinCap = 2048;                     // 1024-element windows of a run the shared-memory selection covers
+constexpr int kScWin = 1024;                      // ... and the windows a run may have for warps to calibrate candidate thresholds themselves
+constexpr float kScRatio = 0.8f;                  // a warp's own candidate threshold: this fraction of the exponential estimate from its last chunk
 static_assert(kSlotPre * kComp >= 2 * kOutCache, "the ordered survivors reuse the candidate values' space");
 constexpr float kSpecRatio = 0.85f;                // candidate threshold = this fraction of the last eta
 constexpr int kMaxStages = 8;
@@ -587,7 +589,7 @@ __device__ inline Fit publish_stage(const Args& A, unsigned call_id, SegDev* sg,
 // n_nz nonzero magnitudes (gamma).
 // EXACT: the exact forms of Corollary 1.2 are compiled in (a kernel instantiation of its own, so that the default
 // one does not carry their code and registers).
-template <bool EXACT>
+template <int SID, bool EXACT>
 __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, double S1, double S2_or_SL,
                                  int n_nz, int cap, const LnTab& T) {
     int M;
@@ -609,9 +611,9 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
     } else if (S1 == 0.0) {
         status |= kStAllZero;
         eta = __longlong_as_double(0x7ff0000000000000ll);
-    } else if (A.sid == kSidExp) {
+    } else if (SID == kSidExp) {
         eta = exp_step(S1 / n, T.ln_inv[slot]);
-    } else if (A.sid == kSidGpd) {
+    } else if (SID == kSidGpd) {
         const double mu = S1 / n;
         eta = gpd_step(mu, S2_or_SL / n - mu * mu, T.ln[slot], T.ln_inv[slot], status);
     } else {
@@ -646,6 +648,7 @@ __device__ inline Fit fit_stage1(const Args& A, SegDev* sg, int M_state, int n, 
 
 // Stage index m >= 1 (eta_{m+1} in the paper's numbering) of an M_eff-stage segment from the shifted peaks
 // over prev = eta_m: n_e = #{|x| > eta_m}, Sy = sum(|x| - eta_m), Sy2 = sum(|x| - eta_m)^2.
+template <int SID>
 __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, double prev, int n_e, double Sy,
                                   double Sy2, const LnTab& T, int n_seg) {
     double eta = prev;
@@ -662,7 +665,7 @@ __device__ inline Fit fit_stage_m(const Args& A, SegDev* sg, int m, int M_eff, d
         }
         const double ybar = Sy / n_e;
         double inc;
-        if (A.sid == kSidExp) inc = exp_step(ybar, ln_inv);
+        if (SID == kSidExp) inc = exp_step(ybar, ln_inv);
         else inc = gpd_step(ybar, Sy2 / n_e - ybar * ybar, ln, ln_inv, status);
         eta = prev + inc;
     }
@@ -845,7 +848,8 @@ constexpr int kSidePre4 = 2;                      // the same in the sweeps that
 // small on purpose: what shared memory takes, the L1 loses, and the first sweep's bandwidth suffers.)
 constexpr int kStageRow = kChunk / kSlots + 8;    // floats of staging per warp: one slot row plus the carried tail
 constexpr int kStageBytes = kWarps * kStageRow * (int)sizeof(float);
-constexpr int kDynSmemBytes = kStageBytes + kSlotPre * kComp * (int)sizeof(float) + kSlotCap * ((int)sizeof(int) + 1);
+constexpr int kDynSmemBytes = kStageBytes + kSlotPre * kComp * (int)sizeof(float) + kSlotCap * ((int)sizeof(int) + 1)
+                            + kScWin * ((int)sizeof(float) + (int)sizeof(unsigned short) + 1);
 static_assert(kStageBytes >= kOutCache * 8 + kWinCap * 8, "survivor list and window counters fit over the staging area");
 
 // Positions of a lane's kept elements in the chunk's dense, index-ordered side region.  `mask` has bit
@@ -1016,32 +1020,23 @@ __device__ __forceinline__ void view_load(const Args& A, const RunSegs& R, SegVi
 // fitted at once; one shared with other runs is fitted by the run that arrives last.
 // The fitting thread also puts the result into this CTA's own parameter cache, tagged for the phase that
 // uses it next, so that the CTA does not wait for its own publication to come back through L2.
-template <bool EXACT, class AfterSweep>
-__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
-                                               int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3],
-                                               int stamp_slot, const AfterSweep& after_sweep) {
-    __threadfence();
-    __syncthreads();
-    after_sweep();       // (the CTA's sweep is over and its stores are fenced)
-    SIDCO_STAMP(if (threadIdx.x == 0) {                       // this CTA's sweep is over
-        const unsigned long long now = global_ns();
-        A.cta_ns[4 * blockIdx.x + (stage < 2 ? stage : 2)] = now;
-        if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
-    });
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // one warp: its first lane fits segment i2 of the run from its sums (M_state and r are that lane's),
-    // publishes, and fills the CTA's own cache entry; all lanes then write the stage's record
-    auto fit_and_cache = [&](SegDev* sg, int i2, int M_state, const Sums& r) {
+// One warp: its first lane fits segment i2 of the run from its sums (M_state and r are that lane's), publishes, and
+// fills the CTA's own cache entry; all lanes then write the stage's record.
+template <int SID, bool EXACT>
+__device__ __forceinline__ void fit_and_cache(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
+                                              SegDev* sg, int i2, int M_state, const Sums& r) {
+    const int lane = threadIdx.x & 31;
+    {
         const bool cached = i2 < kSegCache;
         Fit f{};
         if (lane == 0) {
             if (stage == 0) {
-                f = fit_stage1<EXACT>(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
+                f = fit_stage1<SID, EXACT>(A, sg, M_state, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2], r.a, r.b, r.n, cap, T);
             } else {
                 // this run swept the segment in the phase that just ended, so its cache holds eta_{stage}
                 const int M_eff = cached ? R.m_eff[i2] : seg_stages(A, R.seg_lo + i2, cap);
                 const double prev = cached ? R.eta_prev[i2] : ld_cg(&sg->eta[stage - 1]);
-                f = fit_stage_m(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2]);
+                f = fit_stage_m<SID>(A, sg, stage, M_eff, prev, r.n, r.a, r.b, T, cached ? R.n[i2] : A.seg_n[R.seg_lo + i2]);
             }
             if (cached) {
                 R.thr[i2] = f.thr;
@@ -1051,6 +1046,15 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
             }
         }
         record_stage(sg, stage, warp_broadcast(f), lane, 32);
+    }
+}
+
+template <int SID, bool EXACT>
+__device__ __forceinline__ void fit_phase(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
+                                          int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    auto fit_and_cache = [&](SegDev* sg, int i2, int M_state, const Sums& r) {
+        sidco::fit_and_cache<SID, EXACT>(A, R, stage, cap, T, sg, i2, M_state, r);
     };
     for (int base = 0; base < R.n_seg; base += kThreads) {
         const int i = base + (int)threadIdx.x;
@@ -1161,6 +1165,21 @@ __device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, 
     }
 }
 
+template <int SID, bool EXACT, class AfterSweep>
+__device__ __forceinline__ void arrive_and_fit(const Args& A, const RunSegs& R, int stage, int cap, const LnTab& T,
+                                               int* sm_small, int* sm_large, int* sm_count, double (*sm_red)[3],
+                                               int stamp_slot, const AfterSweep& after_sweep) {
+    __threadfence();
+    __syncthreads();
+    after_sweep();       // (the CTA's sweep is over and its stores are fenced)
+    SIDCO_STAMP(if (threadIdx.x == 0) {                       // this CTA's sweep is over
+        const unsigned long long now = global_ns();
+        A.cta_ns[4 * blockIdx.x + (stage < 2 ? stage : 2)] = now;
+        if (blockIdx.x == 0) A.ctl->t_ns[stamp_slot] = now;
+    });
+    fit_phase<SID, EXACT>(A, R, stage, cap, T, sm_small, sm_large, sm_count, sm_red);
+}
+
 // ----------------------------------------------------------------------------
 // the kernel
 // ----------------------------------------------------------------------------
@@ -1196,6 +1215,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     float* const sm_slot_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sm_stage) + kStageBytes);
     int* const sm_slot_e = reinterpret_cast<int*>(sm_slot_val + kSlotPre * kComp);
     unsigned char* const sm_slot_seg = reinterpret_cast<unsigned char*>(sm_slot_e + kSlotCap);
+    // A segment without a candidate threshold from the previous call (the first call on a fresh residual): a warp
+    // derives one from the chunk of the segment it read last.  Per window: the threshold used (0: none), the chunk
+    // (relative to the run) and the cached segment, for the check against the fitted threshold.
+    float* const sm_wtau = reinterpret_cast<float*>(sm_slot_seg + kSlotCap);
+    unsigned short* const sm_wchunk = reinterpret_cast<unsigned short*>(sm_wtau + kScWin);
+    unsigned char* const sm_wseg = reinterpret_cast<unsigned char*>(sm_wchunk + kScWin);
     int* const sm_cidx = reinterpret_cast<int*>(sm_slot_val);
     float* const sm_cval = sm_slot_val + kOutCache;
     __shared__ unsigned sm_call;
@@ -1221,6 +1246,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     if (threadIdx.x == 0) sm_mloc = 1;
     if (threadIdx.x == 0) { sm_next = kWarps; sm_resweep = 0; sm_nrest = 0; sm_nslot = 0; sm_nfetched = 0; sm_nsurv = 0; }
     if (threadIdx.x < 2) sm_count[threadIdx.x] = 0;
+    if (threadIdx.x < kScWin) sm_wtau[threadIdx.x] = 0.0f;
     if (threadIdx.x < 2) sm_run_e[threadIdx.x] = __ldg(A.chunk_start + (threadIdx.x ? c1 : c0));
     // What changes from call to call lives in the workspace (and is advanced by the CTA that finishes the call
     // last, long after every CTA has read it here).  The loads are issued now and their values handed to the
@@ -1243,7 +1269,9 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             sm_q0[i] = q0; sm_q1[i] = q1; sm_runs[i] = A.seg_runs[run_seg_lo + i];
             sm_meff[i] = m;
             sm_segn[i] = A.seg_n[run_seg_lo + i];
-            const float tau = A.seg[run_seg_lo + i].spec_thr;
+            // (a segment of one window at most records every slot that is not all zero: its threshold moves too
+            // much from call to call for a fraction of the last one to hold)
+            const float tau = A.seg_n[run_seg_lo + i] <= kChunk ? 1.17549435e-38f : A.seg[run_seg_lo + i].spec_thr;
             sm_tau[i] = (A.spec_enable && m <= 2 && tau > 0.0f) ? tau : -1.0f;
             sm_ok[i] = 0;
             sm_segk[i] = 0;
@@ -1258,6 +1286,13 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     const bool res_zero = sm_reszero != 0;
     RunSegs R{call_id, run_seg_lo, run_n_seg, sm_q0, sm_q1, sm_runs, sm_meff, sm_segn, sm_tau, sm_thr, sm_eta, sm_ok, c0, c1};
     const LnTab T{A.ln_ratio, A.ln_inv_ratio, call_id};
+    const int sc_win0 = sm_run_e[0] >> 10;
+    const bool sc_on = A.spec_enable && vec_ok && c1 > c0 && run_n_seg <= kSegCache && c1 - c0 < 65536 &&
+                       ((sm_run_e[1] - 1) >> 10) - sc_win0 + 1 <= kScWin;
+    auto sc_note = [&](int wb, float t, int c, int seg_i) {
+        const int w = (wb >> 10) - sc_win0;
+        if (SIDCO_IN_RANGE(A, w, kScWin)) { sm_wtau[w] = t; sm_wchunk[w] = (unsigned short)(c - c0); sm_wseg[w] = (unsigned char)seg_i; }
+    };
 
     // Candidate threshold of a segment for this call (segments with one or two stages use one: the sweep
     // that precedes their last fit records which slots may hold survivors).  It depends on state the
@@ -1306,6 +1341,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     {
         int tau_seg = -1, seg_m = 1;
         float tau = 3.4e38f;       // candidate threshold of the chunk's segment (huge: none)
+        const float sc_ln = sc_on ? kScRatio * (float)T.ln_inv[1] : 0.0f;
         const bool keep = true;    // ask for L2 residency of the acc lines
         Desc cur = first_desc;
         while (cur.c >= 0) {
@@ -1339,7 +1375,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
             };
 
+            bool sc_chunk = false;
+            float bigs[kSlots];
             if (vec_ok && lo == wb && hi == wb + kChunk && SIDCO_IN_RANGE(A, wb + kChunk - 1, A.d) && SIDCO_IN_RANGE(A, c, A.C)) {
+                // no threshold from the previous call: the candidates are chosen below, by an estimate from the chunk itself
+                sc_chunk = sc_on && seg_m == 1 && !(tau < 3.0e38f);
                 #pragma unroll
                 for (int b = 0; b < kSlots; b += 2) {
                     F8 g8[2], r8[2];
@@ -1359,10 +1399,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             big = fmaxf(big, fabsf(a));
                         }
                         st8_res(A.residual + e0 + (b + j) * 256, r8[j], keep);
+                        bigs[b + j] = big;
                         if (big >= tau) list_slot(e0 + (b + j) * 256, cur.seg - R.seg_lo);
                     }
                 }
-                if (seg_m == 1 && !(tau < 3.0e38f)) list_chunk(c);        // single stage, no candidates recorded
+                if (seg_m == 1 && !(tau < 3.0e38f) && !sc_chunk) list_chunk(c);      // single stage, no candidates recorded
             } else {
                 // a ragged chunk made of whole slots records candidates like a full one
                 const bool whole_slots = vec_ok && ((lo | hi) & (kComp - 1)) == 0;
@@ -1418,10 +1459,20 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 A.part[3 * (size_t)c + 1] = SID == kSidGamma ? second : r.b;
                 A.part_n[c] = r.n;
             }
+            if (sc_chunk) {
+                // (the exponential form of the threshold, on this chunk's mean, scaled down; whether it was low
+                // enough is checked against the fitted threshold before its candidates are used)
+                const float mean = __shfl_sync(kFull, (float)r.a, 0) * (1.0f / kChunk);
+                const float tau_c = mean > 0.0f ? mean * sc_ln : 1.17549435e-38f;
+                #pragma unroll
+                for (int j = 0; j < kSlots; ++j)
+                    if (bigs[j] >= tau_c) list_slot(e0 + j * 256, cur.seg - R.seg_lo);
+                if (lane == 0) sc_note(wb, tau_c, c, cur.seg - R.seg_lo);
+            }
             cur = nxt;
         }
     }
-    arrive_and_fit<EXACT>(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6, fetch_slots);
+    arrive_and_fit<SID, EXACT>(A, R, 0, cap, T, sm_list, sm_scan, sm_count, sm_red, 6, fetch_slots);
     if (threadIdx.x == 0) sm_next = 0;
     __syncthreads();
     const int M_max_eff = sm_mloc;       // phases this CTA runs; other CTAs may run more or fewer
@@ -1432,6 +1483,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         publish_params(A, R, 1, 0, 1);
         {
             SegView sv;
+            const float sc_ln = sc_on ? kScRatio * (float)T.ln_inv[2] : 0.0f;
             Desc cur = fetch_desc(A, queue.next(!p1_desc), false);
             while (cur.c >= 0) {
                 const Desc nxt = fetch_desc(A, queue.next(!p1_desc), false);
@@ -1446,7 +1498,10 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     // Stage 2 is the last stage of a two-stage segment: nothing reads its exceedances again except
                     // the final selection, which can work from slot flags (as after P1 for one stage).
                     const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
-                    const bool flag_chunk = tau2 > 0.0f && vec_ok && ((lo | hi) & (kComp - 1)) == 0;
+                    // (without one from the previous call: by an estimate from the chunk itself, below)
+                    const bool sc_chunk = sc_on && sv.M_eff == 2 && !(tau2 > 0.0f) && lo == wb && hi == wb + kChunk;
+                    const bool flag_chunk = sc_chunk || (tau2 > 0.0f && vec_ok && ((lo | hi) & (kComp - 1)) == 0);
+                    float bigs[kSlots];
                     // (elements outside the chunk read as zero and the threshold is never negative, so they
                     // pass no strict compare)
                     unsigned mask = 0;
@@ -1468,7 +1523,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         }
                         sy += sj;
                         if (SID != kSidExp) sy2 += sj2;
-                        if (flag_chunk && big >= tau2) list_slot(wb + lane * kComp + j * 256, cur.seg - R.seg_lo);
+                        bigs[j] = big;
+                        if (flag_chunk && !sc_chunk && big >= tau2) list_slot(wb + lane * kComp + j * 256, cur.seg - R.seg_lo);
                     }
                     if (!flag_chunk) {
                         list_chunk(c);
@@ -1521,11 +1577,22 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         A.part[3 * (size_t)c + 1] = r.b;
                         A.part_n[c] = r.n;              // exceedances (the next fit's count)
                     }
+                    if (sc_chunk) {
+                        // (the exponential form of the stage's increment on this chunk's mean exceedance, scaled down)
+                        const float sum_y = __shfl_sync(kFull, (float)r.a, 0);
+                        const int n_y = __shfl_sync(kFull, r.n, 0);
+                        float tau_c = n_y > 0 ? (float)sv.eta_prev + sum_y / (float)n_y * sc_ln : sv.thr_gt;
+                        if (!(tau_c > 0.0f)) tau_c = 1.17549435e-38f;
+                        #pragma unroll
+                        for (int j = 0; j < kSlots; ++j)
+                            if (bigs[j] >= tau_c) list_slot(wb + lane * kComp + j * 256, cur.seg - R.seg_lo);
+                        if (lane == 0) sc_note(wb, tau_c, c, cur.seg - R.seg_lo);
+                    }
                 }
                 cur = nxt;
             }
         }
-        arrive_and_fit<EXACT>(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8, fetch_slots);
+        arrive_and_fit<SID, EXACT>(A, R, 1, cap, T, sm_list, sm_scan, sm_count, sm_red, 8, fetch_slots);
         if (threadIdx.x == 0) sm_next = 0;
         __syncthreads();
         SIDCO_STAMP(if (stamper) A.ctl->t_ns[9] = A.ctl->t_ns[2] = A.ctl->t_ns[3] = global_ns());
@@ -1575,7 +1642,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     cur = nxt;
                 }
             }
-            arrive_and_fit<EXACT>(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10, [] {});
+            arrive_and_fit<SID, EXACT>(A, R, m, cap, T, sm_list, sm_scan, sm_count, sm_red, 10, [] {});
             if (threadIdx.x == 0) sm_next = 0;
             __syncthreads();
             SIDCO_STAMP(if (stamper) A.ctl->t_ns[11] = A.ctl->t_ns[3] = global_ns());
@@ -1595,8 +1662,11 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     publish_params(A, R, 0, -1, 100);          // one thread per segment waits (bounded) for its last threshold
     cp_async_wait_all();                       // this thread's share of the candidate slots has arrived
     __syncthreads();
+    SIDCO_STAMP(if (threadIdx.x == 0 && M_max_eff == 1) A.cta_ns[4 * cta + 1] = global_ns());     // (single-stage runs: thresholds known)
     // the recorded candidates of cached segment i contain all its survivors among the chunks that recorded some
     auto seg_cand_ok = [&](int i) -> bool { return sm_tau[i] > 0.0f && R.thr[i] >= sm_tau[i]; };
+    // the same for a full chunk whose warp used its own estimate (0 if it used none)
+    auto sc_tau_of = [&](int e) -> float { return sc_on ? sm_wtau[(e >> 10) - sc_win0] : 0.0f; };
     const int run_e0 = sm_run_e[0], run_e1 = sm_run_e[1];
     const int win0 = run_e0 >> 10;
     const int n_win = c1 > c0 ? ((run_e1 - 1) >> 10) - win0 + 1 : 0;
@@ -1653,10 +1723,12 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             }
             const int c = cur.c, lo = cur.lo, hi = cur.hi;
             const int wb = lo & ~(kChunk - 1);
-            const bool cand_chunk = seg_cand && vec_ok && ((lo | hi) & (kComp - 1)) == 0;
+            const float wt = (lo == wb && hi == wb + kChunk) ? sc_tau_of(wb) : 0.0f;
+            const bool cand_chunk = (seg_cand && vec_ok && ((lo | hi) & (kComp - 1)) == 0) || wt > 0.0f;
             int cnt = 0;
             const bool chunk_ok = SIDCO_IN_RANGE(A, c, A.C) && SIDCO_IN_RANGE(A, lo, A.d) && SIDCO_IN_RANGE(A, hi - 1, A.d);
-            if (chunk_ok && !(skip_covered && cand_chunk && seg_covered)) {
+            const bool covered = wt > 0.0f ? sv.thr_ge >= wt : seg_covered;
+            if (chunk_ok && !(skip_covered && cand_chunk && covered)) {
                 unsigned surv = 0;
                 float v[kSlots][kComp];
                 // a whole-slot chunk of a candidate-recording two-stage segment has no side region: it is read from acc
@@ -1772,19 +1844,56 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     }
                 }
             }
+            // likewise a full chunk whose warp estimated too high
+            if (sc_on)
+                for (int w = threadIdx.x; w < n_win; w += kThreads) {
+                    const float t = sm_wtau[w];
+                    if (t > 0.0f && !(R.thr[sm_wseg[w]] >= t)) {
+                        const int q = atomicAdd(&sm_nrest, 1);
+                        if (q < kThreads) sm_rest[q] = sm_wchunk[w];
+                    }
+                }
             __syncthreads();
             if (threadIdx.x == 0) sm_count[0] = 0;
         }
         __syncthreads();
+        // The few listed chunks that are made of whole slots join the candidates, slot by slot and without
+        // condition (this keeps them out of the warps' pass, whose set-up costs more than the comparisons here).
+        const int n_cand = sm_nslot, n_rest0 = sm_nrest;
+        const int n_pre = sm_nfetched;          // candidates whose values were copied to shared memory
+        __syncthreads();
+        if (vec_ok && n_rest0 > 0 && n_rest0 <= kThreads && n_cand + (kChunk / kComp) * n_rest0 <= kSlotCap) {
+            for (int r = warp; r < n_rest0; r += kWarps) {
+                const int c = c0 + sm_rest[r];
+                const int lo = __ldg(A.chunk_start + c), hi = __ldg(A.chunk_start + c + 1);
+                if (((lo | hi) & (kComp - 1)) == 0) {
+                    const int seg_i = __ldg(A.chunk_seg + c) - R.seg_lo;
+                    #pragma unroll
+                    for (int j = 0; j < kSlots; ++j) {
+                        const int e = (lo & ~(kChunk - 1)) + lane * kComp + j * 256;
+                        if (e >= lo && e + kComp <= hi) list_slot(e, seg_i);
+                    }
+                } else if (lane == 0) {
+                    sm_list[atomicAdd(&sm_count[0], 1)] = sm_rest[r];
+                }
+            }
+            __syncthreads();
+            const int n_keep = sm_count[0];
+            if ((int)threadIdx.x < n_keep) sm_rest[threadIdx.x] = sm_list[threadIdx.x];
+            __syncthreads();
+            if (threadIdx.x == 0) { sm_nrest = n_keep; sm_count[0] = 0; }
+            __syncthreads();
+        }
         const int n_slot = sm_nslot;
         const size_t spill0 = (size_t)(run_e0 >> 3) + blockIdx.x;
         for (int q = threadIdx.x; q < n_slot; q += kThreads) {
             const int i = q < kSlotCap ? sm_slot_seg[q] : A.slot_spill_seg[spill0 + (q - kSlotCap)];
-            if (seg_cand_ok(i)) {
-                const float thr = R.thr[i];
-                const int e = q < kSlotCap ? sm_slot_e[q] : __ldcg(A.slot_spill_e + spill0 + (q - kSlotCap));
+            const int e = q < kSlotCap ? sm_slot_e[q] : __ldcg(A.slot_spill_e + spill0 + (q - kSlotCap));
+            const float thr = R.thr[i];
+            const float wt = sm_tau[i] > 0.0f ? 0.0f : sc_tau_of(e);
+            if (q >= n_cand || seg_cand_ok(i) || (wt > 0.0f && thr >= wt)) {
                 float x[kComp];
-                if (q < kSlotPre) {
+                if (q < n_pre) {
                     #pragma unroll
                     for (int cc = 0; cc < kComp; ++cc) x[cc] = sm_slot_val[q * kComp + cc];
                 } else {
@@ -1804,6 +1913,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                 }
             }
         }
+        SIDCO_STAMP(if (threadIdx.x == 0 && M_max_eff == 1) A.cta_ns[4 * cta + 2] = global_ns());     // (... and candidates compared)
         const bool scan_all = sm_nrest > kThreads;
         warp_pass(scan_all ? -1 : sm_nrest, true, true);
         __syncthreads();
@@ -1915,7 +2025,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     // are done here, spread over the grid.
     for (int s = cta * kThreads + (int)threadIdx.x; s < A.S; s += A.G * kThreads)
         if (A.seg_chunk0[s + 1] == A.seg_chunk0[s]) {
-            const Fit f = fit_stage1<EXACT>(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
+            const Fit f = fit_stage1<SID, EXACT>(A, &A.seg[s], A.seg[s].M, 0, 0.0, 0.0, 0, cap, T);
             record_stage(&A.seg[s], 0, f, 0, 1);
             seg_finish(s, f.M_eff, 0, f.thr);
         }
