@@ -312,8 +312,10 @@ int sidco_release_all(void);
 /* Switches for tests; production code has no reason to call this.
  *   grid                  > 0: launch with at most this many CTAs (contexts created afterwards); 0: all the device
  *                         holds.  Starts from the environment variable SIDCO_GRID, if set.
- *   spec_enable           0: the first sweep records no candidate slots and the final selection re-reads acc in full
- *                         (results are the same either way).  Starts from SIDCO_SPEC, if set.
+ *   spec_enable           0: the sweeps record no candidate slots and the final selection re-reads acc in full;
+ *                         2: candidate thresholds are set too high on purpose, so that the final selection finds
+ *                         most of them unusable and takes its other routes (results are the same in every mode).
+ *                         Starts from SIDCO_SPEC, if set.
  *   spin_limit            polls after which a bounded wait inside the kernel gives up and raises SIDCO_ST_TIMEOUT;
  *                         0 restores the default (about one second).
  *   drop_publication_seg  >= 0: the kernel withholds the published threshold words of this segment, so that the

@@ -117,7 +117,7 @@ Hooks& hooks() {
             const int want = atoi(env);
             if (want >= 1) g_hooks.grid = want;
         }
-        if (const char* env = getenv("SIDCO_SPEC")) g_hooks.spec_enable = env[0] == '0' ? 0 : 1;
+        if (const char* env = getenv("SIDCO_SPEC")) g_hooks.spec_enable = env[0] == '0' ? 0 : (env[0] == '2' ? 2 : 1);
     }
     return g_hooks;
 }
@@ -851,7 +851,7 @@ int sidco_set_test_hooks(int grid, int spec_enable, long long spin_limit, int dr
     std::lock_guard<std::mutex> lock(g_mu);
     Hooks& h = hooks();
     h.grid = grid;
-    h.spec_enable = spec_enable ? 1 : 0;
+    h.spec_enable = spec_enable == 2 ? 2 : (spec_enable ? 1 : 0);
     h.spin_limit = spin_limit ? spin_limit : sidco::kSpinLimit;
     h.drop_pub_seg = drop_publication_seg;
     return 0;

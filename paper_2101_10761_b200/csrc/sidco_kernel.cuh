@@ -1341,7 +1341,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
     {
         int tau_seg = -1, seg_m = 1;
         float tau = 3.4e38f;       // candidate threshold of the chunk's segment (huge: none)
-        const float sc_ln = sc_on ? kScRatio * (float)T.ln_inv[1] : 0.0f;
+        const float sc_ln = sc_on ? (A.spec_enable == 2 ? 2.0f : kScRatio) * (float)T.ln_inv[1] : 0.0f;
         const bool keep = true;    // ask for L2 residency of the acc lines
         Desc cur = first_desc;
         while (cur.c >= 0) {
@@ -1483,7 +1483,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
         publish_params(A, R, 1, 0, 1);
         {
             SegView sv;
-            const float sc_ln = sc_on ? kScRatio * (float)T.ln_inv[2] : 0.0f;
+            const float sc_ln = sc_on ? (A.spec_enable == 2 ? 2.0f : kScRatio) * (float)T.ln_inv[2] : 0.0f;
             Desc cur = fetch_desc(A, queue.next(!p1_desc), false);
             while (cur.c >= 0) {
                 const Desc nxt = fetch_desc(A, queue.next(!p1_desc), false);
@@ -1983,7 +1983,8 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
             sg->calls = calls;
             sg->k_sum = k_sum;
         }
-        sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? kSpecRatio * thr : -1.0f;
+        // (test mode 2 sets it too high on purpose, so that the next call finds its candidates unusable)
+        sg->spec_thr = (thr > 0.0f && thr < 3.0e38f) ? (A.spec_enable == 2 ? 1.25f : kSpecRatio) * thr : -1.0f;
     };
     for (int ib = 0; ib < R.n_seg; ib += kThreads) {
         const int i = ib + (int)threadIdx.x;

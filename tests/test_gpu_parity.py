@@ -241,6 +241,41 @@ print(json.dumps([[d.eta[m].hex() for m in range(3)] for d in out["debug"]] + [i
     assert outs[0] == outs[1] == outs[2]
 
 
+@pytest.mark.parametrize("mode", ["0", "2"])
+def test_selection_routes_agree_with_the_oracle(mode):
+    """The final selection has several routes (recorded candidate slots, listed chunks joined to them slot by slot,
+    the warps' pass over chunks, the per-chunk staging).  Mode 0 records no candidates at all; mode 2 sets every
+    candidate threshold too high, so that most recorded candidates are found unusable.  Both must reproduce the
+    oracle over several calls, for one- and two-stage segments, ragged and tiny segments included."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import sys, numpy as np
+sys.path.insert(0, %r); sys.path.insert(0, %r)
+from oracle import sidco_oracle as O
+from paper_2101_10761_b200 import workloads as W
+from parity_util import GpuRun, check_parity, f32
+sizes = [40_000, 64, 300_000, 7, 1024, 123_457, 2048, 16, 700_000, 33]
+off = W.offsets_from_sizes(sizes)
+for sid, ms, delta in ((0, 1, 0.001), (0, -2, 0.001), (2, 3, 0.01), (1, -2, 0.05)):
+    run = GpuRun(off)
+    res_o = np.zeros(int(off[-1]), np.float32)
+    state = O.new_state(len(sizes))
+    for call in range(4):
+        g = W.ragged_case(900 + call, sizes, 1e-3)
+        ora = O.sidco_compress(g, res_o, off, f32(delta), sid, ms, state=state)
+        out = run.step(g, f32(delta), sid, ms)
+        check_parity(out, ora, off)
+        res_o = ora.residual
+    run.close()
+print("ok")
+''' % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SIDCO_SPEC=mode)
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and r.stdout.strip().endswith("ok"), (r.stdout[-500:], r.stderr[-3000:])
+
+
 @pytest.mark.parametrize("sid", SIDS)
 @pytest.mark.parametrize("M", [2, 3])
 def test_ties_with_the_first_threshold(sid, M):
