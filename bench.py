@@ -68,7 +68,8 @@ FLUSH_BYTES = 256 << 20    # L2 flush between cold calls: one write of this many
 # DRAM bytes per launch of the persistent kernel on config 4 (dram__bytes_read.sum + dram__bytes_write.sum of
 # one ncu capture, mean over the ten launches of a run, summarised under profiles/), keyed by (sid, max_stages).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    (0, 4): 237.9e6,
+    (0, 4): 231.4e6,
+    (0, -4): 371.7e6,
 }
 
 
