@@ -1358,19 +1358,24 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
 
             double s1 = 0.0, s2 = 0.0, prod = 1.0;
             int esum = 0, nnz = 0;
-            auto accumulate = [&](float x) {
+            // `cc` is the element's place in its slot.  Sum of log|x| = (sum of exponents) * ln 2 + log(product of
+            // mantissas): the magnitudes are multiplied in fp64 as they are, and after every fourth place of a slot
+            // the product's exponent moves to an integer sum (four fp32 magnitudes cannot leave the fp64 range);
+            // one log per chunk.
+            auto accumulate = [&](float x, int cc) {
                 const float a = fabsf(x);
                 const double ad = (double)a;
                 s1 += ad;
                 if (SID == kSidGpd) s2 = fma(ad, ad, s2);
                 if (SID == kSidGamma) {
                     if (a > 0.0f) {
-                        // log|x| = exponent * ln 2 + log(mantissa): exponents are summed as integers,
-                        // mantissas multiplied in fp64, one log per chunk.
-                        const long long bits = __double_as_longlong(ad);
-                        esum += (int)(bits >> 52) - 1023;
-                        prod *= __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
+                        prod *= ad;
                         ++nnz;
+                    }
+                    if ((cc & 3) == 3) {
+                        const long long bits = __double_as_longlong(prod);
+                        esum += (int)(bits >> 52) - 1023;
+                        prod = __longlong_as_double((bits & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
                     }
                 }
             };
@@ -1395,7 +1400,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         for (int cc = 0; cc < kComp; ++cc) {
                             const float a = res_zero ? g8[j].v[cc] : g8[j].v[cc] + r8[j].v[cc];
                             r8[j].v[cc] = a;
-                            accumulate(a);
+                            accumulate(a, cc);
                             big = fmaxf(big, fabsf(a));
                         }
                         st8_res(A.residual + e0 + (b + j) * 256, r8[j], keep);
@@ -1421,7 +1426,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                         #pragma unroll
                         for (int cc = 0; cc < kComp; ++cc) {
                             r.v[cc] = res_zero ? g.v[cc] : g.v[cc] + r.v[cc];
-                            accumulate(r.v[cc]);
+                            accumulate(r.v[cc], cc);
                             big = fmaxf(big, fabsf(r.v[cc]));
                         }
                         st8_res(A.residual + e, r, keep);
@@ -1431,7 +1436,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                             if (e + cc >= lo && e + cc < hi) {
                                 const float a = ld1_grad(A.grad, e + cc, g_bf16) + (res_zero ? 0.0f : A.residual[e + cc]);
                                 A.residual[e + cc] = a;
-                                accumulate(a);
+                                accumulate(a, cc);
                             }
                         }
                     }
