@@ -5,8 +5,8 @@
 // (one per SM, 32 warps) owns one contiguous run of chunks for the whole call, so
 // what it wrote in one phase (acc, side buffers) it re-reads itself in the next.
 // Inside a run the warps pull chunks from a shared-memory queue and work on them
-// without any block-level synchronisation: a chunk is loaded, reduced with warp
-// shuffles, and compacted with ballots by one warp.  A CTA moves from one phase to
+// without any block-level synchronisation: a chunk is loaded and reduced with warp
+// shuffles by one warp.  A CTA moves from one phase to
 // the next on its own: a run that needs a segment's threshold waits (bounded) on
 // that segment's published word {call number, stages fitted, threshold}, which
 // the run completing the segment's statistics stores.  There is no grid-wide
@@ -17,31 +17,38 @@
 //   P1  acc = grad + residual (stored over residual) and the stage-1 statistics
 //       of every chunk; the CTA whose run completes a segment sums the per-chunk
 //       partials in chunk order and fits eta_1 (Corollaries 1.1-1.3).  For
-//       single-stage segments the sweep also records, per lane and 8-element
-//       slot, whether some |x| >= tau, tau being 0.8 times the segment's threshold
-//       of the previous call: if the new eta turns out >= tau (checked per segment)
-//       P5a fetches only the flagged slots of acc instead of all of it; otherwise
-//       it reads all of acc, so the result never depends on tau
+//       single-stage segments the sweep also notes, in shared memory, the place of
+//       every 8-element slot of a lane in which some |x| >= tau, tau being 0.85
+//       times the segment's final threshold of the previous call (without one --
+//       the first call on a fresh residual -- 0.8 times the exponential-form
+//       threshold of the chunk's own mean, remembered per window).  If the new
+//       threshold turns out >= tau (checked per segment or window) the final
+//       selection compares only the noted slots; otherwise it reads the chunks
+//       concerned again, so the result never depends on tau
 //   P3  (segments with M >= 2) statistics of the shifted peaks |x| - eta_1 over
 //       the exceedances |x| > eta_1 (Lemma 2 / Corollary 2.1) and fit of eta_2.
-//       Two-stage segments record slot flags here (as P1 does for one stage);
+//       Two-stage segments note candidate slots here (as P1 does for one stage);
 //       segments with more stages copy their exceedances into the chunk's side
-//       region, lane by lane (each lane keeps the values it holds, and a 32-bit mask
-//       says which of its 32 elements they are), with no ordering work at all: the
-//       later statistics need no order, and the few final survivors get theirs back
-//       from the mask
+//       region, dense and in index order (positions from two packed warp scans,
+//       one slot row at a time through a shared-memory staging row, 16-byte
+//       stores), together with a 32-bit mask per lane that says which of its 32
+//       elements they are
 //   P4  (m = 3..M) statistics of side-region entries above eta_{m-1}; fit eta_m
-//   P5a survivors |x| >= eta_M staged per chunk in ascending order, selected
-//       residual entries zeroed.  A block-wide pass lists the flagged slots of
-//       the run's full chunks (and all slots of its ragged chunks) in shared
-//       memory and fetches them in one wave; a per-warp loop takes what that
-//       pass cannot (invalid flags: all of acc; three or more stages: the side
-//       region)
+//   P5a survivors |x| >= eta_M.  The usual way stays in shared memory: one thread
+//       per noted slot compares it with the final threshold (the first noted slots
+//       have their values in shared memory already, copied asynchronously behind
+//       the fits), the few chunks without usable candidates are added slot by slot
+//       or read by the warps (three or more stages: from the side region), and all
+//       survivors of the run end up in one unordered list that is put in index
+//       order by counting per 1024-element window and ranking inside a window.
+//       Nothing is modified before the list is known to fit; otherwise (a large
+//       fraction selected) the warps stage every chunk's survivors in order in the
+//       chunk's staging region
 //   P5b base of the run = published counts of the runs below; survivors copied
-//       to their final ascending positions (from shared memory, or from the
-//       staging regions through a block scan of the chunk counts); per-segment
-//       counts and stage adaptation (Algorithm 1, Adapt_Stages) by the thread
-//       whose report completes the segment
+//       to their final ascending positions (from the ordered list, or from the
+//       staging regions through a block scan of the chunk counts) and zeroed in
+//       the residual; per-segment counts and stage adaptation (Algorithm 1,
+//       Adapt_Stages) by the thread whose report completes the segment
 //
 // Reductions are deterministic and independent of the grid: per-lane sequential
 // accumulation in a fixed order, a fixed shuffle tree per chunk, and a fixed-order
