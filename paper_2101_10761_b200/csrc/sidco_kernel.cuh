@@ -1508,7 +1508,7 @@ __global__ void __launch_bounds__(kThreads, 1) sidco_persistent_kernel(const __g
                     if (!SIDCO_IN_RANGE(A, hi - 1, A.d) || !SIDCO_IN_RANGE(A, lo, A.d) || !SIDCO_IN_RANGE(A, c, A.C)) { cur = nxt; continue; }
                     const unsigned valid = load_chunk(A.residual, lo, hi, wb, vec_ok, true, v);
                     // Stage 2 is the last stage of a two-stage segment: nothing reads its exceedances again except
-                    // the final selection, which can work from slot flags (as after P1 for one stage).
+                    // the final selection, which can work from the noted candidate slots (as after P1 for one stage).
                     const float tau2 = sv.M_eff == 2 ? spec_tau(cur.seg) : -1.0f;
                     // (without one from the previous call: by an estimate from the chunk itself, below)
                     const bool sc_chunk = sc_on && sv.M_eff == 2 && !(tau2 > 0.0f) && lo == wb && hi == wb + kChunk;
